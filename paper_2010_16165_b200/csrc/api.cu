@@ -1,0 +1,973 @@
+// C-ABI entry points and the host-side fused-graph builder.
+//
+// fp_fuse walks the node list, recognises conv-BN-(ReLU) chains and residual blocks, and
+// emits a list of fused operators: convolutions whose epilogue carries the folded BN shift,
+// the shortcut operand and the ReLU, max pools, and one head (average pool + FC).  Where a
+// block is flagged aggressive the paper's rewriting (Sec. IV-B) is applied instead: identity
+// filters are stacked under conv1 along K, the shortcut's filters beside conv2 along C, and
+// no residual operand remains.  fp_prune selects masks on the device and re-derives every
+// packed filter bank, activation shape and launch plan from them.
+#include "../../include/fupruner.h"
+#include "fp_internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+namespace {
+
+thread_local std::string g_err;
+
+fp_status fail(fp_status st, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return st;
+}
+
+#define CK(call)                                                                                        \
+    do {                                                                                                \
+        cudaError_t e_ = (call);                                                                        \
+        if (e_ != cudaSuccess)                                                                          \
+            return fail(e_ == cudaErrorMemoryAllocation ? FP_ERR_NOMEM : FP_ERR_CUDA, "%s: %s (%s:%d)", \
+                        #call, cudaGetErrorString(e_), __FILE__, __LINE__);                             \
+    } while (0)
+
+#define TRY(expr)                          \
+    do {                                   \
+        fp_status s_ = (expr);             \
+        if (s_ != FP_OK) return s_;        \
+    } while (0)
+
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+struct Tensor {
+    int C_full = 0;            // channels before pruning
+    int C = 0;                 // channels stored (kept)
+    int C_pad = 0;             // storage width, multiple of 16
+    int H = 0, W = 0;
+    std::vector<int> keep;     // stored channel j holds original channel keep[j]
+    void* d = nullptr;
+    size_t bytes = 0;
+    int producer = -1;         // index into ops, -1 = network input
+};
+
+struct FConv {
+    int conv_index = -1;       // number among the description's FP_CONV nodes
+    int src = -1, out = -1;    // tensor ids
+    int K = 0, C = 0, R = 0, S = 0, stride = 1, pad = 0;   // fused, unpruned geometry
+    int n_orig = 0;            // filter count of the original operator (Algorithm 1's m)
+    int role = 0;              // 0 plain, 1 aggressive conv1 (identity filters stacked), 2 aggressive conv2
+    int relu = 0;
+    int res_mode = 0, res_tid = -1, res_pad_lo = 0, res_stride = 1;
+    float* d_w32 = nullptr;    // fused fp32 filters, K x C x R x S
+    float* d_b32 = nullptr;    // fused bias, K
+    std::vector<uint8_t> mask;
+    std::vector<int32_t> rank;
+    // derived by replan()
+    int compact = 0;           // 1: pruned filters are physically removed from the output tensor
+    int K_kept = 0, K_rows = 0, K_pad = 0, C_kept = 0, C_pad = 0;
+    void* d_wp = nullptr;      // packed filters in the compute type, K_pad x R x S x C_pad
+    float* d_bp = nullptr;
+    fp::ConvArgs args;
+    fp::ConvPlanTC tc;
+};
+
+struct Pool { int src, out, R, stride, pad; };
+
+struct Op { int kind; int idx; };   // kind: 0 conv, 1 pool, 2 head, 3 input conversion
+
+struct GraphKey {
+    int batch; const void* in; const void* out; cudaStream_t st;
+    bool operator<(const GraphKey& o) const {
+        if (batch != o.batch) return batch < o.batch;
+        if (in != o.in) return in < o.in;
+        if (out != o.out) return out < o.out;
+        return st < o.st;
+    }
+};
+
+}  // namespace
+
+struct fp_handle_s {
+    std::vector<fp_node> nodes;
+    int in_C = 0, in_H = 0, in_W = 0, in_dtype = 0, compute = 0, use_graph = 0, keep_outputs = 0;
+    float eps = 1e-5f;
+    int max_batch = 0;
+    int n_desc_convs = 0;
+    std::vector<int> conv_to_fused;        // description conv number -> index into convs, -1 absorbed
+    std::vector<FConv> convs;
+    std::vector<Pool> pools;
+    std::vector<Tensor> tensors;           // tensor 0 = network input (after layout conversion)
+    std::vector<Op> ops;
+    // head
+    int head_src = -1, n_classes = 0, fc_C = 0;
+    const float* d_fcw = nullptr;          // classes x fc_C (copy of the description's FC weights)
+    const float* d_fcb = nullptr;
+    float* d_fcw_packed = nullptr;         // classes x C_pad, scaled by 1/(H*W)
+    // buffers
+    std::vector<void*> act_buffers;        // activation storage (re-planned by fp_prune)
+    std::vector<void*> pack_buffers;       // packed filters / biases / index arrays
+    std::vector<void*> fixed_buffers;      // fused fp32 filters etc. (live until fp_destroy)
+    void* d_in_stage = nullptr;            // device staging for fp_forward_host
+    float* d_logits_stage = nullptr;
+    int* d_status = nullptr;
+    double* d_scores = nullptr; int32_t* d_rank = nullptr; uint8_t* d_mask = nullptr;
+    std::map<GraphKey, cudaGraphExec_t> graphs;
+    const void* last_input = nullptr; int last_batch = 0;
+    int act_is_bf16() const { return compute != FP_COMPUTE_FP32; }
+    size_t act_elem() const { return act_is_bf16() ? 2 : 4; }
+    size_t in_elem() const { return in_dtype == FP_DTYPE_BF16 ? 2 : 4; }
+};
+
+namespace {
+
+void drop_graphs(fp_handle h) {
+    for (auto& kv : h->graphs) cudaGraphExecDestroy(kv.second);
+    h->graphs.clear();
+}
+
+void free_list(std::vector<void*>& v) {
+    for (void* p : v) cudaFree(p);
+    v.clear();
+}
+
+fp_status dev_alloc(std::vector<void*>& owner, void** out, size_t bytes) {
+    void* p = nullptr;
+    if (bytes == 0) bytes = 16;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(FP_ERR_NOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+    }
+    owner.push_back(p);
+    *out = p;
+    return FP_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// description -> fused operators
+// ---------------------------------------------------------------------------------------
+
+struct Builder {
+    fp_handle h;
+    const float* d_weights; const float* d_bn;   // the handle's own copies
+    size_t n_weights, n_bn;
+    std::vector<std::vector<int>> cons;
+    std::vector<int> node_tensor;     // node id -> tensor id (or -1)
+    std::vector<int> conv_number;     // node id -> description conv number
+    cudaStream_t st = 0;
+
+    int tensor_of(int node) const { return node < 0 ? 0 : node_tensor[node]; }
+
+    fp_status check_conv_node(int id) {
+        const fp_node& n = h->nodes[id];
+        if (n.K <= 0 || n.C <= 0 || n.R <= 0 || n.S <= 0 || n.stride <= 0 || n.pad < 0)
+            return fail(FP_ERR_DESC, "node %d: bad convolution geometry", id);
+        if (n.w_off < 0 || (size_t)n.w_off + (size_t)n.K * n.C * n.R * n.S > n_weights)
+            return fail(FP_ERR_DESC, "node %d: weights outside the weight array", id);
+        if (cons[id].size() != 1 || h->nodes[cons[id][0]].op != FP_BN)
+            return fail(FP_ERR_DESC, "node %d: a convolution must feed exactly one batch norm", id);
+        const fp_node& b = h->nodes[cons[id][0]];
+        if (b.K != n.K)
+            return fail(FP_ERR_SHAPE, "node %d: batch norm has %d channels, convolution %d", cons[id][0], b.K, n.K);
+        if (b.bn_off < 0 || (size_t)b.bn_off + 4 * (size_t)b.K > n_bn)
+            return fail(FP_ERR_DESC, "node %d: BN parameters outside the BN array", cons[id][0]);
+        return FP_OK;
+    }
+
+    // New fused conv from description node `conv_id`: a zeroed (K+extra_K) x (C+extra_C) bank with the
+    // node's BN-folded filters in rows [0,K), columns [0,C) and the folded shift in bias [0,K).
+    fp_status emit_conv(int conv_id, int src_tid, int relu, int extra_C, int* out_index) {
+        TRY(check_conv_node(conv_id));
+        const fp_node& n = h->nodes[conv_id];
+        const Tensor src = h->tensors[src_tid];
+        if (src.C_full != n.C + extra_C)
+            return fail(FP_ERR_SHAPE, "node %d: convolution expects %d input channels, producer has %d", conv_id,
+                        n.C + extra_C, src.C_full);
+        if (src.H + 2 * n.pad < n.R || src.W + 2 * n.pad < n.S)
+            return fail(FP_ERR_SHAPE, "node %d: window larger than the padded input", conv_id);
+        FConv f;
+        f.conv_index = conv_number[conv_id];
+        f.src = src_tid;
+        f.K = n.K; f.C = n.C + extra_C; f.R = n.R; f.S = n.S; f.stride = n.stride; f.pad = n.pad;
+        f.n_orig = n.K; f.relu = relu;
+        const size_t cnt = (size_t)f.K * f.C * f.R * f.S;
+        TRY(dev_alloc(h->fixed_buffers, (void**)&f.d_w32, cnt * sizeof(float)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&f.d_b32, (size_t)f.K * sizeof(float)));
+        CK(cudaMemsetAsync(f.d_w32, 0, cnt * sizeof(float), st));
+        CK(cudaMemsetAsync(f.d_b32, 0, (size_t)f.K * sizeof(float), st));
+        const fp_node& b = h->nodes[cons[conv_id][0]];
+        fp::launch_fold_weights(d_weights + n.w_off, d_bn + b.bn_off, n.K, n.C, n.R, n.S, h->eps, f.d_w32, f.C, f.R,
+                                f.S, 0, 0, 0, 0, st);
+        fp::launch_fold_bias(d_bn + b.bn_off, n.K, h->eps, f.d_b32, 0, 0, st);
+        Tensor t;
+        t.C_full = f.K;
+        t.H = (src.H + 2 * f.pad - f.R) / f.stride + 1;
+        t.W = (src.W + 2 * f.pad - f.S) / f.stride + 1;
+        t.producer = (int)h->ops.size();
+        h->tensors.push_back(t);
+        f.out = (int)h->tensors.size() - 1;
+        h->convs.push_back(f);
+        h->conv_to_fused[f.conv_index] = (int)h->convs.size() - 1;
+        h->ops.push_back({0, (int)h->convs.size() - 1});
+        *out_index = (int)h->convs.size() - 1;
+        return FP_OK;
+    }
+
+    bool is_relu_output(int tid) const {
+        const int px = h->tensors[tid].producer;
+        if (px < 0) return false;
+        if (h->ops[px].kind == 0) return h->convs[h->ops[px].idx].relu != 0;
+        if (h->ops[px].kind == 1) return is_relu_output(h->pools[h->ops[px].idx].src);   // max of non-negatives
+        return false;
+    }
+
+    fp_status handle_add(int id) {
+        const fp_node& n = h->nodes[id];
+        if (cons[id].size() != 1 || h->nodes[cons[id][0]].op != FP_RELU)
+            return fail(FP_ERR_DESC, "node %d: an add must feed exactly one ReLU", id);
+        const int relu_id = cons[id][0];
+        if (n.in0 < 0 || h->nodes[n.in0].op != FP_BN || h->nodes[n.in0].in0 < 0 ||
+            h->nodes[h->nodes[n.in0].in0].op != FP_CONV)
+            return fail(FP_ERR_DESC, "node %d: first add operand must be the batch norm of a convolution", id);
+        const int conv2_id = h->nodes[n.in0].in0;
+        const fp_node& c2 = h->nodes[conv2_id];
+        int mode;   // 0 identity tensor, 1 subsample + zero-channel pad, 2 projection
+        int x_node, proj_id = -1;
+        const fp_node* sc = n.in1 >= 0 ? &h->nodes[n.in1] : nullptr;
+        if (n.in1 < 0 || node_tensor[n.in1] >= 0) { mode = 0; x_node = n.in1; }
+        else if (sc->op == FP_SHORTCUT_A) { mode = 1; x_node = sc->in0; }
+        else if (sc->op == FP_BN && sc->in0 >= 0 && h->nodes[sc->in0].op == FP_CONV) {
+            mode = 2; proj_id = sc->in0; x_node = h->nodes[proj_id].in0;
+        } else return fail(FP_ERR_DESC, "node %d: unsupported shortcut operand", id);
+        const int x_tid = tensor_of(x_node);
+        const int h_tid = tensor_of(c2.in0);
+        if (x_tid < 0 || h_tid < 0) return fail(FP_ERR_DESC, "node %d: operands are not materialised tensors", id);
+        int ci;
+        if (!n.aggressive) {
+            int res_mode = 1, res_tid = x_tid, pad_lo = 0, rstride = 1;
+            if (mode == 1) { res_mode = 2; pad_lo = sc->pad_lo; rstride = sc->stride; }
+            if (mode == 2) {
+                int pi;
+                TRY(emit_conv(proj_id, x_tid, 0, 0, &pi));
+                res_tid = h->convs[pi].out;
+            }
+            TRY(emit_conv(conv2_id, h_tid, 1, 0, &ci));
+            FConv& f = h->convs[ci];
+            const Tensor& o = h->tensors[f.out];
+            const Tensor& r = h->tensors[res_tid];
+            if (res_mode == 1) {
+                if (r.C_full != f.K || r.H != o.H || r.W != o.W)
+                    return fail(FP_ERR_SHAPE, "node %d: add operands differ in shape", id);
+            } else {
+                if (rstride <= 0 || (r.H + rstride - 1) / rstride != o.H || (r.W + rstride - 1) / rstride != o.W ||
+                    pad_lo < 0 || pad_lo + r.C_full > f.K || sc->K != f.K || sc->C != r.C_full)
+                    return fail(FP_ERR_SHAPE, "node %d: shortcut does not match the main branch", id);
+            }
+            f.res_mode = res_mode; f.res_tid = res_tid; f.res_pad_lo = pad_lo; f.res_stride = rstride;
+        } else {
+            // ---- aggressive fusion (Sec. IV-B): conv1'' = [W1' ; I], conv2'' = [W2' | S_w], no add ----
+            const int p1 = h->tensors[h_tid].producer;
+            if (p1 < 0 || h->ops[p1].kind != 0)
+                return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion needs a two-convolution block", id);
+            const int f1i = h->ops[p1].idx;
+            const FConv f1c = h->convs[f1i];
+            if (f1c.src != x_tid || !f1c.relu || f1c.res_mode != 0 || f1c.role != 0 || f1c.R != 3 || f1c.S != 3 ||
+                f1c.pad != 1 || c2.R != 3 || c2.S != 3 || c2.stride != 1 || c2.pad != 1)
+                return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion supports 3x3 two-convolution blocks only", id);
+            // the pass-through channels go through conv1's ReLU: the block input must be non-negative
+            if (!is_relu_output(x_tid))
+                return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion needs a block input that is a ReLU output", id);
+            if (mode == 1 && sc->stride != f1c.stride)
+                return fail(FP_ERR_SHAPE, "node %d: shortcut stride differs from conv1", id);
+            if (mode == 2) {
+                TRY(check_conv_node(proj_id));
+                const fp_node& pr = h->nodes[proj_id];
+                if (pr.R != 1 || pr.S != 1 || pr.pad != 0 || pr.stride != f1c.stride || pr.C != f1c.C)
+                    return fail(FP_ERR_UNSUPPORTED, "node %d: projection shortcut must be 1x1 with conv1's stride", id);
+            }
+            const int C = f1c.C, K1 = f1c.K;
+            {   // widen conv1: C extra identity filters (the auxiliary convolution), zero shift for them
+                float *nw, *nb;
+                const size_t cnt = (size_t)(K1 + C) * C * 9;
+                TRY(dev_alloc(h->fixed_buffers, (void**)&nw, cnt * sizeof(float)));
+                TRY(dev_alloc(h->fixed_buffers, (void**)&nb, (size_t)(K1 + C) * sizeof(float)));
+                CK(cudaMemsetAsync(nw, 0, cnt * sizeof(float), st));
+                CK(cudaMemsetAsync(nb, 0, (size_t)(K1 + C) * sizeof(float), st));
+                CK(cudaMemcpyAsync(nw, f1c.d_w32, (size_t)K1 * C * 9 * sizeof(float), cudaMemcpyDeviceToDevice, st));
+                CK(cudaMemcpyAsync(nb, f1c.d_b32, (size_t)K1 * sizeof(float), cudaMemcpyDeviceToDevice, st));
+                fp::launch_identity_filters(nw, C, 3, 3, K1, 0, C, C, 0, st);
+                FConv& f1 = h->convs[f1i];
+                f1.d_w32 = nw; f1.d_b32 = nb; f1.K = K1 + C; f1.role = 1;
+                h->tensors[f1.out].C_full = K1 + C;
+            }
+            TRY(emit_conv(conv2_id, h_tid, 1, C, &ci));     // K2 x (K1 + C), conv2 folded into columns [0,K1)
+            FConv& f = h->convs[ci];
+            f.role = 2;
+            if (mode == 0) {
+                if (f.K != C) return fail(FP_ERR_SHAPE, "node %d: identity shortcut needs K2 == C", id);
+                fp::launch_identity_filters(f.d_w32, f.C, 3, 3, 0, K1, f.K, C, 0, st);
+            } else if (mode == 1) {
+                if (sc->pad_lo < 0 || sc->pad_lo + C > f.K || sc->K != f.K || sc->C != C)
+                    return fail(FP_ERR_SHAPE, "node %d: shortcut does not match the main branch", id);
+                fp::launch_identity_filters(f.d_w32, f.C, 3, 3, 0, K1, f.K, C, sc->pad_lo, st);
+            } else {
+                const fp_node& pr = h->nodes[proj_id];
+                if (pr.K != f.K) return fail(FP_ERR_SHAPE, "node %d: projection has %d filters, conv2 %d", id, pr.K, f.K);
+                const fp_node& pb = h->nodes[cons[proj_id][0]];
+                // the 1x1 projection padded with zeros to 3x3 (centre tap), folded with its own BN
+                fp::launch_fold_weights(d_weights + pr.w_off, d_bn + pb.bn_off, pr.K, pr.C, 1, 1, h->eps, f.d_w32, f.C, 3, 3,
+                                        0, K1, 1, 1, st);
+                fp::launch_fold_bias(d_bn + pb.bn_off, pr.K, h->eps, f.d_b32, 0, 1, st);
+                h->conv_to_fused[conv_number[proj_id]] = -1;
+            }
+            const Tensor& o = h->tensors[f.out];
+            const Tensor& xin = h->tensors[x_tid];
+            if ((xin.H + f1c.stride - 1) / f1c.stride != o.H || (xin.W + f1c.stride - 1) / f1c.stride != o.W)
+                return fail(FP_ERR_SHAPE, "node %d: shortcut spatial size mismatch", id);
+        }
+        node_tensor[relu_id] = h->convs[ci].out;
+        return FP_OK;
+    }
+
+    fp_status run() {
+        const int nn = (int)h->nodes.size();
+        cons.assign(nn, {});
+        node_tensor.assign(nn, -1);
+        conv_number.assign(nn, -1);
+        int nc = 0;
+        for (int i = 0; i < nn; ++i) {
+            const fp_node& n = h->nodes[i];
+            if (n.op < FP_CONV || n.op > FP_FC) return fail(FP_ERR_DESC, "node %d: unknown op %d", i, n.op);
+            if (n.in0 < -1 || n.in0 >= i) return fail(FP_ERR_DESC, "node %d: in0 must name an earlier node", i);
+            if (n.op == FP_ADD && (n.in1 < -1 || n.in1 >= i)) return fail(FP_ERR_DESC, "node %d: in1 must name an earlier node", i);
+            if (n.in0 >= 0) cons[n.in0].push_back(i);
+            if (n.op == FP_ADD && n.in1 >= 0) cons[n.in1].push_back(i);
+            if (n.op == FP_CONV) conv_number[i] = nc++;
+        }
+        h->n_desc_convs = nc;
+        h->conv_to_fused.assign(nc, -1);
+        Tensor in;
+        in.C_full = h->in_C; in.H = h->in_H; in.W = h->in_W; in.producer = -1;
+        h->tensors.push_back(in);
+        h->ops.push_back({3, 0});
+        for (int i = 0; i < nn; ++i) {
+            const fp_node& n = h->nodes[i];
+            switch (n.op) {
+                case FP_CONV: {
+                    TRY(check_conv_node(i));
+                    const int bn_id = cons[i][0];
+                    const std::vector<int>& nxt = cons[bn_id];
+                    if (nxt.size() == 1 && h->nodes[nxt[0]].op == FP_ADD) break;   // emitted with its add
+                    const int src = tensor_of(n.in0);
+                    if (src < 0) return fail(FP_ERR_DESC, "node %d: input is not a materialised tensor", i);
+                    int ci;
+                    if (nxt.size() == 1 && h->nodes[nxt[0]].op == FP_RELU) {
+                        TRY(emit_conv(i, src, 1, 0, &ci));
+                        node_tensor[nxt[0]] = h->convs[ci].out;
+                    } else {
+                        TRY(emit_conv(i, src, 0, 0, &ci));
+                        node_tensor[bn_id] = h->convs[ci].out;
+                    }
+                    break;
+                }
+                case FP_ADD: TRY(handle_add(i)); break;
+                case FP_MAXPOOL: {
+                    const int src = tensor_of(n.in0);
+                    if (src < 0) return fail(FP_ERR_DESC, "node %d: input is not a materialised tensor", i);
+                    const Tensor s = h->tensors[src];
+                    if (n.R <= 0 || n.stride <= 0 || n.pad < 0 || n.pad >= n.R || s.H + 2 * n.pad < n.R || s.W + 2 * n.pad < n.R)
+                        return fail(FP_ERR_DESC, "node %d: bad pooling geometry", i);
+                    Tensor t;
+                    t.C_full = s.C_full;
+                    t.H = (s.H + 2 * n.pad - n.R) / n.stride + 1;
+                    t.W = (s.W + 2 * n.pad - n.R) / n.stride + 1;
+                    t.producer = (int)h->ops.size();
+                    h->tensors.push_back(t);
+                    h->pools.push_back({src, (int)h->tensors.size() - 1, n.R, n.stride, n.pad});
+                    h->ops.push_back({1, (int)h->pools.size() - 1});
+                    node_tensor[i] = (int)h->tensors.size() - 1;
+                    break;
+                }
+                case FP_GAVGPOOL: {
+                    const int src = tensor_of(n.in0);
+                    if (src < 0) return fail(FP_ERR_DESC, "node %d: input is not a materialised tensor", i);
+                    if (cons[i].size() != 1 || h->nodes[cons[i][0]].op != FP_FC)
+                        return fail(FP_ERR_DESC, "node %d: global average pool must feed the FC layer", i);
+                    const fp_node& f = h->nodes[cons[i][0]];
+                    if (f.C != h->tensors[src].C_full || f.K <= 0)
+                        return fail(FP_ERR_SHAPE, "node %d: FC expects %d inputs, producer has %d", cons[i][0], f.C, h->tensors[src].C_full);
+                    if (f.w_off < 0 || (size_t)f.w_off + (size_t)f.K * f.C > n_weights ||
+                        (f.b_off >= 0 && (size_t)f.b_off + f.K > n_weights))
+                        return fail(FP_ERR_DESC, "node %d: FC weights outside the weight array", cons[i][0]);
+                    if (h->head_src >= 0) return fail(FP_ERR_DESC, "node %d: more than one head", i);
+                    h->head_src = src; h->n_classes = f.K; h->fc_C = f.C;
+                    h->d_fcw = d_weights + f.w_off;
+                    h->d_fcb = f.b_off >= 0 ? d_weights + f.b_off : nullptr;
+                    h->ops.push_back({2, 0});
+                    break;
+                }
+                default: break;   // BN, ReLU, shortcut, FC are consumed by the patterns above
+            }
+        }
+        if (h->head_src < 0) return fail(FP_ERR_DESC, "description has no global-average-pool + FC head");
+        if (h->ops.back().kind != 2) return fail(FP_ERR_DESC, "the head must be the last operator");
+        return FP_OK;
+    }
+};
+
+// ---------------------------------------------------------------------------------------
+// masks -> shapes, packed filters, activation memory, launch plans
+// ---------------------------------------------------------------------------------------
+
+struct Use { int op; int how; };   // how: 0 main input, 1 residual operand
+
+std::vector<std::vector<Use>> tensor_uses(fp_handle h) {
+    std::vector<std::vector<Use>> u(h->tensors.size());
+    for (int i = 0; i < (int)h->ops.size(); ++i) {
+        const Op& op = h->ops[i];
+        if (op.kind == 0) {
+            const FConv& f = h->convs[op.idx];
+            u[f.src].push_back({i, 0});
+            if (f.res_mode) u[f.res_tid].push_back({i, 1});
+        } else if (op.kind == 1) {
+            u[h->pools[op.idx].src].push_back({i, 0});
+        } else if (op.kind == 2) {
+            u[h->head_src].push_back({i, 0});
+        }
+    }
+    return u;
+}
+
+// Channels of a tensor can be physically dropped iff every reader is a convolution's main input
+// (or a pool whose own result is compactable).  Residual streams keep their full width.
+bool compactable(fp_handle h, const std::vector<std::vector<Use>>& uses, int tid) {
+    if (uses[tid].empty()) return false;
+    for (const Use& u : uses[tid]) {
+        if (u.how == 1) return false;
+        const Op& op = h->ops[u.op];
+        if (op.kind == 0) continue;
+        if (op.kind == 1) { if (!compactable(h, uses, h->pools[op.idx].out)) return false; continue; }
+        return false;
+    }
+    return true;
+}
+
+fp_status upload_i32(fp_handle h, const std::vector<int32_t>& v, int32_t** out) {
+    TRY(dev_alloc(h->pack_buffers, (void**)out, v.size() * sizeof(int32_t)));
+    CK(cudaMemcpy(*out, v.data(), v.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    return FP_OK;
+}
+
+fp_status replan(fp_handle h) {
+    drop_graphs(h);
+    CK(cudaDeviceSynchronize());
+    free_list(h->act_buffers);
+    free_list(h->pack_buffers);
+    const auto uses = tensor_uses(h);
+    const int bf16 = h->act_is_bf16();
+    cudaStream_t st = 0;
+
+    // --- shapes in execution order ---
+    {
+        Tensor& t = h->tensors[0];
+        t.C = t.C_full; t.C_pad = round_up(t.C, 16);
+        t.keep.resize(t.C);
+        for (int c = 0; c < t.C; ++c) t.keep[c] = c;
+    }
+    for (const Op& op : h->ops) {
+        if (op.kind == 0) {
+            FConv& f = h->convs[op.idx];
+            const Tensor& src = h->tensors[f.src];
+            Tensor& out = h->tensors[f.out];
+            std::vector<int> kept;
+            for (int k = 0; k < f.K; ++k) if (f.mask[k]) kept.push_back(k);
+            if (kept.empty()) return fail(FP_ERR_EMPTY_LAYER, "convolution %d keeps no filter", f.conv_index);
+            f.K_kept = (int)kept.size();
+            f.compact = (f.res_mode == 0 && compactable(h, uses, f.out)) ? 1 : 0;
+            f.C_kept = src.C; f.C_pad = src.C_pad;
+            std::vector<int32_t> row_src, chan_src(f.C_pad, -1);
+            if (f.compact) {
+                f.K_rows = f.K_kept;
+                out.keep = kept;
+                for (int k : kept) row_src.push_back(k);
+            } else {
+                f.K_rows = f.K;
+                out.keep.resize(f.K);
+                for (int k = 0; k < f.K; ++k) { out.keep[k] = k; row_src.push_back(f.mask[k] ? k : -1); }
+            }
+            f.K_pad = round_up(f.K_rows, 16);
+            row_src.resize(f.K_pad, -1);
+            for (int c = 0; c < src.C; ++c) chan_src[c] = src.keep[c];
+            out.C = f.K_rows; out.C_pad = f.K_pad;
+            // pack filters and bias
+            int32_t *d_row, *d_chan;
+            TRY(upload_i32(h, row_src, &d_row));
+            TRY(upload_i32(h, chan_src, &d_chan));
+            const size_t cnt = (size_t)f.K_pad * f.R * f.S * f.C_pad;
+            TRY(dev_alloc(h->pack_buffers, &f.d_wp, cnt * h->act_elem()));
+            TRY(dev_alloc(h->pack_buffers, (void**)&f.d_bp, (size_t)f.K_pad * sizeof(float)));
+            fp::launch_repack(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad, 1.0f,
+                              bf16 ? (__nv_bfloat16*)f.d_wp : nullptr, bf16 ? nullptr : (float*)f.d_wp, st);
+            fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);
+        } else if (op.kind == 1) {
+            const Pool& p = h->pools[op.idx];
+            const Tensor& src = h->tensors[p.src];
+            Tensor& out = h->tensors[p.out];
+            out.C = src.C; out.C_pad = src.C_pad; out.keep = src.keep;
+        } else if (op.kind == 2) {
+            const Tensor& src = h->tensors[h->head_src];
+            std::vector<int32_t> row_src(h->n_classes), chan_src(src.C_pad, -1);
+            for (int k = 0; k < h->n_classes; ++k) row_src[k] = k;
+            for (int c = 0; c < src.C; ++c) chan_src[c] = src.keep[c];
+            int32_t *d_row, *d_chan;
+            TRY(upload_i32(h, row_src, &d_row));
+            TRY(upload_i32(h, chan_src, &d_chan));
+            TRY(dev_alloc(h->pack_buffers, (void**)&h->d_fcw_packed, (size_t)h->n_classes * src.C_pad * sizeof(float)));
+            // the average's 1/(H*W) is folded into the FC weights
+            fp::launch_repack(h->d_fcw, h->fc_C, 1, d_row, h->n_classes, d_chan, src.C_pad, 1.0f / (float)(src.H * src.W),
+                              nullptr, h->d_fcw_packed, st);
+        }
+    }
+    CK(cudaGetLastError());
+
+    // --- activation memory: buffers are reused once their last reader has run ---
+    {
+        const int nt = (int)h->tensors.size();
+        std::vector<int> last_use(nt, -1);
+        for (int t = 0; t < nt; ++t)
+            for (const Use& u : uses[t]) last_use[t] = std::max(last_use[t], u.op);
+        struct Buf { void* p; size_t bytes; int free_after; };
+        std::vector<Buf> bufs;
+        for (int i = 0; i < (int)h->ops.size(); ++i) {
+            const Op& op = h->ops[i];
+            int tid = -1;
+            if (op.kind == 0) tid = h->convs[op.idx].out;
+            else if (op.kind == 1) tid = h->pools[op.idx].out;
+            else if (op.kind == 3) tid = 0;
+            if (tid < 0) continue;
+            Tensor& t = h->tensors[tid];
+            t.bytes = (size_t)h->max_batch * t.H * t.W * t.C_pad * h->act_elem();
+            int best = -1;
+            if (!h->keep_outputs)
+                for (int b = 0; b < (int)bufs.size(); ++b)
+                    if (bufs[b].free_after < i && bufs[b].bytes >= t.bytes && (best < 0 || bufs[b].bytes < bufs[best].bytes)) best = b;
+            if (best < 0) {
+                void* p;
+                TRY(dev_alloc(h->act_buffers, &p, t.bytes));
+                CK(cudaMemsetAsync(p, 0, t.bytes, st));
+                bufs.push_back({p, t.bytes, 0});
+                best = (int)bufs.size() - 1;
+            }
+            t.d = bufs[best].p;
+            bufs[best].free_after = std::max(last_use[tid], i);
+        }
+    }
+
+    // --- launch arguments and tensor-core plans ---
+    for (FConv& f : h->convs) {
+        const Tensor& src = h->tensors[f.src];
+        const Tensor& out = h->tensors[f.out];
+        fp::ConvArgs& a = f.args;
+        memset(&a, 0, sizeof(a));
+        a.x = src.d; a.y = out.d; a.w = f.d_wp; a.bias = f.d_bp;
+        a.N = h->max_batch; a.H = src.H; a.W = src.W; a.C_pad = f.C_pad; a.P = out.H; a.Q = out.W;
+        a.K_pad = f.K_pad; a.R = f.R; a.S = f.S; a.stride = f.stride; a.pad = f.pad; a.relu = f.relu;
+        a.res_mode = f.res_mode;
+        if (f.res_mode) {
+            const Tensor& r = h->tensors[f.res_tid];
+            a.res = r.d; a.res_H = r.H; a.res_W = r.W; a.res_C_pad = r.C_pad; a.res_C = r.C;
+            a.res_pad_lo = f.res_pad_lo; a.res_stride = f.res_stride;
+        }
+        f.tc.valid = 0;
+        if (h->compute == FP_COMPUTE_BF16_TC) {
+            char msg[256];
+            if (fp::plan_conv_tc(a, &f.tc, msg, sizeof(msg)) != 0)
+                return fail(FP_ERR_UNSUPPORTED, "convolution %d: %s", f.conv_index, msg);
+        }
+    }
+    CK(cudaDeviceSynchronize());
+    return FP_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// execution
+// ---------------------------------------------------------------------------------------
+
+void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
+    const int bf16 = h->act_is_bf16();
+    if (op.kind == 3) {
+        const Tensor& t = h->tensors[0];
+        fp::launch_input_to_nhwc(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, st);
+    } else if (op.kind == 0) {
+        FConv& f = h->convs[op.idx];
+        fp::ConvArgs a = f.args;
+        a.N = batch;
+        if (h->compute == FP_COMPUTE_BF16_TC) fp::launch_conv_tc(f.tc, a, h->d_status, st);
+        else fp::launch_conv_simt(a, bf16, st);
+    } else if (op.kind == 1) {
+        const Pool& p = h->pools[op.idx];
+        const Tensor& s = h->tensors[p.src];
+        const Tensor& o = h->tensors[p.out];
+        fp::launch_maxpool(s.d, o.d, bf16, batch, s.H, s.W, s.C_pad, o.H, o.W, p.R, p.stride, p.pad, st);
+    } else {
+        const Tensor& s = h->tensors[h->head_src];
+        fp::launch_head(s.d, bf16, batch, s.H * s.W, s.C_pad, h->d_fcw_packed, h->d_fcb, h->n_classes, d_logits, st);
+    }
+}
+
+void launch_all(fp_handle h, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
+    for (const Op& op : h->ops) launch_op(h, op, d_input, batch, d_logits, st);
+}
+
+fp_status all_ones_masks(fp_handle h) {
+    for (FConv& f : h->convs) {
+        f.mask.assign(f.K, 1);
+        f.rank.assign(f.K, 0);
+        for (int k = 0; k < f.K; ++k) f.rank[k] = k;
+    }
+    return FP_OK;
+}
+
+}  // namespace
+
+// =========================================================================================
+// C ABI
+// =========================================================================================
+
+extern "C" const char* fp_last_error(void) { return g_err.c_str(); }
+
+extern "C" fp_status fp_destroy(fp_handle h) {
+    if (!h) return FP_OK;
+    cudaDeviceSynchronize();
+    drop_graphs(h);
+    free_list(h->act_buffers);
+    free_list(h->pack_buffers);
+    free_list(h->fixed_buffers);
+    delete h;
+    return FP_OK;
+}
+
+extern "C" fp_status fp_fuse(const fp_model_desc* desc, const float* d_weights, size_t n_weights, const float* d_bn,
+                             size_t n_bn, int32_t max_batch, fp_handle* out) {
+    if (!desc || !out || !d_weights || !desc->nodes) return fail(FP_ERR_ARG, "fp_fuse: NULL argument");
+    if (!d_bn && n_bn) return fail(FP_ERR_ARG, "fp_fuse: NULL BN array");
+    if (desc->n_nodes <= 0 || max_batch <= 0) return fail(FP_ERR_ARG, "fp_fuse: n_nodes and max_batch must be positive");
+    if (desc->in_C <= 0 || desc->in_H <= 0 || desc->in_W <= 0) return fail(FP_ERR_ARG, "fp_fuse: bad input shape");
+    if (desc->in_dtype != FP_DTYPE_F32 && desc->in_dtype != FP_DTYPE_BF16) return fail(FP_ERR_ARG, "fp_fuse: bad in_dtype");
+    if (desc->compute < 0 || desc->compute > 2) return fail(FP_ERR_ARG, "fp_fuse: bad compute mode");
+    if (!(desc->bn_eps > 0.0f) || !std::isfinite(desc->bn_eps)) return fail(FP_ERR_ARG, "fp_fuse: bn_eps must be positive");
+    int dev = 0;
+    cudaDeviceProp prop;
+    CK(cudaGetDevice(&dev));
+    CK(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return fail(FP_ERR_UNSUPPORTED, "fp_fuse: needs a compute-capability 10.x GPU (found %d.%d)", prop.major, prop.minor);
+
+    fp_handle h = new fp_handle_s();
+    h->nodes.assign(desc->nodes, desc->nodes + desc->n_nodes);
+    h->in_C = desc->in_C; h->in_H = desc->in_H; h->in_W = desc->in_W;
+    h->in_dtype = desc->in_dtype; h->compute = desc->compute; h->use_graph = desc->use_graph;
+    h->keep_outputs = desc->keep_outputs;
+    h->eps = desc->bn_eps; h->max_batch = max_batch;
+    fp_status s = FP_OK;
+    auto body = [&]() -> fp_status {
+        // own copies of the parameters, checked for NaN/Inf on the device
+        float *wcopy, *bcopy;
+        int* d_bad;
+        TRY(dev_alloc(h->fixed_buffers, (void**)&wcopy, n_weights * sizeof(float)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&bcopy, n_bn * sizeof(float)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&d_bad, sizeof(int)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_status, sizeof(int)));
+        CK(cudaMemcpy(wcopy, d_weights, n_weights * sizeof(float), cudaMemcpyDeviceToDevice));
+        if (n_bn) CK(cudaMemcpy(bcopy, d_bn, n_bn * sizeof(float), cudaMemcpyDeviceToDevice));
+        CK(cudaMemset(d_bad, 0, sizeof(int)));
+        CK(cudaMemset(h->d_status, 0, sizeof(int)));
+        fp::launch_count_nonfinite(wcopy, n_weights, d_bad, 0);
+        fp::launch_count_nonfinite(bcopy, n_bn, d_bad, 0);
+        int bad = 0;
+        CK(cudaMemcpy(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost));
+        if (bad) return fail(FP_ERR_NONFINITE, "fp_fuse: %d non-finite values in the weights or BN statistics", bad);
+        Builder b;
+        b.h = h; b.d_weights = wcopy; b.d_bn = bcopy; b.n_weights = n_weights; b.n_bn = n_bn;
+        TRY(b.run());
+        CK(cudaGetLastError());
+        int max_K = 1;
+        for (const FConv& f : h->convs) max_K = std::max(max_K, f.K);
+        if ((size_t)max_K * sizeof(double) > 48 * 1024) return fail(FP_ERR_UNSUPPORTED, "fp_fuse: more than 6144 filters in one convolution");
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_scores, (size_t)max_K * sizeof(double)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_rank, (size_t)max_K * sizeof(int32_t)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_mask, (size_t)max_K));
+        TRY(dev_alloc(h->fixed_buffers, &h->d_in_stage, (size_t)max_batch * h->in_C * h->in_H * h->in_W * h->in_elem()));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_logits_stage, (size_t)max_batch * h->n_classes * sizeof(float)));
+        all_ones_masks(h);
+        TRY(replan(h));
+        return FP_OK;
+    };
+    s = body();
+    if (s != FP_OK) {
+        std::string keep = g_err;
+        fp_destroy(h);
+        g_err = keep;
+        return s;
+    }
+    *out = h;
+    return FP_OK;
+}
+
+static fp_status score_conv(fp_handle h, const FConv& f, int norm) {
+    fp::launch_score_filters(f.d_w32, f.K, f.C * f.R * f.S, norm, h->d_scores, 0);
+    CK(cudaGetLastError());
+    return FP_OK;
+}
+
+extern "C" fp_status fp_score(fp_handle h, int32_t conv_index, int32_t norm, double* h_scores) {
+    if (!h || !h_scores) return fail(FP_ERR_ARG, "fp_score: NULL argument");
+    if (norm != FP_NORM_L1 && norm != FP_NORM_L2) return fail(FP_ERR_ARG, "fp_score: bad norm");
+    if (conv_index < 0 || conv_index >= h->n_desc_convs || h->conv_to_fused[conv_index] < 0)
+        return fail(FP_ERR_ARG, "fp_score: convolution %d does not exist in the fused graph", conv_index);
+    const FConv& f = h->convs[h->conv_to_fused[conv_index]];
+    TRY(score_conv(h, f, norm));
+    CK(cudaMemcpy(h_scores, h->d_scores, (size_t)f.K * sizeof(double), cudaMemcpyDeviceToHost));
+    return FP_OK;
+}
+
+extern "C" fp_status fp_prune(fp_handle h, int32_t norm, const double* h_ratios, const uint8_t* const* h_masks) {
+    if (!h) return fail(FP_ERR_ARG, "fp_prune: NULL handle");
+    if (norm != FP_NORM_L1 && norm != FP_NORM_L2) return fail(FP_ERR_ARG, "fp_prune: bad norm");
+    // select every mask first (all scores are taken on the unpruned fused weights), then apply
+    std::vector<std::vector<uint8_t>> masks(h->convs.size());
+    std::vector<std::vector<int32_t>> ranks(h->convs.size());
+    for (size_t i = 0; i < h->convs.size(); ++i) {
+        const FConv& f = h->convs[i];
+        masks[i].resize(f.K);
+        ranks[i].resize(f.K);
+        TRY(score_conv(h, f, norm));
+        const uint8_t* given = h_masks ? h_masks[f.conv_index] : nullptr;
+        int q;
+        if (f.role != 0) q = f.K - f.n_orig;               // fused operator: back to its original filter count
+        else {
+            const double r = h_ratios ? h_ratios[f.conv_index] : 0.0;
+            if (!(r >= 0.0) || r > 1.0) return fail(FP_ERR_ARG, "fp_prune: ratio of convolution %d outside [0,1]", f.conv_index);
+            q = (int)std::floor(r * (double)f.K + 1e-9);
+        }
+        fp::launch_rank_mask(h->d_scores, f.K, q, h->d_rank, h->d_mask, 0);
+        CK(cudaGetLastError());
+        CK(cudaMemcpy(ranks[i].data(), h->d_rank, (size_t)f.K * sizeof(int32_t), cudaMemcpyDeviceToHost));
+        if (given) {
+            for (int k = 0; k < f.K; ++k) {
+                if (given[k] > 1) return fail(FP_ERR_ARG, "fp_prune: mask of convolution %d has a value other than 0/1", f.conv_index);
+                masks[i][k] = given[k];
+            }
+        } else {
+            CK(cudaMemcpy(masks[i].data(), h->d_mask, (size_t)f.K, cudaMemcpyDeviceToHost));
+        }
+        int kept = 0;
+        for (int k = 0; k < f.K; ++k) kept += masks[i][k];
+        if (kept == 0) return fail(FP_ERR_EMPTY_LAYER, "fp_prune: convolution %d would keep no filter", f.conv_index);
+    }
+    for (size_t i = 0; i < h->convs.size(); ++i) { h->convs[i].mask = masks[i]; h->convs[i].rank = ranks[i]; }
+    return replan(h);
+}
+
+extern "C" fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch, float* d_logits, void* stream) {
+    if (!h || !d_input || !d_logits) return fail(FP_ERR_ARG, "fp_forward: NULL argument");
+    if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward: batch must be positive");
+    if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward: batch %d exceeds max_batch %d", batch, h->max_batch);
+    cudaStream_t st = (cudaStream_t)stream;
+    h->last_input = d_input; h->last_batch = batch;
+    const bool graphable = h->use_graph && st != 0 && st != cudaStreamLegacy && st != cudaStreamPerThread;
+    if (!graphable) {
+        launch_all(h, d_input, batch, d_logits, st);
+        CK(cudaGetLastError());
+        return FP_OK;
+    }
+    GraphKey key{batch, d_input, d_logits, st};
+    auto it = h->graphs.find(key);
+    if (it == h->graphs.end()) {
+        cudaStreamCaptureStatus cs;
+        CK(cudaStreamIsCapturing(st, &cs));
+        if (cs != cudaStreamCaptureStatusNone) {   // already inside someone else's capture: just record the launches
+            launch_all(h, d_input, batch, d_logits, st);
+            CK(cudaGetLastError());
+            return FP_OK;
+        }
+        cudaGraph_t g;
+        CK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+        launch_all(h, d_input, batch, d_logits, st);
+        cudaError_t e = cudaStreamEndCapture(st, &g);
+        if (e != cudaSuccess) return fail(FP_ERR_CUDA, "graph capture failed: %s", cudaGetErrorString(e));
+        cudaGraphExec_t ge;
+        e = cudaGraphInstantiate(&ge, g, 0);
+        cudaGraphDestroy(g);
+        if (e != cudaSuccess) return fail(FP_ERR_CUDA, "graph instantiate failed: %s", cudaGetErrorString(e));
+        if (h->graphs.size() >= 16) drop_graphs(h);
+        it = h->graphs.emplace(key, ge).first;
+    }
+    CK(cudaGraphLaunch(it->second, st));
+    return FP_OK;
+}
+
+extern "C" fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t batch, float* h_logits, void* stream) {
+    if (!h || !h_input || !h_logits) return fail(FP_ERR_ARG, "fp_forward_host: NULL argument");
+    if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward_host: batch must be positive");
+    if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward_host: batch %d exceeds max_batch %d", batch, h->max_batch);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t in_bytes = (size_t)batch * h->in_C * h->in_H * h->in_W * h->in_elem();
+    CK(cudaMemcpyAsync(h->d_in_stage, h_input, in_bytes, cudaMemcpyHostToDevice, st));
+    TRY(fp_forward(h, h->d_in_stage, batch, h->d_logits_stage, stream));
+    CK(cudaMemcpyAsync(h_logits, h->d_logits_stage, (size_t)batch * h->n_classes * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    return FP_OK;
+}
+
+static void fill_op_info(fp_handle h, int i, fp_op_info* o) {
+    memset(o, 0, sizeof(*o));
+    const Op& op = h->ops[i];
+    const double e = (double)h->act_elem();
+    o->kind = op.kind; o->conv_index = -1;
+    if (op.kind == 0) {
+        const FConv& f = h->convs[op.idx];
+        const Tensor& s = h->tensors[f.src];
+        const Tensor& t = h->tensors[f.out];
+        o->conv_index = f.conv_index;
+        o->K = f.K_kept; o->C = f.C_kept; o->R = f.R; o->S = f.S; o->stride = f.stride; o->pad = f.pad;
+        o->K_pad = f.K_pad; o->C_pad = f.C_pad; o->H = s.H; o->W = s.W; o->P = t.H; o->Q = t.W;
+        o->res_mode = f.res_mode; o->relu = f.relu;
+        o->flops_per_image = 2.0 * t.H * t.W * (double)f.K_kept * f.C_kept * f.R * f.S;
+        double b = (double)s.H * s.W * s.C * e + (double)t.H * t.W * t.C * e;
+        if (f.res_mode == 1) b += (double)t.H * t.W * t.C * e;
+        if (f.res_mode == 2) b += (double)t.H * t.W * h->tensors[f.res_tid].C * e;
+        o->bytes_per_image = b;
+        o->bytes_fixed = (double)f.K_kept * f.C_kept * f.R * f.S * e + 4.0 * f.K_kept;
+    } else if (op.kind == 1) {
+        const Pool& p = h->pools[op.idx];
+        const Tensor& s = h->tensors[p.src];
+        const Tensor& t = h->tensors[p.out];
+        o->K = o->C = s.C; o->K_pad = o->C_pad = s.C_pad; o->R = o->S = p.R; o->stride = p.stride; o->pad = p.pad;
+        o->H = s.H; o->W = s.W; o->P = t.H; o->Q = t.W;
+        o->bytes_per_image = ((double)s.H * s.W + (double)t.H * t.W) * s.C * e;
+    } else if (op.kind == 2) {
+        const Tensor& s = h->tensors[h->head_src];
+        o->K = h->n_classes; o->C = s.C; o->K_pad = h->n_classes; o->C_pad = s.C_pad; o->H = s.H; o->W = s.W; o->P = o->Q = 1;
+        o->R = o->S = 1; o->stride = 1;
+        o->flops_per_image = 2.0 * h->n_classes * s.C + (double)s.H * s.W * s.C;
+        o->bytes_per_image = (double)s.H * s.W * s.C * e + 4.0 * h->n_classes;
+        o->bytes_fixed = 4.0 * h->n_classes * (s.C + 1);
+    } else {
+        const Tensor& t = h->tensors[0];
+        o->K = o->C = t.C; o->K_pad = o->C_pad = t.C_pad; o->H = o->P = t.H; o->W = o->Q = t.W; o->R = o->S = 1; o->stride = 1;
+        o->bytes_per_image = (double)t.H * t.W * t.C * ((double)h->in_elem() + e);
+    }
+}
+
+extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_out, size_t bytes) {
+    if (!h || !h_out) return fail(FP_ERR_ARG, "fp_query: NULL argument");
+    auto need = [&](size_t n) -> fp_status {
+        return bytes >= n ? FP_OK : fail(FP_ERR_ARG, "fp_query: output buffer too small (%zu < %zu)", bytes, n);
+    };
+    auto conv_of = [&](const FConv** f) -> fp_status {
+        if (index < 0 || index >= h->n_desc_convs) return fail(FP_ERR_ARG, "fp_query: convolution %d out of range", index);
+        *f = h->conv_to_fused[index] >= 0 ? &h->convs[h->conv_to_fused[index]] : nullptr;
+        return FP_OK;
+    };
+    const FConv* f = nullptr;
+    switch (what) {
+        case FP_Q_N_CONVS: TRY(need(4)); *(int32_t*)h_out = h->n_desc_convs; return FP_OK;
+        case FP_Q_N_CLASSES: TRY(need(4)); *(int32_t*)h_out = h->n_classes; return FP_OK;
+        case FP_Q_N_OPS: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size(); return FP_OK;
+        case FP_Q_N_LAUNCHES: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size(); return FP_OK;
+        case FP_Q_CONV_K_FUSED: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K : 0; return FP_OK;
+        case FP_Q_CONV_K_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K_kept : 0; return FP_OK;
+        case FP_Q_CONV_C_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->C_kept : 0; return FP_OK;
+        case FP_Q_MASK:
+            TRY(conv_of(&f));
+            if (!f) return fail(FP_ERR_ARG, "fp_query: convolution %d was absorbed by fusion", index);
+            TRY(need(f->K)); memcpy(h_out, f->mask.data(), f->K); return FP_OK;
+        case FP_Q_RANK:
+            TRY(conv_of(&f));
+            if (!f) return fail(FP_ERR_ARG, "fp_query: convolution %d was absorbed by fusion", index);
+            TRY(need((size_t)f->K * 4)); memcpy(h_out, f->rank.data(), (size_t)f->K * 4); return FP_OK;
+        case FP_Q_FLOPS: {
+            TRY(need(8));
+            double s = 0;
+            for (int i = 0; i < (int)h->ops.size(); ++i) { fp_op_info o; fill_op_info(h, i, &o); s += o.flops_per_image; }
+            *(double*)h_out = s; return FP_OK;
+        }
+        case FP_Q_BYTES: {
+            TRY(need(16));
+            double a = 0, b = 0;
+            for (int i = 0; i < (int)h->ops.size(); ++i) { fp_op_info o; fill_op_info(h, i, &o); a += o.bytes_per_image; b += o.bytes_fixed; }
+            ((double*)h_out)[0] = a; ((double*)h_out)[1] = b; return FP_OK;
+        }
+        case FP_Q_OP_INFO:
+            if (index < 0 || index >= (int)h->ops.size()) return fail(FP_ERR_ARG, "fp_query: operator %d out of range", index);
+            TRY(need(sizeof(fp_op_info)));
+            fill_op_info(h, index, (fp_op_info*)h_out);
+            return FP_OK;
+        case FP_Q_OP_OUTPUT: {
+            if (index < 0 || index >= (int)h->ops.size() || h->ops[index].kind == 2)
+                return fail(FP_ERR_ARG, "fp_query: operator %d has no activation output", index);
+            if (h->last_batch <= 0) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
+            const Op& op = h->ops[index];
+            const int tid = op.kind == 0 ? h->convs[op.idx].out : op.kind == 1 ? h->pools[op.idx].out : 0;
+            const Tensor& t = h->tensors[tid];
+            const size_t cnt = (size_t)h->last_batch * t.C * t.H * t.W;
+            TRY(need(cnt * sizeof(float)));
+            std::vector<int32_t> chan_dst(t.C_pad, -1);
+            for (int c = 0; c < t.C; ++c) chan_dst[c] = c;
+            float* d_tmp; int32_t* d_chan;
+            CK(cudaDeviceSynchronize());
+            CK(cudaMalloc(&d_tmp, cnt * sizeof(float)));
+            CK(cudaMalloc(&d_chan, chan_dst.size() * 4));
+            CK(cudaMemcpy(d_chan, chan_dst.data(), chan_dst.size() * 4, cudaMemcpyHostToDevice));
+            fp::launch_nhwc_to_nchw_f32(t.d, h->act_is_bf16(), d_tmp, h->last_batch, t.H, t.W, t.C_pad, d_chan, t.C, 0);
+            cudaError_t e = cudaMemcpy(h_out, d_tmp, cnt * sizeof(float), cudaMemcpyDeviceToHost);
+            cudaFree(d_tmp); cudaFree(d_chan);
+            if (e != cudaSuccess) return fail(FP_ERR_CUDA, "fp_query: copy failed: %s", cudaGetErrorString(e));
+            return FP_OK;
+        }
+        case FP_Q_DEVICE_STATUS: {
+            TRY(need(4));
+            int v = 0;
+            CK(cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+            *(int32_t*)h_out = v ? FP_ERR_TIMEOUT : 0;
+            return FP_OK;
+        }
+        case FP_Q_OP_TIMES: {
+            const int n = (int)h->ops.size();
+            TRY(need((size_t)n * sizeof(float)));
+            if (h->last_batch <= 0 || !h->last_input) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
+            const int reps = index > 0 ? index : 5;
+            std::vector<cudaEvent_t> ev(n + 1);
+            for (auto& e : ev) CK(cudaEventCreate(&e));
+            std::vector<float> acc(n, 0.f);
+            cudaStream_t st;
+            CK(cudaStreamCreate(&st));
+            for (int r = 0; r < reps + 1; ++r) {
+                CK(cudaEventRecord(ev[0], st));
+                for (int i = 0; i < n; ++i) {
+                    launch_op(h, h->ops[i], h->last_input, h->last_batch, h->d_logits_stage, st);
+                    CK(cudaEventRecord(ev[i + 1], st));
+                }
+                CK(cudaStreamSynchronize(st));
+                if (r == 0) continue;   // warm-up
+                for (int i = 0; i < n; ++i) { float ms; CK(cudaEventElapsedTime(&ms, ev[i], ev[i + 1])); acc[i] += ms; }
+            }
+            for (int i = 0; i < n; ++i) ((float*)h_out)[i] = acc[i] / reps;
+            for (auto& e : ev) cudaEventDestroy(e);
+            cudaStreamDestroy(st);
+            return FP_OK;
+        }
+        default: return fail(FP_ERR_ARG, "fp_query: unknown query %d", what);
+    }
+}

@@ -1,0 +1,164 @@
+// Filter preparation kernels: BN folding (Eq. 3-5 merged into the convolution), identity
+// filters of the auxiliary convolutions (Sec. IV-B.1), filter scoring (Eq. 6), ranking and
+// masking (Algorithm 1), and repacking of the surviving filters into K,R,S,C order.
+#include "fp_internal.h"
+
+namespace fp {
+
+// omega_k with one rounded fp32 operation per step: t = var + eps; r = sqrt(t); omega = gamma / r.
+__device__ __forceinline__ float bn_omega(const float* bn, int K, int k, float eps) {
+    const float t = __fadd_rn(bn[3 * K + k], eps);
+    const float r = __fsqrt_rn(t);
+    return __fdiv_rn(bn[k], r);
+}
+
+__global__ void fold_weights_kernel(const float* __restrict__ w, const float* __restrict__ bn, int K, int C, int R,
+                                    int S, float eps, float* __restrict__ dst, int C_dst, int R_dst, int S_dst,
+                                    int k0, int c0, int r0, int s0) {
+    const int per = C * R * S;
+    const size_t total = (size_t)K * per;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int k = (int)(i / per);
+        int rem = (int)(i - (size_t)k * per);
+        const int c = rem / (R * S);
+        rem -= c * R * S;
+        const int r = rem / S, s = rem - r * S;
+        const float omega = bn_omega(bn, K, k, eps);
+        dst[(((size_t)(k0 + k) * C_dst + (c0 + c)) * R_dst + (r + r0)) * S_dst + (s + s0)] = __fmul_rn(omega, w[i]);
+    }
+}
+
+// lambda = beta - omega * mean, the product and the difference rounded separately.
+__global__ void fold_bias_kernel(const float* __restrict__ bn, int K, float eps, float* __restrict__ dst, int k0,
+                                 int accumulate) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const float omega = bn_omega(bn, K, k, eps);
+    const float m = __fmul_rn(omega, bn[2 * K + k]);
+    const float lam = __fsub_rn(bn[K + k], m);
+    dst[k0 + k] = accumulate ? __fadd_rn(dst[k0 + k], lam) : lam;
+}
+
+__global__ void identity_filters_kernel(float* dst, int C_dst, int R, int S, int k0, int c0, int K_id, int C_id,
+                                        int shift) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K_id) return;
+    const int c = k - shift;
+    if (c < 0 || c >= C_id) return;
+    dst[(((size_t)(k0 + k) * C_dst + (c0 + c)) * R + R / 2) * S + S / 2] = 1.0f;
+}
+
+__global__ void count_nonfinite_kernel(const float* __restrict__ p, size_t n, int* count) {
+    int bad = 0;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        bad += !isfinite(p[i]);
+    if (bad) atomicAdd(count, bad);
+}
+
+// One warp per filter.  Lane l accumulates elements l, l+32, ... in increasing order in fp64
+// (each |w| or w*w is exact in fp64), then the 32 partial sums are combined pairwise with
+// partners at distance 16, 8, 4, 2, 1.  The order is part of the definition of the score, so
+// that the resulting double - and therefore the ranking - does not depend on the launch shape.
+__global__ void score_filters_kernel(const float* __restrict__ w, int K, int per, int norm, double* __restrict__ scores) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= K) return;
+    const float* f = w + (size_t)warp * per;
+    double s = 0.0;
+    for (int t = lane; t < per; t += 32) {
+        const double v = (double)f[t];
+        s = __dadd_rn(s, norm ? __dmul_rn(v, v) : fabs(v));
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) s = __dadd_rn(s, __shfl_xor_sync(0xffffffffu, s, d));
+    if (lane == 0) scores[warp] = s;
+}
+
+// rank[k] = number of filters ordered before k in ascending (score, index) order; the first q are masked.
+__global__ void rank_mask_kernel(const double* __restrict__ scores, int K, int q, int32_t* __restrict__ rank,
+                                 uint8_t* __restrict__ mask) {
+    extern __shared__ double sh[];
+    for (int i = threadIdx.x; i < K; i += blockDim.x) sh[i] = scores[i];
+    __syncthreads();
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        const double sk = sh[k];
+        int before = 0;
+        for (int j = 0; j < K; ++j) {
+            const double sj = sh[j];
+            before += (sj < sk) || (sj == sk && j < k);
+        }
+        rank[k] = before;
+        mask[k] = before >= q ? 1 : 0;
+    }
+}
+
+__global__ void repack_kernel(const float* __restrict__ w, int C, int RS, const int32_t* __restrict__ row_src,
+                              int K_pad, const int32_t* __restrict__ chan_src, int C_pad, float scale,
+                              __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32) {
+    const size_t total = (size_t)K_pad * RS * C_pad;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int cp = (int)(i % C_pad);
+        const size_t t = i / C_pad;
+        const int rs = (int)(t % RS);
+        const int kr = (int)(t / RS);
+        const int ks = row_src[kr], cs = chan_src[cp];
+        float v = 0.0f;
+        if (ks >= 0 && cs >= 0) v = w[((size_t)ks * C + cs) * RS + rs] * scale;
+        if (out_bf16) out_bf16[i] = __float2bfloat16_rn(v);
+        if (out_f32) out_f32[i] = v;
+    }
+}
+
+__global__ void pack_bias_kernel(const float* __restrict__ b, const int32_t* __restrict__ row_src, int K_pad,
+                                 float* __restrict__ out) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K_pad) return;
+    out[k] = row_src[k] >= 0 ? b[row_src[k]] : 0.0f;
+}
+
+static inline int blocks_for(size_t n, int threads, int cap = 148 * 8) {
+    size_t b = (n + threads - 1) / threads;
+    if (b < 1) b = 1;
+    return (int)(b > (size_t)cap ? cap : b);
+}
+
+void launch_fold_weights(const float* w, const float* bn, int K, int C, int R, int S, float eps, float* dst,
+                         int C_dst, int R_dst, int S_dst, int k0, int c0, int r0, int s0, cudaStream_t st) {
+    const size_t n = (size_t)K * C * R * S;
+    fold_weights_kernel<<<blocks_for(n, 256), 256, 0, st>>>(w, bn, K, C, R, S, eps, dst, C_dst, R_dst, S_dst, k0, c0, r0, s0);
+}
+
+void launch_fold_bias(const float* bn, int K, float eps, float* dst_b, int k0, int accumulate, cudaStream_t st) {
+    fold_bias_kernel<<<(K + 127) / 128, 128, 0, st>>>(bn, K, eps, dst_b, k0, accumulate);
+}
+
+void launch_identity_filters(float* dst, int C_dst, int R, int S, int k0, int c0, int K_id, int C_id, int shift,
+                             cudaStream_t st) {
+    identity_filters_kernel<<<(K_id + 127) / 128, 128, 0, st>>>(dst, C_dst, R, S, k0, c0, K_id, C_id, shift);
+}
+
+void launch_count_nonfinite(const float* p, size_t n, int* d_count, cudaStream_t st) {
+    if (n == 0) return;
+    count_nonfinite_kernel<<<blocks_for(n, 256), 256, 0, st>>>(p, n, d_count);
+}
+
+void launch_score_filters(const float* w, int K, int per_filter, int norm, double* scores, cudaStream_t st) {
+    const int warps_per_block = 8;
+    score_filters_kernel<<<(K + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(w, K, per_filter, norm, scores);
+}
+
+void launch_rank_mask(const double* scores, int K, int q, int32_t* rank, uint8_t* mask, cudaStream_t st) {
+    rank_mask_kernel<<<1, 256, (size_t)K * sizeof(double), st>>>(scores, K, q, rank, mask);
+}
+
+void launch_repack(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
+                   int C_pad, float scale, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st) {
+    const size_t n = (size_t)K_pad * RS * C_pad;
+    repack_kernel<<<blocks_for(n, 256), 256, 0, st>>>(w, C, RS, row_src, K_pad, chan_src, C_pad, scale, out_bf16, out_f32);
+}
+
+void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st) {
+    pack_bias_kernel<<<(K_pad + 127) / 128, 128, 0, st>>>(b, row_src, K_pad, out);
+}
+
+}  // namespace fp

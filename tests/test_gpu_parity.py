@@ -1,0 +1,394 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+
+Tolerances (stated by the workload definition):
+  masks / ranks / scores              bit-exact
+  BF16 tensor-core activations        max|err| <= 2e-2 * max|ref|
+  FP32 validation path                max|err| <= 1e-4 * max|ref|
+"""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from paper_2010_16165_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_FP32 = 1e-4
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2010_16165_b200 import binding
+    binding.lib()
+    return binding
+
+
+def to_dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+class Gpu:
+    """One fused model on the device."""
+
+    def __init__(self, B, w, compute, max_batch=None, use_graph=0, keep_outputs=0, in_bf16=None):
+        self.B, self.w = B, w
+        self.dw, self.dbn = to_dev(w.weights), to_dev(w.bn)
+        self.in_bf16 = w.in_bf16 if in_bf16 is None else in_bf16
+        self.h = B.fp_fuse(w.net, self.dw, self.dbn, max_batch or w.batch, compute,
+                           B.FP_DTYPE_BF16 if self.in_bf16 else B.FP_DTYPE_F32, use_graph, keep_outputs)
+        self.n_classes = B.fp_query_int(self.h, B.FP_Q_N_CLASSES)
+
+    def forward(self, x, stream=None):
+        dx = to_dev(x)
+        if self.in_bf16:
+            dx = dx.to(torch.bfloat16)
+        out = torch.full((x.shape[0], self.n_classes), float("nan"), device="cuda", dtype=torch.float32)
+        if stream is not None:
+            stream.wait_stream(torch.cuda.current_stream())
+        self.B.fp_forward(self.h, dx, x.shape[0], out, stream)
+        torch.cuda.synchronize()
+        assert self.B.fp_query_int(self.h, self.B.FP_Q_DEVICE_STATUS) == 0, "a device-side wait timed out"
+        return out.cpu().numpy().astype(np.float64)
+
+    def close(self):
+        self.B.fp_destroy(self.h)
+
+
+def err(got, ref):
+    return np.abs(got - ref).max() / np.abs(ref).max()
+
+
+def oracle_pruned(fpo, w, masks=None):
+    gp, m, ranks, scores = fpo.pruned_model(w.net, w.weights, w.bn, w.ratios, masks=masks)
+    return gp, m, ranks, scores
+
+
+TINY = {
+    "cifar": lambda **k: wl.tiny_cifar(**k),
+    "cifar_odd": lambda **k: wl.tiny_cifar(widths=(7, 12, 23), in_hw=12, batch=3, **k),
+    "cifar_centered": lambda **k: wl.tiny_cifar(pad_lo_centered=True, n_per_stage=2, **k),
+    "cifar_wide": lambda **k: wl.tiny_cifar(widths=(16, 48, 80), in_hw=16, batch=5, **k),
+    "imagenet_basic": lambda **k: wl.tiny_imagenet_basic(**k),
+    "imagenet_wide": lambda **k: wl.tiny_imagenet_basic(widths=(32, 64, 96), in_hw=48, batch=3, **k),
+}
+
+
+# ------------------------------------------------------------------------------------------
+# scoring, ranking, masks: bit-exact
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name", ["cifar", "cifar_odd", "imagenet_basic"])
+@pytest.mark.parametrize("aggressive", [False, True])
+@pytest.mark.parametrize("norm", [0, 1])
+def test_scores_masks_bit_exact_tiny(B, fpo, name, aggressive, norm):
+    w = TINY[name](aggressive=aggressive, p=0.3)
+    g = Gpu(B, w, B.FP_COMPUTE_FP32)
+    try:
+        g32 = fpo.fuse(w.net, w.weights, w.bn, "f32")
+        masks, ranks, scores = fpo.select_masks(g32, w.ratios, norm)
+        B.fp_prune(g.h, w.ratios, None, norm)
+        got = B.masks_and_ranks(g.h)
+        for ci in range(w.net.n_convs()):
+            if masks[ci] is None:
+                assert got[ci][0] is None
+                continue
+            s = B.fp_score(g.h, ci, norm)
+            assert s.tobytes() == scores[ci].tobytes(), f"conv {ci}: scores differ"
+            np.testing.assert_array_equal(got[ci][1], ranks[ci])
+            np.testing.assert_array_equal(got[ci][0], masks[ci])
+    finally:
+        g.close()
+
+
+def test_masks_bit_exact_resnet20_and_bottleneck(B, fpo):
+    for w in (wl.workload(1), wl.tiny_bottleneck(p=0.4)):
+        g = Gpu(B, w, B.FP_COMPUTE_FP32, max_batch=2)
+        try:
+            g32 = fpo.fuse(w.net, w.weights, w.bn, "f32")
+            masks, ranks, scores = fpo.select_masks(g32, w.ratios, 0)
+            B.fp_prune(g.h, w.ratios)
+            got = B.masks_and_ranks(g.h)
+            for ci in range(w.net.n_convs()):
+                np.testing.assert_array_equal(got[ci][0], masks[ci])
+                np.testing.assert_array_equal(got[ci][1], ranks[ci])
+                assert B.fp_score(g.h, ci, 0).tobytes() == scores[ci].tobytes()
+                assert B.fp_query_int(g.h, B.FP_Q_CONV_K_KEPT, ci) == int(masks[ci].sum())
+        finally:
+            g.close()
+
+
+def test_caller_masks_are_used(B, fpo):
+    w = wl.tiny_cifar(p=0.0)
+    rng = np.random.default_rng(5)
+    masks = {}
+    for ci, nid in enumerate(w.net.conv_ids()):
+        m = (rng.random(w.net.nodes[nid]["K"]) > 0.4).astype(np.uint8)
+        m[0] = 1
+        masks[ci] = m
+    g = Gpu(B, w, B.FP_COMPUTE_FP32)
+    try:
+        B.fp_prune(g.h, None, masks)
+        got = g.forward(w.x)
+        gp, _, _, _ = oracle_pruned(fpo, w, masks)
+        assert err(got, fpo.fused_forward(gp, w.x)) < TOL_FP32
+    finally:
+        g.close()
+
+
+# ------------------------------------------------------------------------------------------
+# activations, tiny networks, every compute path
+# ------------------------------------------------------------------------------------------
+
+def _compare_ops(B, g, w, gp, fpo, tol):
+    """Per-operator comparison (needs keep_outputs=1): reports the first operator that is off."""
+    ref_all = fpo.fused_forward(gp, w.x, return_all=True)
+    infos = B.op_infos(g.h)
+    conv_ops = [op for op in gp.ops]
+    oi = 0
+    for i, info in enumerate(infos):
+        if info.kind in (2, 3):
+            continue
+        ref = ref_all[conv_ops[oi]["out"]]
+        oi += 1
+        cnt = w.x.shape[0] * info.K_pad * info.P * info.Q   # upper bound
+        C = ref.shape[1]
+        got = B.fp_query_array(g.h, B.FP_Q_OP_OUTPUT, i, np.float32, w.x.shape[0] * C * info.P * info.Q)
+        got = got.reshape(ref.shape).astype(np.float64)
+        e = np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30)
+        assert e < tol, f"operator {i} (kind {info.kind}, conv {info.conv_index}, K={info.K} C={info.C} " \
+                        f"R={info.R} stride={info.stride} res={info.res_mode}): rel err {e:.3e}"
+
+
+@pytest.mark.parametrize("name", list(TINY))
+@pytest.mark.parametrize("aggressive", [False, True])
+@pytest.mark.parametrize("p", [0.0, 0.3])
+@pytest.mark.parametrize("compute", ["fp32", "simt", "tc"])
+def test_tiny_networks(B, fpo, name, aggressive, p, compute):
+    w = TINY[name](aggressive=aggressive, p=p)
+    mode = {"fp32": B.FP_COMPUTE_FP32, "simt": B.FP_COMPUTE_BF16_SIMT, "tc": B.FP_COMPUTE_BF16_TC}[compute]
+    tol = TOL_FP32 if compute == "fp32" else TOL_BF16
+    g = Gpu(B, w, mode, keep_outputs=1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        got = g.forward(w.x)
+        gp, masks, _, _ = oracle_pruned(fpo, w)
+        ref = fpo.fused_forward(gp, w.x)
+        if not err(got, ref) < tol:
+            _compare_ops(B, g, w, gp, fpo, tol)
+        assert err(got, ref) < tol
+        if p == 0.0:
+            # fusion is an equivalence: the unfused description gives the same logits
+            assert err(got, fpo.unfused_forward(w.net, w.weights, w.bn, w.x)) < tol
+    finally:
+        g.close()
+
+
+@pytest.mark.parametrize("compute", ["fp32", "tc"])
+def test_tiny_bottleneck(B, fpo, compute):
+    w = wl.tiny_bottleneck(p=0.4)
+    mode = B.FP_COMPUTE_FP32 if compute == "fp32" else B.FP_COMPUTE_BF16_TC
+    tol = TOL_FP32 if compute == "fp32" else TOL_BF16
+    g = Gpu(B, w, mode, keep_outputs=1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        got = g.forward(w.x)
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        ref = fpo.fused_forward(gp, w.x)
+        if not err(got, ref) < tol:
+            _compare_ops(B, g, w, gp, fpo, tol)
+        assert err(got, ref) < tol
+    finally:
+        g.close()
+
+
+def test_per_operator_outputs_tc(B, fpo):
+    """Every fused operator's activation, not only the logits (several tiles, ragged tails)."""
+    w = wl.tiny_cifar(widths=(16, 32, 64), in_hw=20, batch=3, n_per_stage=2, p=0.3)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, keep_outputs=1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        g.forward(w.x)
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        _compare_ops(B, g, w, gp, fpo, TOL_BF16)
+    finally:
+        g.close()
+
+
+def test_prune_ratio_zero_restores_unpruned(B, fpo):
+    w = wl.tiny_cifar(n_per_stage=2, p=0.5)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC)
+    try:
+        before = g.forward(w.x)
+        B.fp_prune(g.h, w.ratios)
+        pruned = g.forward(w.x)
+        B.fp_prune(g.h, np.zeros_like(w.ratios))
+        after = g.forward(w.x)
+        np.testing.assert_array_equal(before, after)
+        assert np.abs(before - pruned).max() > 1e-3
+    finally:
+        g.close()
+
+
+def test_batch_edges_and_graph_and_host(B, fpo):
+    w = wl.tiny_cifar(batch=7, p=0.3)
+    gp, _, _, _ = oracle_pruned(fpo, w)
+    ref = fpo.fused_forward(gp, w.x)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, max_batch=9, use_graph=1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        full = g.forward(w.x)
+        assert err(full, ref) < TOL_BF16
+        # images are independent: any sub-batch reproduces its rows bit for bit
+        for b in (1, 2, 5):
+            np.testing.assert_array_equal(g.forward(w.x[:b]), full[:b])
+        # CUDA-graph replay on a side stream gives the same bits, twice
+        st = torch.cuda.Stream()
+        a1 = g.forward(w.x, st)
+        a2 = g.forward(w.x, st)
+        np.testing.assert_array_equal(a1, full)
+        np.testing.assert_array_equal(a2, full)
+        # host-buffer entry point
+        out = np.empty((7, g.n_classes), dtype=np.float32)
+        B.fp_forward_host(g.h, w.x, 7, out)
+        np.testing.assert_array_equal(out.astype(np.float64), full)
+        with pytest.raises(B.FpError) as e:
+            B.fp_forward(g.h, to_dev(w.x), 10, torch.empty(10, g.n_classes, device="cuda"))
+        assert e.value.status == B.FP_ERR_BOUNDS
+    finally:
+        g.close()
+
+
+def test_error_codes(B):
+    w = wl.tiny_cifar()
+    dw, dbn = to_dev(w.weights), to_dev(w.bn)
+    # NaN in the weights
+    bad = w.weights.copy(); bad[3] = np.nan
+    with pytest.raises(B.FpError) as e:
+        B.fp_fuse(w.net, to_dev(bad), dbn, 2, B.FP_COMPUTE_FP32)
+    assert e.value.status == B.FP_ERR_NONFINITE
+    # a convolution whose channel count does not match its producer
+    import copy
+    net = copy.deepcopy(w.net)
+    net.nodes[net.conv_ids()[1]]["C"] += 1
+    with pytest.raises(B.FpError) as e:
+        B.fp_fuse(net, dw, dbn, 2, B.FP_COMPUTE_FP32)
+    assert e.value.status in (B.FP_ERR_SHAPE, B.FP_ERR_DESC)
+    # forward reference
+    net = copy.deepcopy(w.net)
+    net.nodes[2]["in0"] = 5
+    with pytest.raises(B.FpError) as e:
+        B.fp_fuse(net, dw, dbn, 2, B.FP_COMPUTE_FP32)
+    assert e.value.status == B.FP_ERR_DESC
+    # pruning everything
+    h = B.fp_fuse(w.net, dw, dbn, 2, B.FP_COMPUTE_FP32)
+    try:
+        with pytest.raises(B.FpError) as e:
+            B.fp_prune(h, np.ones(w.net.n_convs()))
+        assert e.value.status == B.FP_ERR_EMPTY_LAYER
+        with pytest.raises(B.FpError) as e:
+            B.fp_prune(h, np.full(w.net.n_convs(), -0.5))
+        assert e.value.status == B.FP_ERR_ARG
+    finally:
+        B.fp_destroy(h)
+    # aggressive fusion of a bottleneck block is not supported
+    wb = wl.tiny_bottleneck()
+    net = copy.deepcopy(wb.net)
+    for n in net.nodes:
+        if n["block_id"] >= 0:
+            n["aggressive"] = 1
+    with pytest.raises(B.FpError) as e:
+        B.fp_fuse(net, to_dev(wb.weights), to_dev(wb.bn), 2, B.FP_COMPUTE_FP32)
+    assert e.value.status == B.FP_ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------------------------------
+# the benchmark-shaped workloads at full size
+# ------------------------------------------------------------------------------------------
+
+def _sample_images(n, k):
+    idx = sorted(set([0, n - 1] + list(range(0, n, 37))))
+    return idx[:k] if len(idx) > k else idx
+
+
+def _full_config(B, fpo, w, n_oracle, also_fp32=True, aggressive_note=""):
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, use_graph=1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        st = torch.cuda.Stream()
+        got = g.forward(w.x, st)
+        assert np.isfinite(got).all()
+        # masks bit-exact at full size
+        g32 = fpo.fuse(w.net, w.weights, w.bn, "f32")
+        masks, ranks, _ = fpo.select_masks(g32, w.ratios, 0)
+        mr = B.masks_and_ranks(g.h)
+        for ci in range(w.net.n_convs()):
+            if masks[ci] is not None:
+                np.testing.assert_array_equal(mr[ci][0], masks[ci])
+                np.testing.assert_array_equal(mr[ci][1], ranks[ci])
+        # sampled images against the oracle
+        idx = _sample_images(w.batch, n_oracle)
+        gp = fpo.prune_remove(fpo.fuse(w.net, w.weights, w.bn), masks)
+        ref = fpo.fused_forward(gp, w.x[idx])
+        e = err(got[idx], ref)
+        assert e < TOL_BF16, f"{w.name}: bf16 tensor-core path rel err {e:.3e}"
+    finally:
+        g.close()
+    if also_fp32:
+        # every image: FP32 validation path (itself within 1e-4 of the oracle on the samples)
+        g = Gpu(B, w, B.FP_COMPUTE_FP32)
+        try:
+            B.fp_prune(g.h, w.ratios)
+            got32 = g.forward(w.x)
+            assert err(got32[idx], ref) < TOL_FP32
+            assert err(got, got32) < TOL_BF16
+        finally:
+            g.close()
+
+
+def test_config1_resnet20_b8(B, fpo):
+    w = wl.workload(1)
+    _full_config(B, fpo, w, 8)
+
+
+@pytest.mark.parametrize("p", [0.0, 0.3, 0.5])
+def test_config2_resnet56_b256(B, fpo, p):
+    w = wl.workload(2, prune=p)
+    _full_config(B, fpo, w, 12)
+
+
+def test_config3_resnet110_b1024(B, fpo):
+    w = wl.workload(3)
+    _full_config(B, fpo, w, 6)
+
+
+def test_config4_resnet18_b64(B, fpo):
+    w = wl.workload(4)
+    _full_config(B, fpo, w, 2)
+
+
+def test_config5_resnet50(B, fpo):
+    w = wl.workload(5, batch=16)     # the oracle covers two images; all 16 go through both GPU paths
+    _full_config(B, fpo, w, 2)
+    w1 = wl.workload(5, batch=1)
+    _full_config(B, fpo, w1, 1, also_fp32=False)
+
+
+def test_config1_aggressive_fused_unpruned_and_pruned(B, fpo):
+    """The paper's own graph: dilated convolutions, no add; then pruned back by n-m filters."""
+    w = wl.workload(1, aggressive=True)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC)
+    try:
+        got = g.forward(w.x)
+        ref = fpo.unfused_forward(w.net, w.weights, w.bn, w.x)
+        assert err(got, ref) < TOL_BF16
+        B.fp_prune(g.h, np.zeros(w.net.n_convs()))          # conservative: fused operators lose n-m
+        gp, masks, _, _ = fpo.pruned_model(w.net, w.weights, w.bn, np.zeros(w.net.n_convs()))
+        assert err(g.forward(w.x), fpo.fused_forward(gp, w.x)) < TOL_BF16
+        for ci, m in B.masks_and_ranks(g.h).items():
+            np.testing.assert_array_equal(m[0], masks[ci])
+    finally:
+        g.close()
