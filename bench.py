@@ -1,0 +1,324 @@
+"""Benchmark: images/s of the fused + pruned ResNet forward (ResNet-56, batch 256, 30 % of every
+convolution's filters pruned by L1 norm) through the C-ABI library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--prune P] [--config C]
+
+One step = one fp_forward of the whole fused graph over one batch of synthetic, seeded images that
+are already in HBM.  Between timed steps L2 is flushed by writing a 256 MiB buffer; each step is timed
+with CUDA events on the launching stream and the K step times are summed.  Prints one JSON line.
+`--impl reference` times the CPU oracle on the host cores instead (a deliberately plain program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "images/s of fused+pruned ResNet forward on 1 B200; % of BF16 tensor/HBM roofline"
+UNIT = "images/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# multi-process plumbing (one process per GPU; the path has no collective: replicas of the
+# same batch-sharded work, timing reduced as max over ranks)
+# ------------------------------------------------------------------------------------------
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def init_dist(backend):
+    import torch.distributed as dist
+    rank, world, _ = dist_env()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def aggregate(elapsed_ms, units, device="cpu"):
+    """Whole-job figures: time = max over ranks, units = sum over ranks."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(elapsed_ms), float(units)
+    t = torch.tensor([float(elapsed_ms)], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        inside = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.06] or [r for (_, r) in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in inside:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+                for n, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------
+
+def oracle_images_per_s(w, n_images, repeats=1):
+    """The oracle as it stands: fused + pruned forward in fp64 on the host cores."""
+    from oracle import fpo
+    gp, _, _, _ = fpo.pruned_model(w.net, w.weights, w.bn, w.ratios)
+    x = w.x[:n_images]
+    best = None
+    for _ in range(repeats):
+        t = time.perf_counter()
+        fpo.fused_forward(gp, x)
+        dt = time.perf_counter() - t
+        best = dt if best is None else min(best, dt)
+    return n_images / best, fpo.num_threads(), best
+
+
+def run_reference(args):
+    from paper_2010_16165_b200 import workloads as wl
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    from oracle import fpo
+    w = wl.workload(args.config, prune=args.prune)
+    cores = fpo.num_threads()
+    n_img = min(w.batch, max(2 * cores, 8))
+    gp, _, _, _ = fpo.pruned_model(w.net, w.weights, w.bn, w.ratios)
+    x = w.x[:n_img]
+    steps = min(args.steps, 20)
+    for _ in range(min(args.warmup, 2)):
+        fpo.fused_forward(gp, x)
+    t = time.perf_counter()
+    for _ in range(steps):
+        fpo.fused_forward(gp, x)
+    dt = time.perf_counter() - t
+    v = n_img * steps / dt
+    sample = f"{n_img} of {w.batch} images per step, {steps} steps (per-image cost does not depend on batch)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 2), "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "net": w.net.name, "batch": w.batch, "prune": w.ratio_spec},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------
+# the GPU arm
+# ------------------------------------------------------------------------------------------
+
+def run_gpu(args):
+    import torch
+    from paper_2010_16165_b200 import binding as B, workloads as wl
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    if world > 1:
+        init_dist("nccl")
+    dev = torch.device("cuda", local)
+    peaks, peak_kind = load_peaks()
+
+    w = wl.workload(args.config, prune=args.prune)
+    dw, dbn = torch.from_numpy(w.weights).to(dev), torch.from_numpy(w.bn).to(dev)
+    h = B.fp_fuse(w.net, dw, dbn, w.batch, B.FP_COMPUTE_BF16_TC, B.FP_DTYPE_BF16 if w.in_bf16 else B.FP_DTYPE_F32,
+                  1, 0)
+    B.fp_prune(h, w.ratios)
+    n_classes = B.fp_query_int(h, B.FP_Q_N_CLASSES)
+    x_host = torch.from_numpy(w.x)
+    if w.in_bf16:
+        x_host = x_host.to(torch.bfloat16)
+    x_pinned = x_host.pin_memory()
+    dx = x_host.to(dev)
+    logits = torch.empty(w.batch, n_classes, device=dev)
+    logits_pinned = torch.empty(w.batch, n_classes).pin_memory()
+    stream = torch.cuda.Stream(device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than the 126 MB L2
+
+    def step_device():
+        B.fp_forward(h, dx, w.batch, logits, stream)
+
+    def step_host():
+        B.fp_forward_host(h, x_pinned, w.batch, logits_pinned, stream)
+
+    def timed(step, steps, warmup):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                flush.fill_(1)
+                step()
+            torch.cuda.synchronize()
+            barrier()
+            torch.cuda.synchronize()
+            t0 = time.time()
+            for a, b in ev:
+                flush.fill_(1)
+                a.record(stream)
+                step()
+                b.record(stream)
+            torch.cuda.synchronize()
+            barrier()
+            torch.cuda.synchronize()
+            t1 = time.time()
+        return sum(a.elapsed_time(b) for a, b in ev), t0, t1
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.3 if sampler else 0.0)
+    ms, t0, t1 = timed(step_device, args.steps, max(args.warmup, 3))
+    clocks = sampler.stop(t0, t1) if sampler else None
+    assert B.fp_query_int(h, B.FP_Q_DEVICE_STATUS) == 0, "a device-side wait timed out"
+    ms_e2e, _, _ = timed(step_host, args.steps, max(args.warmup, 3))
+    tot_ms, tot_units = aggregate(ms, w.batch * args.steps, dev)
+    tot_ms_e2e, _ = aggregate(ms_e2e, w.batch * args.steps, dev)
+
+    # ---- per-operator times (CUDA events around every launch, same stream order as a forward) ----
+    ops = B.op_infos(h)
+    op_ms = B.fp_query_array(h, B.FP_Q_OP_TIMES, 20, np.float32, len(ops))
+    conv = [(o, t) for o, t in zip(ops, op_ms) if o.kind == 0]
+    conv_bytes = sum(o.bytes_per_image * w.batch + o.bytes_fixed for o, _ in conv)
+    conv_flops = sum(o.flops_per_image * w.batch for o, _ in conv)
+    conv_ms = float(sum(t for _, t in conv))
+    n_conv = len(conv)
+    t_hbm = conv_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_flop = conv_flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    if t_hbm >= t_flop:
+        roof = {"bound": "hbm", "achieved": conv_bytes / (conv_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": conv_flops / (conv_ms * 1e-3) / 1e12,
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["peak_source"] = peak_kind
+    roof["kernel"] = "conv_tc_kernel"
+    roof["launches_per_step"] = n_conv
+    roof["avg_launch_us"] = 1e3 * conv_ms / n_conv
+    roof["algorithmic_bytes_per_step"] = conv_bytes
+    roof["algorithmic_flops_per_step"] = conv_flops
+    roof["share_of_step"] = conv_ms / float(sum(op_ms))
+    flops_img = B.fp_query_array(h, B.FP_Q_FLOPS, 0, np.float64, 1)[0]
+    bytes2 = B.fp_query_array(h, B.FP_Q_BYTES, 0, np.float64, 2)
+    n_launch = B.fp_query_int(h, B.FP_Q_N_LAUNCHES)
+
+    out = None
+    if rank == 0:
+        value = tot_units / (tot_ms * 1e-3)
+        step_ms = tot_ms / args.steps
+        whole_bytes = bytes2[0] * w.batch + bytes2[1]
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "net": w.net.name, "batch_per_gpu": w.batch, "prune": w.ratio_spec,
+                       "norm": "l1", "fusion": "bn folded, shortcut+relu in conv epilogue", "cuda_graph": True,
+                       "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world}"},
+            "e2e": {"value": tot_units / (tot_ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size()),
+                    "d2h_bytes_per_step": int(logits_pinned.numel() * 4), "ms_per_step": tot_ms_e2e / args.steps},
+            "gpu_launches": int(n_launch * args.steps),
+            "clocks": clocks,
+            "roofline": roof,
+            "whole_step": {"flops": flops_img * w.batch, "algorithmic_bytes": whole_bytes,
+                           "hbm_frac": whole_bytes / (step_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                           "tensor_frac": flops_img * w.batch / (step_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                           "sum_op_ms_no_graph": float(sum(op_ms))},
+        }
+    B.fp_destroy(h)
+    if rank == 0:
+        if world == 1 and not args.no_cpu:
+            n_img = min(w.batch, max(2 * (os.cpu_count() or 8), 8))
+            v, cores, secs = oracle_images_per_s(w, n_img, repeats=2)
+            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                   "sample": f"{n_img} of {w.batch} images, best of 2 ({secs:.2f} s each)"}
+        print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--prune", type=float, default=None)
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -173,6 +173,9 @@ def test_tiny_networks(B, fpo, name, aggressive, p, compute):
     tol = TOL_FP32 if compute == "fp32" else TOL_BF16
     g = Gpu(B, w, mode, keep_outputs=1)
     try:
+        if p == 0.0:
+            # fusion alone is an equivalence: the fused graph reproduces the network as described
+            assert err(g.forward(w.x), fpo.unfused_forward(w.net, w.weights, w.bn, w.x)) < tol
         B.fp_prune(g.h, w.ratios)
         got = g.forward(w.x)
         gp, masks, _, _ = oracle_pruned(fpo, w)
@@ -180,9 +183,6 @@ def test_tiny_networks(B, fpo, name, aggressive, p, compute):
         if not err(got, ref) < tol:
             _compare_ops(B, g, w, gp, fpo, tol)
         assert err(got, ref) < tol
-        if p == 0.0:
-            # fusion is an equivalence: the unfused description gives the same logits
-            assert err(got, fpo.unfused_forward(w.net, w.weights, w.bn, w.x)) < tol
     finally:
         g.close()
 
