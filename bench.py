@@ -294,6 +294,17 @@ def run_gpu(args):
                            "tensor_frac": flops_img * w.batch / (step_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                            "sum_op_ms_no_graph": float(sum(op_ms))},
         }
+    if rank == 0 and args.per_op:
+        groups = {}
+        for o, t in zip(ops, op_ms):
+            key = (("conv", "maxpool", "head", "input")[o.kind], o.C, o.K, o.R, o.stride, o.H, o.res_mode)
+            g = groups.setdefault(key, [0, 0.0, 0.0, 0.0])
+            g[0] += 1; g[1] += float(t) * 1e3
+            g[2] += o.bytes_per_image * w.batch + o.bytes_fixed; g[3] += o.flops_per_image * w.batch
+        out["per_op"] = [{"op": k[0], "C": k[1], "K": k[2], "R": k[3], "stride": k[4], "H": k[5], "res": k[6],
+                          "launches": g[0], "us_per_launch": round(g[1] / g[0], 2),
+                          "GBps": round(g[2] / g[0] / (g[1] / g[0] * 1e-6) / 1e9, 1),
+                          "TFLOPs": round(g[3] / g[0] / (g[1] / g[0] * 1e-6) / 1e12, 2)} for k, g in groups.items()]
     B.fp_destroy(h)
     if rank == 0:
         if world == 1 and not args.no_cpu:
@@ -312,7 +323,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--prune", type=float, default=None)
-    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--per-op", action="store_true", help="add per-operator-class times to the JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
