@@ -421,6 +421,8 @@ struct Builder {
             }
         }
         if (h->head_src < 0) return fail(FP_ERR_DESC, "description has no global-average-pool + FC head");
+        for (const Tensor& t : h->tensors)
+            if (t.W > fp::kMaxWidth) return fail(FP_ERR_UNSUPPORTED, "images wider than %d pixels are not supported", fp::kMaxWidth);
         if (h->ops.back().kind != 2) return fail(FP_ERR_DESC, "the head must be the last operator");
         return FP_OK;
     }
@@ -517,8 +519,8 @@ fp_status replan(fp_handle h) {
             const size_t cnt = (size_t)f.K_pad * f.R * f.S * f.C_pad;
             TRY(dev_alloc(h->pack_buffers, &f.d_wp, cnt * h->act_elem()));
             TRY(dev_alloc(h->pack_buffers, (void**)&f.d_bp, (size_t)f.K_pad * sizeof(float)));
-            fp::launch_repack(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad, 1.0f,
-                              bf16 ? (__nv_bfloat16*)f.d_wp : nullptr, bf16 ? nullptr : (float*)f.d_wp, st);
+            fp::launch_repack_conv(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad,
+                                   bf16 ? (__nv_bfloat16*)f.d_wp : nullptr, bf16 ? nullptr : (float*)f.d_wp, st);
             fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);
         } else if (op.kind == 1) {
             const Pool& p = h->pools[op.idx];
@@ -527,16 +529,14 @@ fp_status replan(fp_handle h) {
             out.C = src.C; out.C_pad = src.C_pad; out.keep = src.keep;
         } else if (op.kind == 2) {
             const Tensor& src = h->tensors[h->head_src];
-            std::vector<int32_t> row_src(h->n_classes), chan_src(src.C_pad, -1);
-            for (int k = 0; k < h->n_classes; ++k) row_src[k] = k;
+            std::vector<int32_t> chan_src(src.C_pad, -1);
             for (int c = 0; c < src.C; ++c) chan_src[c] = src.keep[c];
-            int32_t *d_row, *d_chan;
-            TRY(upload_i32(h, row_src, &d_row));
+            int32_t* d_chan;
             TRY(upload_i32(h, chan_src, &d_chan));
             TRY(dev_alloc(h->pack_buffers, (void**)&h->d_fcw_packed, (size_t)h->n_classes * src.C_pad * sizeof(float)));
             // the average's 1/(H*W) is folded into the FC weights
-            fp::launch_repack(h->d_fcw, h->fc_C, 1, d_row, h->n_classes, d_chan, src.C_pad, 1.0f / (float)(src.H * src.W),
-                              nullptr, h->d_fcw_packed, st);
+            fp::launch_repack_fc(h->d_fcw, h->fc_C, h->n_classes, d_chan, src.C_pad, 1.0f / (float)(src.H * src.W),
+                                 h->d_fcw_packed, st);
         }
     }
     CK(cudaGetLastError());
@@ -557,7 +557,9 @@ fp_status replan(fp_handle h) {
             else if (op.kind == 3) tid = 0;
             if (tid < 0) continue;
             Tensor& t = h->tensors[tid];
-            t.bytes = (size_t)h->max_batch * t.H * t.W * t.C_pad * h->act_elem();
+            // planar-8 with border, plus guard vectors before and after (halo reads of the first/last tiles)
+            const size_t vec_bytes = 8 * h->act_elem();
+            t.bytes = ((size_t)(t.C_pad / 8) * h->max_batch * (t.H + 2) * (t.W + 2) + 2 * (size_t)fp::kGuardVectors) * vec_bytes;
             int best = -1;
             if (!h->keep_outputs)
                 for (int b = 0; b < (int)bufs.size(); ++b)
@@ -569,7 +571,7 @@ fp_status replan(fp_handle h) {
                 bufs.push_back({p, t.bytes, 0});
                 best = (int)bufs.size() - 1;
             }
-            t.d = bufs[best].p;
+            t.d = (uint8_t*)bufs[best].p + (size_t)fp::kGuardVectors * vec_bytes;
             bufs[best].free_after = std::max(last_use[tid], i);
         }
     }
@@ -608,7 +610,7 @@ void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float*
     const int bf16 = h->act_is_bf16();
     if (op.kind == 3) {
         const Tensor& t = h->tensors[0];
-        fp::launch_input_to_nhwc(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, st);
+        fp::launch_input_to_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, st);
     } else if (op.kind == 0) {
         FConv& f = h->convs[op.idx];
         fp::ConvArgs a = f.args;
@@ -622,7 +624,7 @@ void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float*
         fp::launch_maxpool(s.d, o.d, bf16, batch, s.H, s.W, s.C_pad, o.H, o.W, p.R, p.stride, p.pad, st);
     } else {
         const Tensor& s = h->tensors[h->head_src];
-        fp::launch_head(s.d, bf16, batch, s.H * s.W, s.C_pad, h->d_fcw_packed, h->d_fcb, h->n_classes, d_logits, st);
+        fp::launch_head(s.d, bf16, batch, s.H, s.W, s.C_pad, h->d_fcw_packed, h->d_fcb, h->n_classes, d_logits, st);
     }
 }
 
@@ -923,16 +925,12 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             const Tensor& t = h->tensors[tid];
             const size_t cnt = (size_t)h->last_batch * t.C * t.H * t.W;
             TRY(need(cnt * sizeof(float)));
-            std::vector<int32_t> chan_dst(t.C_pad, -1);
-            for (int c = 0; c < t.C; ++c) chan_dst[c] = c;
-            float* d_tmp; int32_t* d_chan;
+            float* d_tmp;
             CK(cudaDeviceSynchronize());
             CK(cudaMalloc(&d_tmp, cnt * sizeof(float)));
-            CK(cudaMalloc(&d_chan, chan_dst.size() * 4));
-            CK(cudaMemcpy(d_chan, chan_dst.data(), chan_dst.size() * 4, cudaMemcpyHostToDevice));
-            fp::launch_nhwc_to_nchw_f32(t.d, h->act_is_bf16(), d_tmp, h->last_batch, t.H, t.W, t.C_pad, d_chan, t.C, 0);
+            fp::launch_planar_to_nchw_f32(t.d, h->act_is_bf16(), d_tmp, h->last_batch, t.H, t.W, t.C_pad, t.C, 0);
             cudaError_t e = cudaMemcpy(h_out, d_tmp, cnt * sizeof(float), cudaMemcpyDeviceToHost);
-            cudaFree(d_tmp); cudaFree(d_chan);
+            cudaFree(d_tmp);
             if (e != cudaSuccess) return fail(FP_ERR_CUDA, "fp_query: copy failed: %s", cudaGetErrorString(e));
             return FP_OK;
         }

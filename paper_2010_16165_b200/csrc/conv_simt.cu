@@ -1,10 +1,13 @@
 // Plain convolution on CUDA cores with the same fused epilogue as the tensor-core path
-// (folded-BN bias, residual operand, ReLU).  Validation only: one thread per four output
-// channels of one output pixel, fp32 accumulation, no tensor cores.  T = float gives the
-// fp32 validation path; T = bf16 reads and writes the tensor-core path's storage.
+// (folded-BN bias, residual operand, ReLU) on the planar-8 layout.  Validation only: one
+// thread per output vector (8 filters of one output position, border positions included and
+// written as zeros), fp32 accumulation, no tensor cores.  T = float is the fp32 validation
+// path; T = bf16 reads and writes the tensor-core path's storage.
 #include "fp_internal.h"
 
 namespace fp {
+
+namespace {
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
@@ -19,49 +22,68 @@ __global__ void conv_simt_kernel(ConvArgs a) {
     const T* __restrict__ w = (const T*)a.w;
     const T* __restrict__ res = (const T*)a.res;
     T* __restrict__ y = (T*)a.y;
-    const int kq = a.K_pad / 4;
-    const size_t total = (size_t)a.N * a.P * a.Q * kq;
+    const int Wp = a.W + 2, P2i = (a.H + 2) * Wp, Qp = a.Q + 2, P2o = (a.P + 2) * Qp;
+    const size_t plane_i = (size_t)a.N * P2i, plane_o = (size_t)a.N * P2o;
+    const int kchunks = a.K_pad / 8, cchunks = a.C_pad / 8;
+    const size_t total = plane_o * kchunks;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int k4 = (int)(i % kq) * 4;
-        size_t t = i / kq;
-        const int q = (int)(t % a.Q); t /= a.Q;
-        const int p = (int)(t % a.P);
-        const size_t n = t / a.P;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int r = 0; r < a.R; ++r) {
-            const int ih = p * a.stride + r - a.pad;
-            if (ih < 0 || ih >= a.H) continue;
-            for (int s = 0; s < a.S; ++s) {
-                const int iw = q * a.stride + s - a.pad;
-                if (iw < 0 || iw >= a.W) continue;
-                const T* xp = x + ((n * a.H + ih) * a.W + iw) * a.C_pad;
+        const int jo = (int)(i / plane_o);
+        const size_t f = i - (size_t)jo * plane_o;
+        const size_t n = f / P2o;
+        const int rem = (int)(f - n * P2o);
+        const int p = rem / Qp - 1, q = rem % Qp - 1;
+        float acc[8];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const T* wp = w + (((size_t)(k4 + j) * a.R + r) * a.S + s) * a.C_pad;
-                    float sum = acc[j];
-                    for (int c = 0; c < a.C_pad; ++c) sum = fmaf(to_f<T>(xp[c]), to_f<T>(wp[c]), sum);
-                    acc[j] = sum;
+        for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+        const bool inside = p >= 0 && p < a.P && q >= 0 && q < a.Q;
+        if (inside) {
+            for (int r = 0; r < a.R; ++r) {
+                const int ih = p * a.stride + r - a.pad;
+                if (ih < 0 || ih >= a.H) continue;
+                for (int s = 0; s < a.S; ++s) {
+                    const int iw = q * a.stride + s - a.pad;
+                    if (iw < 0 || iw >= a.W) continue;
+                    const int tap = r * a.S + s;
+                    for (int jc = 0; jc < cchunks; ++jc) {
+                        const T* xp = x + ((size_t)jc * plane_i + n * P2i + (size_t)(ih + 1) * Wp + (iw + 1)) * 8;
+                        const T* wp = w + (((size_t)tap * cchunks + jc) * a.K_pad + (size_t)jo * 8) * 8;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            float sum = acc[e];
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) sum = fmaf(to_f<T>(xp[c]), to_f<T>(wp[e * 8 + c]), sum);
+                            acc[e] = sum;
+                        }
+                    }
                 }
             }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int k = jo * 8 + e;
+                float v = acc[e] + a.bias[k];
+                if (a.res_mode == 1) {
+                    v += to_f<T>(res[i * 8 + e]);
+                } else if (a.res_mode == 2) {
+                    const int c = k - a.res_pad_lo;
+                    if (c >= 0 && c < a.res_C) {
+                        const int rWp = a.res_W + 2, rP2 = (a.res_H + 2) * rWp;
+                        const size_t rv = (size_t)(c / 8) * a.N * rP2 + n * rP2 + (size_t)(p * a.res_stride + 1) * rWp +
+                                          (q * a.res_stride + 1);
+                        v += to_f<T>(res[rv * 8 + (c & 7)]);
+                    }
+                }
+                acc[e] = a.relu ? fmaxf(v, 0.0f) : v;
+            }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int k = k4 + j;
-            float v = acc[j] + a.bias[k];
-            if (a.res_mode == 1) {
-                v += to_f<T>(res[((n * a.P + p) * a.Q + q) * a.K_pad + k]);
-            } else if (a.res_mode == 2) {
-                const int c = k - a.res_pad_lo;
-                if (c >= 0 && c < a.res_C)
-                    v += to_f<T>(res[((n * a.res_H + p * a.res_stride) * a.res_W + q * a.res_stride) * a.res_C_pad + c]);
-            }
-            y[((n * a.P + p) * a.Q + q) * a.K_pad + k] = from_f<T>(a.relu ? fmaxf(v, 0.0f) : v);
-        }
+        for (int e = 0; e < 8; ++e) y[i * 8 + e] = from_f<T>(acc[e]);
     }
 }
 
+}  // namespace
+
 void launch_conv_simt(const ConvArgs& a, int is_bf16, cudaStream_t st) {
-    const size_t total = (size_t)a.N * a.P * a.Q * (a.K_pad / 4);
+    const size_t total = (size_t)a.N * (a.P + 2) * (a.Q + 2) * (a.K_pad / 8);
     size_t blocks = (total + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
     if (blocks < 1) blocks = 1;

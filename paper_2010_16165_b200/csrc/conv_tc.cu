@@ -1,18 +1,31 @@
-// Implicit-GEMM convolution for sm_100a: TMA-staged activation and filter tiles, tcgen05 BF16
-// MMA with FP32 accumulators in tensor memory, fused epilogue (folded-BN bias + shortcut +
-// ReLU, BF16 store).
+// Implicit-GEMM convolution for sm_100a: tcgen05 BF16 MMA with FP32 accumulators in tensor
+// memory, operands staged in shared memory by the bulk-copy (TMA) engine, fused epilogue
+// (folded-BN bias + shortcut + ReLU, BF16 store).  Activations use the planar-8 layout with a
+// zero border described in fp_internal.h.
 //
-//   GEMM view     M = N*P*Q output pixels, N = K_pad filters, K = R*S*C_pad.
-//   CTA tile      128 output pixels (a tile_w x tile_h x tile_n box of the NHWC output) x n_tile filters.
-//   K blocks      one filter tap (r,s) x kc channels (kc = 16/32/64 -> 32/64/128-byte swizzled rows).
-//                 The activation block of a tap is one 4-D TMA box of the NHWC input shifted by the
-//                 tap offset; out-of-range coordinates are zero-filled by the TMA unit, which is the
-//                 convolution's zero padding.  Strided convolutions use the tensor map's element strides.
-//   Warp roles    warp 0: TMA producer (one lane).  warp 1: tensor-memory allocation + MMA issue (one lane).
-//                 warps 2-5: epilogue, one thread per accumulator row (TMEM lane).
-//   Pipelines     `stages` shared-memory stages (full/empty mbarriers) between producer and MMA;
-//                 two accumulator stages in tensor memory (tmem_full/tmem_empty) between MMA and
-//                 epilogue, so the epilogue of tile i overlaps the MMAs of tile i+1.  Persistent CTAs.
+//   GEMM view     M = flat output positions (border positions included: they are computed and then
+//                 overwritten with zeros), N = K_pad filters, K = R*S*C_pad.
+//   CTA tile      128 consecutive flat positions x n_tile filters; persistent CTAs walk the tiles.
+//   Operands      K-major, no swizzle: an operand block is a stack of 16-byte rows (8 channels of
+//                 one position / one filter); the two 8-channel halves of a K=16 MMA step live in
+//                 two such stacks ("planes"), `LBO` apart.
+//   FLAT modes    stride-1 "same" convolutions (3x3 pad 1, 1x1 pad 0).  Because every chunk plane
+//                 is contiguous over flat positions, the activations a tile needs - its 128
+//                 positions plus a halo of (W+3) before and after - are ONE contiguous run per
+//                 chunk, fetched with one bulk copy.  The operand of filter tap (r,s) is the same
+//                 shared-memory block read from a start address shifted by (r-1)*(W+2)+(s-1) rows,
+//                 so each activation is fetched once per tile, not once per tap.  The zero border
+//                 in memory is the convolution's padding.  Filters either stay resident in shared
+//                 memory for the whole kernel (small banks) or are streamed per (tap, K block).
+//   GATHER mode   any other geometry (stride 2, 7x7, ...): 128 loader threads fetch the vectors of
+//                 their output position for each (tap, K block) with 16-byte loads, zero where the
+//                 window leaves the image.
+//   Warp roles    warp 0 lane 0: bulk-copy producer.  warp 1: tensor-memory allocation, lane 0 issues
+//                 the MMAs.  warps 2-5: epilogue, one thread per accumulator row.  warp 6 lane 0:
+//                 filter producer when filters are streamed in a FLAT mode.  warps 6-9: loader
+//                 threads in GATHER mode.
+//   Pipelines     full/empty mbarrier rings for the shared-memory stages; two accumulator stages in
+//                 tensor memory so the epilogue of one tile overlaps the MMAs of the next.
 //   Waits         every mbarrier wait is bounded; when one runs out the CTA raises a status word in
 //                 global memory, all roles leave their loops, tensor memory is released and the
 //                 kernel returns (results are then invalid and the host reports FP_ERR_TIMEOUT).
@@ -25,20 +38,20 @@ namespace fp {
 
 namespace {
 
-constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kWaitLimit = 1u << 24;          // polls per wait, and
 constexpr long long kWaitCycles = 2000000000LL;    // SM clock cycles per wait (about a second)
 
+enum { MODE_FLAT_RESIDENT = 0, MODE_FLAT_STREAM = 1, MODE_GATHER = 2 };
+
 struct TcParams {
     ConvArgs a;
-    int tile_w, tile_h, tile_n, tiles_w, tiles_h, tiles_n;
-    int kc, c_blocks, n_tile, n_tiles, stages;
-    int a_bytes, b_bytes;       // bytes per stage
-    int sbo;                    // byte distance between 8-row groups in a staged tile
-    int layout_type;            // shared-memory descriptor swizzle code
-    int tmem_cols;
-    int total_tiles;
+    int Wp_in, P2_in, Qp, P2_out;
+    long long plane_in, plane_out;      // vectors per chunk plane (N * P2)
+    long long m_total;                  // flat output positions
+    int taps, cchunks, cg, groups, halo, rows_a, a_stages, b_stages;
+    int n_tile, n_tiles, tmem_cols, total_tiles;
+    int a_stage_bytes, b_stage_bytes, b_bank_bytes;
     int* status;
 };
 
@@ -79,15 +92,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+// Contiguous global -> shared copy by the bulk-copy engine; completion is counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -114,44 +122,62 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor for a K-major operand tile whose rows are one swizzle span
-// wide: start address, leading offset 16 B, stride offset = 8 rows, descriptor version 1.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int sbo, int layout_type) {
+// Shared-memory matrix descriptor, K-major, no swizzle: rows of 16 bytes, 8 rows contiguous
+// (one 128-byte core matrix), `sbo` = 128 bytes between 8-row groups, `lbo` bytes between the two
+// 8-channel halves of a K=16 step.  Descriptor version 1 (bit 46).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo) {
     uint64_t d = 0;
     d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)(128 >> 4) << 32;
     d |= (uint64_t)1 << 46;
-    d |= (uint64_t)(layout_type & 7) << 61;
     return d;
 }
 
 // Shared-memory control block at the start of dynamic shared memory.
 struct Ctrl {
-    uint64_t full[kMaxStages];
-    uint64_t empty[kMaxStages];
+    uint64_t a_full[kMaxStages];
+    uint64_t a_empty[kMaxStages];
+    uint64_t b_full[kMaxStages];
+    uint64_t b_empty[kMaxStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
 
-__global__ void __launch_bounds__(kThreads)
-conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, const TcParams p) {
+__device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
+    atomicExch(&ctrl->abort_flag, 1);
+    atomicExch(status, code);
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(MODE == MODE_GATHER ? 320 : 224)
+conv_tc_kernel(const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
     const uint32_t ctrl_addr = smem_u32(smem_raw);
-    const uint32_t tiles_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + 1023u) & ~1023u;
+    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + 1023u) & ~1023u;
+    const uint32_t b_region = MODE == MODE_FLAT_RESIDENT ? (uint32_t)p.b_bank_bytes
+                              : MODE == MODE_FLAT_STREAM ? (uint32_t)(p.b_stages * p.b_stage_bytes) : 0u;
+    const uint32_t a_base = b_base + ((b_region + 127u) & ~127u);
     volatile int* abort_flag = &ctrl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = ctrl_addr + (uint32_t)offsetof(Ctrl, full);
-    const uint32_t empty0 = ctrl_addr + (uint32_t)offsetof(Ctrl, empty);
+    const uint32_t a_full0 = ctrl_addr + (uint32_t)offsetof(Ctrl, a_full);
+    const uint32_t a_empty0 = ctrl_addr + (uint32_t)offsetof(Ctrl, a_empty);
+    const uint32_t b_full0 = ctrl_addr + (uint32_t)offsetof(Ctrl, b_full);
+    const uint32_t b_empty0 = ctrl_addr + (uint32_t)offsetof(Ctrl, b_empty);
     const uint32_t tfull0 = ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_full);
     const uint32_t tempty0 = ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_empty);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(a_full0 + 8 * s, MODE == MODE_GATHER ? 129 : 1);   // gather: 128 loaders + the filter producer
+            mbar_init(a_empty0 + 8 * s, 1);
+            mbar_init(b_full0 + 8 * s, 1);
+            mbar_init(b_empty0 + 8 * s, 1);
+        }
         for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 128); }
         ctrl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -167,179 +193,317 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
 
-    const int taps = p.a.R * p.a.S;
-    const int kblocks = taps * p.c_blocks;
-    const int stage_bytes = p.a_bytes + p.b_bytes;
+    const uint4* __restrict__ xv = reinterpret_cast<const uint4*>(p.a.x);
+    const uint4* __restrict__ wv = reinterpret_cast<const uint4*>(p.a.w);
 
     if (warp == 0) {
-        // ------------------------------ TMA producer ------------------------------
+        // ------------------------------ bulk-copy producer ------------------------------
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                int t = tile;
-                const int nt = t % p.n_tiles; t /= p.n_tiles;
-                const int tw = t % p.tiles_w; t /= p.tiles_w;
-                const int th = t % p.tiles_h; t /= p.tiles_h;
-                const int tn = t;
-                const int x0 = tw * p.tile_w * p.a.stride - p.a.pad;
-                const int y0 = th * p.tile_h * p.a.stride - p.a.pad;
-                const int n0 = tn * p.tile_n;
-                for (int tap = 0; tap < taps && ok; ++tap) {
-                    const int r = tap / p.a.S, s = tap - r * p.a.S;
-                    for (int cb = 0; cb < p.c_blocks; ++cb) {
-                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                        const uint32_t fb = full0 + 8 * stage;
-                        const uint32_t sa = tiles_base + stage * stage_bytes;
-                        mbar_expect_tx(fb, (uint32_t)stage_bytes);
-                        tma_load_4d(sa, &tm_x, fb, cb * p.kc, x0 + s, y0 + r, n0);
-                        tma_load_3d(sa + p.a_bytes, &tm_w, fb, cb * p.kc, tap, nt * p.n_tile);
-                        if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+            if (MODE == MODE_FLAT_RESIDENT) {
+                // the whole filter bank, once
+                mbar_expect_tx(b_full0, (uint32_t)p.b_bank_bytes);
+                for (int off = 0; off < p.b_bank_bytes; off += 32768) {
+                    const int n = p.b_bank_bytes - off < 32768 ? p.b_bank_bytes - off : 32768;
+                    bulk_copy(b_base + off, reinterpret_cast<const uint8_t*>(p.a.w) + off, (uint32_t)n, b_full0);
+                }
+            }
+            uint32_t stage = 0, phase = 0;
+            if (MODE != MODE_GATHER) {
+                for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+                    const long long f0 = (long long)(tile / p.n_tiles) * 128;
+                    for (int g = 0; g < p.groups; ++g) {
+                        if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        int cgg = p.cchunks - g * p.cg;
+                        if (cgg > p.cg) cgg = p.cg;
+                        const uint32_t fb = a_full0 + 8 * stage;
+                        const uint32_t dst = a_base + stage * p.a_stage_bytes;
+                        mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
+                        for (int c = 0; c < cgg; ++c)
+                            bulk_copy(dst + c * p.rows_a * 16, xv + (long long)(g * p.cg + c) * p.plane_in + f0 - p.halo,
+                                      (uint32_t)(p.rows_a * 16), fb);
+                        if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
+                    }
+                }
+            } else {
+                // GATHER: filters of each (tap, K block) into the stage the loader threads fill
+                for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+                    const int nt = tile % p.n_tiles;
+                    int nrows = p.a.K_pad - nt * p.n_tile;
+                    if (nrows > p.n_tile) nrows = p.n_tile;
+                    for (int tap = 0; tap < p.taps && ok; ++tap) {
+                        for (int g = 0; g < p.groups; ++g) {
+                            if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                            int cgg = p.cchunks - g * p.cg;
+                            if (cgg > p.cg) cgg = p.cg;
+                            const uint32_t fb = a_full0 + 8 * stage;
+                            const uint32_t dst = a_base + stage * (p.a_stage_bytes + p.b_stage_bytes) + p.a_stage_bytes;
+                            mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
+                            for (int c = 0; c < cgg; ++c)
+                                bulk_copy(dst + c * p.n_tile * 16,
+                                          wv + ((long long)tap * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
+                                          (uint32_t)(nrows * 16), fb);
+                            if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
+                        }
                     }
                 }
             }
-            if (!ok) { atomicExch((int*)&ctrl->abort_flag, 1); atomicExch(p.status, 1); }
+            if (!ok) raise(ctrl, p.status, 1);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------
         if (lane == 0) {
             // instruction descriptor: D = f32, A = B = bf16, both K-major, N = n_tile, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
-            uint32_t stage = 0, phase = 0;
-            uint32_t acc_phase[2] = {0, 0};
+            uint32_t a_stage = 0, a_phase = 0, b_stage = 0, b_phase = 0;
+            uint32_t acc_phase0 = 0, acc_phase1 = 0;
             int local = 0;
             bool ok = true;
+            if (MODE == MODE_FLAT_RESIDENT) ok = mbar_wait(b_full0, 0, abort_flag);
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
-                if (!mbar_wait(tempty0 + 8 * acc, acc_phase[acc] ^ 1, abort_flag)) { ok = false; break; }
-                acc_phase[acc] ^= 1;
+                const uint32_t ph = acc ? acc_phase1 : acc_phase0;
+                if (!mbar_wait(tempty0 + 8 * acc, ph ^ 1, abort_flag)) { ok = false; break; }
+                if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
                 tc_fence_after();
+                const int nt = tile % p.n_tiles;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.n_tile);
                 uint32_t accumulate = 0;
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const int cb = kb % p.c_blocks;
-                    int ksteps = (p.a.C_pad - cb * p.kc);
-                    ksteps = (ksteps < p.kc ? ksteps : p.kc) >> 4;
-                    const uint32_t sa = tiles_base + stage * stage_bytes;
-                    const uint32_t sb = sa + p.a_bytes;
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        const uint64_t da = make_smem_desc(sa + ks * 32, p.sbo, p.layout_type);
-                        const uint64_t db = make_smem_desc(sb + ks * 32, p.sbo, p.layout_type);
-                        umma_bf16(d_tmem, da, db, idesc, accumulate);
-                        accumulate = 1;
+                if (MODE != MODE_GATHER) {
+                    for (int g = 0; g < p.groups && ok; ++g) {
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        int cgg = p.cchunks - g * p.cg;
+                        if (cgg > p.cg) cgg = p.cg;
+                        const uint32_t sa = a_base + a_stage * p.a_stage_bytes;
+                        for (int tap = 0; tap < p.taps; ++tap) {
+                            const int r = tap / p.a.S, s = tap - r * p.a.S;
+                            const int row_off = p.halo + (r - p.a.pad) * p.Wp_in + (s - p.a.pad);
+                            uint32_t sb, lbo_b;
+                            if (MODE == MODE_FLAT_RESIDENT) {
+                                sb = b_base + (uint32_t)((((tap * p.cchunks) + g * p.cg) * p.a.K_pad + nt * p.n_tile) * 16);
+                                lbo_b = (uint32_t)(p.a.K_pad * 16);
+                            } else {
+                                if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag)) { ok = false; break; }
+                                tc_fence_after();
+                                sb = b_base + b_stage * p.b_stage_bytes;
+                                lbo_b = (uint32_t)(p.n_tile * 16);
+                            }
+                            for (int ks = 0; ks < cgg / 2; ++ks) {
+                                const uint64_t da = make_smem_desc(sa + (uint32_t)((2 * ks * p.rows_a + row_off) * 16),
+                                                                   (uint32_t)(p.rows_a * 16));
+                                const uint64_t db = make_smem_desc(sb + (uint32_t)(2 * ks) * lbo_b, lbo_b);
+                                umma_bf16(d_tmem, da, db, idesc, accumulate);
+                                accumulate = 1;
+                            }
+                            if (MODE == MODE_FLAT_STREAM) {
+                                umma_commit(b_empty0 + 8 * b_stage);
+                                if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
+                            }
+                        }
+                        if (!ok) break;
+                        umma_commit(a_empty0 + 8 * a_stage);     // releases the stage once these MMAs have read it
+                        if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
                     }
-                    umma_commit(empty0 + 8 * stage);     // releases the stage once these MMAs have read it
-                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                } else {
+                    const int kblocks = p.taps * p.groups;
+                    const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const int g = kb % p.groups;
+                        int cgg = p.cchunks - g * p.cg;
+                        if (cgg > p.cg) cgg = p.cg;
+                        const uint32_t sa = a_base + a_stage * stage_bytes;
+                        const uint32_t sb = sa + p.a_stage_bytes;
+                        for (int ks = 0; ks < cgg / 2; ++ks) {
+                            const uint64_t da = make_smem_desc(sa + (uint32_t)(2 * ks * 128 * 16), 128 * 16);
+                            const uint64_t db = make_smem_desc(sb + (uint32_t)(2 * ks * p.n_tile * 16), (uint32_t)(p.n_tile * 16));
+                            umma_bf16(d_tmem, da, db, idesc, accumulate);
+                            accumulate = 1;
+                        }
+                        umma_commit(a_empty0 + 8 * a_stage);
+                        if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
+                    }
                 }
                 if (ok) umma_commit(tfull0 + 8 * acc);   // accumulator complete
             }
-            if (!ok) { atomicExch((int*)&ctrl->abort_flag, 1); atomicExch(p.status, 2); }
+            if (!ok) raise(ctrl, p.status, 2);
         }
-    } else {
+    } else if (warp < 6) {
         // ------------------------------ epilogue ----------------------------------
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 belong to this warp
-        const int row = quarter * 32 + lane;          // accumulator row = pixel within the tile
-        const int w_l = row % p.tile_w;
-        const int h_l = (row / p.tile_w) % p.tile_h;
-        const int n_l = row / (p.tile_w * p.tile_h);
-        uint32_t acc_phase[2] = {0, 0};
+        const int row = quarter * 32 + lane;          // accumulator row = position within the tile
+        uint32_t acc_phase0 = 0, acc_phase1 = 0;
         int local = 0;
         bool ok = true;
-        const __nv_bfloat16* __restrict__ res = (const __nv_bfloat16*)p.a.res;
-        __nv_bfloat16* __restrict__ y = (__nv_bfloat16*)p.a.y;
+        const uint4* __restrict__ res = reinterpret_cast<const uint4*>(p.a.res);
+        const __nv_bfloat16* __restrict__ res_s = reinterpret_cast<const __nv_bfloat16*>(p.a.res);
+        uint4* __restrict__ y = reinterpret_cast<uint4*>(p.a.y);
         for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++local) {
-            int t = tile;
-            const int nt = t % p.n_tiles; t /= p.n_tiles;
-            const int tw = t % p.tiles_w; t /= p.tiles_w;
-            const int th = t % p.tiles_h; t /= p.tiles_h;
-            const int tn = t;
-            const int q = tw * p.tile_w + w_l, pp = th * p.tile_h + h_l, n = tn * p.tile_n + n_l;
-            const bool valid = q < p.a.Q && pp < p.a.P && n < p.a.N;
+            const int nt = tile % p.n_tiles;
+            const long long f = (long long)(tile / p.n_tiles) * 128 + row;
+            const bool exists = f < p.m_total;
+            const int n = (int)(f / p.P2_out);
+            const int rem = (int)(f - (long long)n * p.P2_out);
+            const int hp = rem / p.Qp, wq = rem - hp * p.Qp;
+            const bool interior = exists && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
             const int acc = local & 1;
-            ok = mbar_wait(tfull0 + 8 * acc, acc_phase[acc], abort_flag);
+            const uint32_t ph = acc ? acc_phase1 : acc_phase0;
+            ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            acc_phase[acc] ^= 1;
+            if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
             tc_fence_after();
             const int k_base = nt * p.n_tile;
             int cols = p.a.K_pad - k_base;
             if (cols > p.n_tile) cols = p.n_tile;
-            const size_t out_off = (((size_t)n * p.a.P + pp) * p.a.Q + q) * p.a.K_pad + k_base;
-            size_t res_off = 0;
-            if (p.a.res_mode == 2)
-                res_off = (((size_t)n * p.a.res_H + (size_t)pp * p.a.res_stride) * p.a.res_W + (size_t)q * p.a.res_stride) * p.a.res_C_pad;
+            long long res_vec = 0;
+            if (p.a.res_mode == 2) {
+                const int rWp = p.a.res_W + 2, rP2 = (p.a.res_H + 2) * rWp;
+                res_vec = (long long)n * rP2 + (long long)((hp - 1) * p.a.res_stride + 1) * rWp + ((wq - 1) * p.a.res_stride + 1);
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.n_tile);
             for (int c0 = 0; c0 < cols; c0 += 16) {
                 uint32_t v[16];
+                __syncwarp();
                 tmem_ld16(taddr + c0, v);
                 tmem_ld_wait();
-                if (valid) {
-                    float f[16];
+                if (exists) {
+                const long long out_vec = (long long)((k_base + c0) >> 3) * p.plane_out + f;
+                uint4 o[2];
+                o[0] = make_uint4(0, 0, 0, 0);
+                o[1] = o[0];
+                if (interior) {
+                    float fv[16];
                     const float4* b4 = reinterpret_cast<const float4*>(p.a.bias + k_base + c0);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float4 b = __ldg(b4 + i);
-                        f[4 * i + 0] = __uint_as_float(v[4 * i + 0]) + b.x;
-                        f[4 * i + 1] = __uint_as_float(v[4 * i + 1]) + b.y;
-                        f[4 * i + 2] = __uint_as_float(v[4 * i + 2]) + b.z;
-                        f[4 * i + 3] = __uint_as_float(v[4 * i + 3]) + b.w;
+                        fv[4 * i + 0] = __uint_as_float(v[4 * i + 0]) + b.x;
+                        fv[4 * i + 1] = __uint_as_float(v[4 * i + 1]) + b.y;
+                        fv[4 * i + 2] = __uint_as_float(v[4 * i + 2]) + b.z;
+                        fv[4 * i + 3] = __uint_as_float(v[4 * i + 3]) + b.w;
                     }
                     if (p.a.res_mode == 1) {
-                        const uint4* rp = reinterpret_cast<const uint4*>(res + out_off + c0);
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
-                            const uint4 raw = __ldg(rp + hh);
+                            const uint4 raw = __ldg(res + out_vec + hh * p.plane_out);
                             const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const float2 g = __bfloat1622float2(h2[i]);
-                                f[8 * hh + 2 * i] += g.x;
-                                f[8 * hh + 2 * i + 1] += g.y;
+                                fv[8 * hh + 2 * i] += g.x;
+                                fv[8 * hh + 2 * i + 1] += g.y;
                             }
                         }
                     } else if (p.a.res_mode == 2) {
                         // shortcut by subsampling: output channel k takes input channel k - pad_lo
-                        const int cs = k_base + c0 - p.a.res_pad_lo;
-                        if (cs >= 0 && cs + 16 <= p.a.res_C && (cs & 7) == 0) {
-                            const uint4* rp = reinterpret_cast<const uint4*>(res + res_off + cs);
+                        const long long rplane = (long long)p.a.N * (p.a.res_H + 2) * (p.a.res_W + 2);
 #pragma unroll
-                            for (int hh = 0; hh < 2; ++hh) {
-                                const uint4 raw = __ldg(rp + hh);
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const int cs = k_base + c0 + 8 * hh - p.a.res_pad_lo;
+                            if (cs >= 0 && cs + 8 <= p.a.res_C_pad && (cs & 7) == 0) {
+                                const uint4 raw = __ldg(res + (long long)(cs >> 3) * rplane + res_vec);
                                 const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
                                     const float2 g = __bfloat1622float2(h2[i]);
-                                    f[8 * hh + 2 * i] += g.x;
-                                    f[8 * hh + 2 * i + 1] += g.y;
+                                    fv[8 * hh + 2 * i] += g.x;
+                                    fv[8 * hh + 2 * i + 1] += g.y;
                                 }
-                            }
-                        } else if (cs + 16 > 0 && cs < p.a.res_C) {
+                            } else if (cs + 8 > 0 && cs < p.a.res_C) {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int c = cs + i;
-                                if (c >= 0 && c < p.a.res_C) f[i] += __bfloat162float(res[res_off + c]);
+                                for (int i = 0; i < 8; ++i) {
+                                    const int c = cs + i;
+                                    if (c >= 0 && c < p.a.res_C)
+                                        fv[8 * hh + i] += __bfloat162float(res_s[((long long)(c >> 3) * rplane + res_vec) * 8 + (c & 7)]);
+                                }
                             }
                         }
                     }
                     if (p.a.relu) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) f[i] = fmaxf(f[i], 0.0f);
+                        for (int i = 0; i < 16; ++i) fv[i] = fmaxf(fv[i], 0.0f);
                     }
-                    uint4 o[2];
                     __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(o);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) o2[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-                    uint4* yp = reinterpret_cast<uint4*>(y + out_off + c0);
-                    yp[0] = o[0];
-                    yp[1] = o[1];
+                    for (int i = 0; i < 8; ++i) o2[i] = __floats2bfloat162_rn(fv[2 * i], fv[2 * i + 1]);
+                }
+                y[out_vec] = o[0];
+                y[out_vec + p.plane_out] = o[1];
                 }
             }
             tc_fence_before();
             mbar_arrive(tempty0 + 8 * acc);
         }
-        if (!ok && lane == 0) { atomicExch((int*)&ctrl->abort_flag, 1); atomicExch(p.status, 3); }
+        if (!ok && lane == 0) raise(ctrl, p.status, 3);
+    } else if (MODE == MODE_FLAT_STREAM) {
+        // ------------------------------ filter producer (streamed filters) --------------
+        if (warp == 6 && lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+                const int nt = tile % p.n_tiles;
+                int nrows = p.a.K_pad - nt * p.n_tile;
+                if (nrows > p.n_tile) nrows = p.n_tile;
+                for (int g = 0; g < p.groups && ok; ++g) {
+                    int cgg = p.cchunks - g * p.cg;
+                    if (cgg > p.cg) cgg = p.cg;
+                    for (int tap = 0; tap < p.taps; ++tap) {
+                        if (!mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        const uint32_t fb = b_full0 + 8 * stage;
+                        const uint32_t dst = b_base + stage * p.b_stage_bytes;
+                        mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
+                        for (int c = 0; c < cgg; ++c)
+                            bulk_copy(dst + c * p.n_tile * 16,
+                                      wv + ((long long)tap * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
+                                      (uint32_t)(nrows * 16), fb);
+                        if (++stage == (uint32_t)p.b_stages) { stage = 0; phase ^= 1; }
+                    }
+                }
+            }
+            if (!ok) raise(ctrl, p.status, 4);
+        }
+    } else if (MODE == MODE_GATHER) {
+        // ------------------------------ loader threads (gathered activations) -----------
+        const int m = threadIdx.x - 192;             // 0..127: row of the tile this thread fills
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+        for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+            const long long f = (long long)(tile / p.n_tiles) * 128 + m;
+            const int n = (int)(f / p.P2_out);
+            const int rem = (int)(f - (long long)n * p.P2_out);
+            const int hp = rem / p.Qp, wq = rem - hp * p.Qp;
+            const bool interior = f < p.m_total && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
+            const int ih0 = (hp - 1) * p.a.stride - p.a.pad, iw0 = (wq - 1) * p.a.stride - p.a.pad;
+            for (int tap = 0; tap < p.taps && ok; ++tap) {
+                const int r = tap / p.a.S, s = tap - r * p.a.S;
+                const int ih = ih0 + r, iw = iw0 + s;
+                const bool valid = interior && ih >= 0 && ih < p.a.H && iw >= 0 && iw < p.a.W;
+                const long long src = (long long)n * p.P2_in + (long long)(ih + 1) * p.Wp_in + (iw + 1);
+                for (int g = 0; g < p.groups; ++g) {
+                    int cgg = p.cchunks - g * p.cg;
+                    if (cgg > p.cg) cgg = p.cg;
+                    uint4 v[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        v[c] = make_uint4(0, 0, 0, 0);
+                        if (valid && c < cgg) v[c] = __ldg(xv + (long long)(g * p.cg + c) * p.plane_in + src);
+                    }
+                    if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                    uint8_t* dst = smem_raw + (a_base - ctrl_addr) + stage * stage_bytes + m * 16;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        if (c < cgg) *reinterpret_cast<uint4*>(dst + c * 128 * 16) = v[c];
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> MMA reads
+                    mbar_arrive(a_full0 + 8 * stage);
+                    if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+        if (!ok) raise(ctrl, p.status, 5);
     }
 
     // ---- teardown: everyone arrives here, also after a wait that ran out ----
@@ -356,109 +520,91 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
 int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
+
+constexpr unsigned kSmemMax = 232448u - 1024u;     // opt-in dynamic shared memory per CTA
+constexpr unsigned kSmemPerSm = 233472u;           // 228 KB per SM
 
 }  // namespace
 
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len) {
     memset(plan, 0, sizeof(*plan));
-    EncodeTiledFn encode = get_encode();
-    if (!encode) { snprintf(err, err_len, "cuTensorMapEncodeTiled is not available"); return 1; }
     if (a.C_pad % 16 || a.K_pad % 16) { snprintf(err, err_len, "channel counts must be padded to 16"); return 1; }
-    if (a.stride < 1 || a.stride > 8) { snprintf(err, err_len, "stride %d not supported", a.stride); return 1; }
-
-    // --- pixel tile: tile_w x tile_h x tile_n = 128 ---
-    int tw = pow2_at_least(a.Q < 128 ? a.Q : 128);
-    if (tw < 8) tw = 8;
-    while (tw * a.stride > 256) tw >>= 1;
-    int th = pow2_at_least(a.P < 128 / tw ? a.P : 128 / tw);
-    if (th > 128 / tw) th = 128 / tw;
-    while (th * a.stride > 256) th >>= 1;
-    int tn = 128 / (tw * th);
-    plan->tile_w = tw; plan->tile_h = th; plan->tile_n = tn;
-    plan->tiles_w = (a.Q + tw - 1) / tw;
-    plan->tiles_h = (a.P + th - 1) / th;
-    plan->tiles_n = (a.N + tn - 1) / tn;
-
-    // --- K blocking ---
-    plan->kc = a.C_pad >= 64 ? 64 : a.C_pad >= 32 ? 32 : 16;
-    if (a.C_pad == 48) plan->kc = 16;           // three exact 16-channel blocks instead of 64 with padding
-    plan->c_blocks = (a.C_pad + plan->kc - 1) / plan->kc;
-    plan->swizzle_bytes = plan->kc * 2;
+    if (a.W > kMaxWidth || a.Q > kMaxWidth) { snprintf(err, err_len, "images wider than %d are not supported", kMaxWidth); return 1; }
+    const int cchunks = a.C_pad / 8;
+    const int taps = a.R * a.S;
+    plan->flat = (a.stride == 1 && a.R == a.S && a.P == a.H && a.Q == a.W &&
+                  ((a.R == 1 && a.pad == 0) || (a.R == 3 && a.pad == 1))) ? 1 : 0;
+    plan->cg = cchunks < 8 ? cchunks : 8;
+    plan->groups = (cchunks + plan->cg - 1) / plan->cg;
+    const long long m_total = (long long)a.N * (a.P + 2) * (a.Q + 2);
+    const long long m_tiles = (m_total + 127) / 128;
 
     // --- filter tile ---
     int n_tiles = (a.K_pad + 255) / 256;
-    int n_tile = ((a.K_pad + n_tiles - 1) / n_tiles + 15) / 16 * 16;
-    const long m_tiles = (long)plan->tiles_w * plan->tiles_h * plan->tiles_n;
-    while (m_tiles * n_tiles < 148 && n_tile > 64) {      // few pixel tiles: split filters further to fill the SMs
-        n_tiles *= 2;
-        n_tile = ((a.K_pad + n_tiles - 1) / n_tiles + 15) / 16 * 16;
+    int n_tile = round_up_i((a.K_pad + n_tiles - 1) / n_tiles, 16);
+    const long long bank = (long long)taps * a.C_pad * a.K_pad * 2;
+    const bool bank_fits = plan->flat && n_tiles == 1 && bank <= 100 * 1024;
+    if (!bank_fits) {
+        while (m_tiles * n_tiles < 148 && n_tile > 64) {      // few position tiles: split the filters to fill the SMs
+            n_tiles *= 2;
+            n_tile = round_up_i((a.K_pad + n_tiles - 1) / n_tiles, 16);
+        }
     }
     n_tiles = (a.K_pad + n_tile - 1) / n_tile;
     plan->n_tile = n_tile; plan->n_tiles = n_tiles;
     plan->tmem_cols = pow2_at_least(2 * n_tile < 32 ? 32 : 2 * n_tile);
-
-    // --- shared memory ---
-    const int a_bytes = 128 * plan->kc * 2;
-    const int b_bytes = n_tile * plan->kc * 2;
-    int stages = (200 * 1024) / (a_bytes + b_bytes);
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) { snprintf(err, err_len, "tile does not fit shared memory"); return 1; }
-    plan->stages = stages;
-    unsigned smem = (unsigned)(sizeof(Ctrl) + 1024 + (size_t)stages * (a_bytes + b_bytes));
-    // co-resident CTAs must not ask for more than the 512 tensor-memory columns of an SM
     const int tmem_ctas = 512 / plan->tmem_cols;
-    const unsigned min_smem = 232448u / (unsigned)(tmem_ctas + 1) + 1u;
-    if (smem < min_smem && tmem_ctas < 16) smem = min_smem;
-    plan->smem_bytes = smem;
-    int ctas_per_sm = (int)(232448u / (smem + 1024u));
-    if (ctas_per_sm > tmem_ctas) ctas_per_sm = tmem_ctas;
-    if (ctas_per_sm > 4) ctas_per_sm = 4;
-    if (ctas_per_sm < 1) ctas_per_sm = 1;
-    plan->grid = 148 * ctas_per_sm;
 
-    // --- tensor maps ---
-    const CUtensorMapSwizzle sw = plan->swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                  : plan->swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-    {
-        cuuint64_t dims[4] = {(cuuint64_t)a.C_pad, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)a.N};
-        cuuint64_t strides[3] = {(cuuint64_t)a.C_pad * 2, (cuuint64_t)a.W * a.C_pad * 2, (cuuint64_t)a.H * a.W * a.C_pad * 2};
-        cuuint32_t box[4] = {(cuuint32_t)plan->kc, (cuuint32_t)(tw * a.stride), (cuuint32_t)(th * a.stride), (cuuint32_t)tn};
-        cuuint32_t estr[4] = {1, (cuuint32_t)a.stride, (cuuint32_t)a.stride, 1};
-        CUresult r = encode(&plan->tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(a.x), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) { snprintf(err, err_len, "activation tensor map rejected (CUresult %d)", (int)r); return 1; }
+    unsigned smem = (unsigned)sizeof(Ctrl) + 1024u;
+    int want_ctas = 1;
+    if (plan->flat) {
+        plan->halo = a.pad * (a.W + 3);
+        plan->rows_a = round_up_i(128 + 2 * plan->halo, 8);
+        const unsigned a_stage = (unsigned)(plan->cg * plan->rows_a * 16);
+        if (bank_fits) {
+            plan->b_resident = 1;
+            plan->b_stages = 1;
+            plan->a_stages = 4;
+            unsigned fixed = smem + (unsigned)round_up_i((int)bank, 128);
+            while (plan->a_stages > 2 && fixed + plan->a_stages * a_stage > 110 * 1024) --plan->a_stages;
+            smem = fixed + plan->a_stages * a_stage;
+        } else {
+            plan->b_resident = 0;
+            plan->b_stages = 4;
+            const unsigned b_stage = (unsigned)(plan->cg * n_tile * 16);
+            plan->a_stages = 3;
+            while (plan->a_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->a_stages;
+            while (plan->b_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->b_stages;
+            smem += (unsigned)round_up_i((int)(plan->b_stages * b_stage), 128) + plan->a_stages * a_stage;
+        }
+        want_ctas = 4;
+    } else {
+        const unsigned stage = (unsigned)(plan->cg * 128 * 16 + plan->cg * n_tile * 16);
+        plan->a_stages = 6;
+        while (plan->a_stages > 2 && smem + plan->a_stages * stage > 120 * 1024) --plan->a_stages;
+        plan->b_stages = plan->a_stages;
+        smem += plan->a_stages * stage;
+        want_ctas = 2;
     }
-    {
-        cuuint64_t dims[3] = {(cuuint64_t)a.C_pad, (cuuint64_t)(a.R * a.S), (cuuint64_t)a.K_pad};
-        cuuint64_t strides[2] = {(cuuint64_t)a.C_pad * 2, (cuuint64_t)a.R * a.S * a.C_pad * 2};
-        cuuint32_t box[3] = {(cuuint32_t)plan->kc, 1, (cuuint32_t)n_tile};
-        cuuint32_t estr[3] = {1, 1, 1};
-        CUresult r = encode(&plan->tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(a.w), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) { snprintf(err, err_len, "filter tensor map rejected (CUresult %d)", (int)r); return 1; }
-    }
+    if (smem > kSmemMax) { snprintf(err, err_len, "tile does not fit shared memory (%u bytes)", smem); return 1; }
+    // co-resident CTAs must not ask for more than the 512 tensor-memory columns of an SM
+    const unsigned min_smem = kSmemPerSm / (unsigned)(tmem_ctas + 1) + 1u;
+    if (tmem_ctas < 16 && smem < min_smem) smem = min_smem;
+    plan->smem_bytes = smem;
+    int ctas = (int)(kSmemPerSm / (smem + 1024u));
+    if (ctas > tmem_ctas) ctas = tmem_ctas;
+    if (ctas > want_ctas) ctas = want_ctas;
+    if (ctas < 1) ctas = 1;
+    plan->ctas_per_sm = ctas;
+
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024) != cudaSuccess) {
+        cudaError_t e0 = cudaFuncSetAttribute(conv_tc_kernel<MODE_FLAT_RESIDENT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        cudaError_t e1 = cudaFuncSetAttribute(conv_tc_kernel<MODE_FLAT_STREAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        cudaError_t e2 = cudaFuncSetAttribute(conv_tc_kernel<MODE_GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
+        if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess) {
             snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
             cudaGetLastError();
             return 1;
@@ -471,21 +617,28 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
 
 void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st) {
     TcParams p;
+    memset(&p, 0, sizeof(p));
     p.a = a;
-    p.tile_w = plan.tile_w; p.tile_h = plan.tile_h; p.tile_n = plan.tile_n;
-    p.tiles_w = plan.tiles_w; p.tiles_h = plan.tiles_h;
-    p.tiles_n = (a.N + plan.tile_n - 1) / plan.tile_n;
-    p.kc = plan.kc; p.c_blocks = plan.c_blocks; p.n_tile = plan.n_tile; p.n_tiles = plan.n_tiles; p.stages = plan.stages;
-    p.a_bytes = 128 * plan.kc * 2;
-    p.b_bytes = plan.n_tile * plan.kc * 2;
-    p.sbo = 8 * plan.kc * 2;
-    p.layout_type = plan.swizzle_bytes == 128 ? 2 : plan.swizzle_bytes == 64 ? 4 : 6;
-    p.tmem_cols = plan.tmem_cols;
-    p.total_tiles = p.tiles_w * p.tiles_h * p.tiles_n * p.n_tiles;
+    p.Wp_in = a.W + 2; p.P2_in = (a.H + 2) * (a.W + 2);
+    p.Qp = a.Q + 2; p.P2_out = (a.P + 2) * (a.Q + 2);
+    p.plane_in = (long long)a.N * p.P2_in;
+    p.plane_out = (long long)a.N * p.P2_out;
+    p.m_total = p.plane_out;
+    p.taps = a.R * a.S; p.cchunks = a.C_pad / 8; p.cg = plan.cg; p.groups = plan.groups;
+    p.halo = plan.halo; p.rows_a = plan.rows_a; p.a_stages = plan.a_stages; p.b_stages = plan.b_stages;
+    p.n_tile = plan.n_tile; p.n_tiles = plan.n_tiles; p.tmem_cols = plan.tmem_cols;
+    const long long m_tiles = (p.m_total + 127) / 128;
+    p.total_tiles = (int)(m_tiles * plan.n_tiles);
+    p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : plan.cg * 128 * 16;
+    p.b_stage_bytes = plan.cg * plan.n_tile * 16;
+    p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
     p.status = d_status;
-    int grid = plan.grid < p.total_tiles ? plan.grid : p.total_tiles;
+    int grid = 148 * plan.ctas_per_sm;
+    if (grid > p.total_tiles) grid = p.total_tiles;
     if (grid < 1) grid = 1;
-    conv_tc_kernel<<<grid, kThreads, plan.smem_bytes, st>>>(plan.tm_x, plan.tm_w, p);
+    if (!plan.flat) conv_tc_kernel<MODE_GATHER><<<grid, 320, plan.smem_bytes, st>>>(p);
+    else if (plan.b_resident) conv_tc_kernel<MODE_FLAT_RESIDENT><<<grid, 224, plan.smem_bytes, st>>>(p);
+    else conv_tc_kernel<MODE_FLAT_STREAM><<<grid, 224, plan.smem_bytes, st>>>(p);
 }
 
 }  // namespace fp

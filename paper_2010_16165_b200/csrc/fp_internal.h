@@ -1,4 +1,16 @@
 // Internal declarations shared by the host graph builder and the kernel launchers.
+//
+// Activation layout ("planar-8 with border"): channels are grouped in chunks of 8 (one 16-byte
+// vector of bf16, or 32 bytes of fp32); every image carries a one-pixel border of zeros.
+// For a batch of N images of H x W pixels and C_pad channels the vector of chunk j, image n,
+// pixel (h, w) sits at vector index
+//       j * (N * P2)  +  n * P2  +  (h + 1) * (W + 2)  +  (w + 1),      P2 = (H + 2) * (W + 2).
+// So each chunk is one contiguous plane over the whole batch; a run of consecutive "flat
+// positions" f = n*P2 + (h+1)*(W+2) + (w+1) is contiguous in memory for every chunk, and the
+// 3x3 neighbourhood of position f is f + dr*(W+2) + ds.  Every kernel that writes a tensor
+// writes all of its positions, zeros on the border, so the border never has to be cleared.
+// Buffers carry `kGuardVectors` vectors of slack before and after the data, because tiles of
+// flat positions read a halo that may start before the first plane or end after the last.
 #pragma once
 
 #include <cuda.h>
@@ -9,14 +21,17 @@
 
 namespace fp {
 
+constexpr int kGuardVectors = 1024;   // >= 128 + (W + 3) + 8 for every supported width (W <= 512)
+constexpr int kMaxWidth = 512;
+
 // ---------------------------------------------------------------------------------------
 // Convolution launch description (one fused operator: conv + bias + residual + ReLU)
 // ---------------------------------------------------------------------------------------
 struct ConvArgs {
-    const void* x;        // NHWC activations [N][H][W][C_pad]   (bf16 or fp32)
-    void* y;              // NHWC output      [N][P][Q][K_pad]
+    const void* x;        // input activations, planar-8 with border (vector 0 of plane 0)
+    void* y;              // output activations, same layout, P x Q pixels, K_pad channels
     const void* res;      // residual operand or nullptr
-    const void* w;        // packed filters   [K_pad][R][S][C_pad]
+    const void* w;        // packed filters [R*S][C_pad/8][K_pad][8]
     const float* bias;    // [K_pad]
     int N, H, W, C_pad, P, Q, K_pad, R, S, stride, pad;
     int relu;
@@ -37,42 +52,44 @@ void launch_identity_filters(float* dst, int C_dst, int R, int S, int k0, int c0
 void launch_count_nonfinite(const float* p, size_t n, int* d_count, cudaStream_t st);
 void launch_score_filters(const float* w, int K, int per_filter, int norm, double* scores, cudaStream_t st);
 void launch_rank_mask(const double* scores, int K, int q, int32_t* rank, uint8_t* mask, cudaStream_t st);
-// packed[kr][rs][cp] = w[row_src[kr]][chan_src[cp]][rs] (zero where an index is -1); bf16 and/or fp32 copies
-void launch_repack(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
-                   int C_pad, float scale, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st);
+// Convolution filters: packed[rs][cp/8][kr][cp%8] = w[row_src[kr]][chan_src[cp]][rs] (zero where an index is -1)
+void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
+                        int C_pad, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st);
+// FC matrix: packed[k][cp] = w[k][chan_src[cp]] * scale
+void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int C_pad, float scale, float* out,
+                      cudaStream_t st);
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st);
 
 // Memory-bound operators ------------------------------------------------------------------
-void launch_input_to_nhwc(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
-                          int C_pad, cudaStream_t st);
+void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
+                            int C_pad, cudaStream_t st);
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
                     int stride, int pad, cudaStream_t st);
-void launch_head(const void* x, int is_bf16, int N, int HW, int C_pad, const float* fcw, const float* fcb,
+void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
                  int n_classes, float* logits, cudaStream_t st);
-void launch_nhwc_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad,
-                             const int32_t* chan_dst, int C_out, cudaStream_t st);
+void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
+                               cudaStream_t st);
 
 // Convolutions ------------------------------------------------------------------------------
 // CUDA-core validation kernels: fp32 activations/filters, or bf16 activations/filters with
 // fp32 accumulation (same storage as the tensor-core path, used to localise differences).
 void launch_conv_simt(const ConvArgs& a, int is_bf16, cudaStream_t st);
 
-// Tensor-core path: per-layer plan (tile shape, TMA descriptors) built once per fp_prune.
+// Tensor-core path: per-layer plan built once per fp_prune.
 struct ConvPlanTC {
-    CUtensorMap tm_x;     // activations, 4-D {C, W, H, N}
-    CUtensorMap tm_w;     // filters, 3-D {C, R*S, K}
     int valid;
-    int tile_w, tile_h, tile_n;   // output pixels per CTA tile = tile_w * tile_h * tile_n = 128
-    int tiles_w, tiles_h, tiles_n;
-    int kc;               // channels per K block (16, 32 or 64)
-    int c_blocks;         // K blocks per filter tap
-    int n_tile;           // filters per CTA tile (multiple of 16, <= 256)
-    int n_tiles;
-    int stages;
+    int flat;             // 1: stride-1 "same" convolution, activation tiles fetched as contiguous runs
+                          //    of flat positions (bulk copies); 0: gathered by loader threads
+    int b_resident;       // flat only: the whole filter bank stays in shared memory
+    int cg;               // channel chunks (of 8) per K block
+    int groups;           // K blocks per filter tap = ceil((C_pad/8) / cg)
+    int halo;             // flat: vectors fetched before and after the 128 positions of a tile
+    int rows_a;           // flat: vectors per chunk per tile (128 + 2*halo, rounded up to 8)
+    int a_stages, b_stages;
+    int n_tile, n_tiles;  // filters per CTA tile (multiple of 16, <= 256)
     int tmem_cols;
-    int swizzle_bytes;    // 32, 64 or 128
     unsigned smem_bytes;
-    int grid;
+    int ctas_per_sm;
 };
 // Returns 0 on success, otherwise writes a message.
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len);

@@ -1,175 +1,212 @@
-// Memory-bound operators of the fused graph: boundary layout conversion, max pooling,
-// the global-average-pool + FC head, and a debug dump.  Activations are NHWC with the
-// channel count padded to a multiple of 16; padded channels always hold zeros.
+// Memory-bound operators of the fused graph in the planar-8 layout with a zero border (see
+// fp_internal.h): boundary layout conversion, max pooling, the global-average-pool + FC head,
+// and a debug dump.  One thread handles one vector (8 channels of one pixel), so a warp touches
+// 32 consecutive vectors of a chunk plane: 512 contiguous bytes of bf16.
 #include "fp_internal.h"
 
 namespace fp {
 
-__device__ __forceinline__ float ld_act(const void* p, size_t i, int is_bf16) {
-    return is_bf16 ? __bfloat162float(((const __nv_bfloat16*)p)[i]) : ((const float*)p)[i];
-}
+namespace {
 
-// NCHW (fp32 or bf16) -> NHWC (bf16 or fp32), channels zero-padded to C_pad.
-// One thread per output pixel writes its C_pad channels with 16-byte stores; reads are
-// coalesced across pixels for every channel plane.
-template <typename OutT, int CP>
-__global__ void input_to_nhwc_kernel(const void* __restrict__ in, int in_is_bf16, OutT* __restrict__ out, int N, int C,
-                                     int HW) {
-    const size_t total = (size_t)N * HW;
-    for (size_t pix = blockIdx.x * (size_t)blockDim.x + threadIdx.x; pix < total;
-         pix += (size_t)gridDim.x * blockDim.x) {
-        const size_t n = pix / HW, hw = pix - n * HW;
-        __align__(16) OutT v[CP];
-#pragma unroll
-        for (int c = 0; c < CP; ++c) {
-            float f = 0.0f;
-            if (c < C) f = ld_act(in, (n * C + c) * HW + hw, in_is_bf16);
-            if constexpr (sizeof(OutT) == 2) v[c] = __float2bfloat16_rn(f); else v[c] = f;
-        }
-        uint4* dst = reinterpret_cast<uint4*>(out + pix * CP);
-        const uint4* src = reinterpret_cast<const uint4*>(v);
-#pragma unroll
-        for (int i = 0; i < (int)(CP * sizeof(OutT) / 16); ++i) dst[i] = src[i];
-    }
-}
+struct __align__(16) Vec8h { __nv_bfloat162 v[4]; };
+struct __align__(32) Vec8f { float v[8]; };
 
-__global__ void input_to_nhwc_generic_kernel(const void* __restrict__ in, int in_is_bf16, void* __restrict__ out,
-                                             int out_is_bf16, int N, int C, int HW, int C_pad) {
-    const size_t total = (size_t)N * HW * C_pad;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % C_pad);
-        const size_t pix = i / C_pad;
-        const size_t n = pix / HW, hw = pix - n * HW;
-        const float f = c < C ? ld_act(in, (n * C + c) * HW + hw, in_is_bf16) : 0.0f;
-        if (out_is_bf16) ((__nv_bfloat16*)out)[i] = __float2bfloat16_rn(f); else ((float*)out)[i] = f;
-    }
-}
-
-// Max pooling over NHWC, 8 channels (16 bytes of bf16) or 4 channels (16 bytes of fp32) per thread.
 template <bool BF16>
-__global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y, int N, int H, int W, int C_pad, int P,
-                               int Q, int R, int stride, int pad) {
-    constexpr int V = BF16 ? 8 : 4;
-    const int cv = C_pad / V;
-    const size_t total = (size_t)N * P * Q * cv;
+__device__ __forceinline__ void load_vec8(const void* base, size_t vec, float (&f)[8]) {
+    if constexpr (BF16) {
+        const Vec8h r = reinterpret_cast<const Vec8h*>(base)[vec];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { const float2 g = __bfloat1622float2(r.v[i]); f[2 * i] = g.x; f[2 * i + 1] = g.y; }
+    } else {
+        const Vec8f r = reinterpret_cast<const Vec8f*>(base)[vec];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = r.v[i];
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void store_vec8(void* base, size_t vec, const float (&f)[8]) {
+    if constexpr (BF16) {
+        Vec8h r;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r.v[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+        reinterpret_cast<Vec8h*>(base)[vec] = r;
+    } else {
+        Vec8f r;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r.v[i] = f[i];
+        reinterpret_cast<Vec8f*>(base)[vec] = r;
+    }
+}
+
+// NCHW (fp32 or bf16) -> planar-8 with border.  Thread = (chunk, flat position); reads of one
+// channel plane are coalesced along w, writes are contiguous vectors.
+template <bool OUT_BF16>
+__global__ void input_to_planar_kernel(const void* __restrict__ in, int in_is_bf16, void* __restrict__ out, int N, int C,
+                                       int H, int W, int chunks) {
+    const int Wp = W + 2, P2 = (H + 2) * Wp;
+    const size_t plane = (size_t)N * P2;
+    const size_t total = plane * chunks;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % cv);
-        size_t t = i / cv;
-        const int q = (int)(t % Q); t /= Q;
-        const int p = (int)(t % P);
-        const size_t n = t / P;
-        float m[V];
+        const int j = (int)(i / plane);
+        const size_t f = i - (size_t)j * plane;
+        const size_t n = f / P2;
+        const int rem = (int)(f - n * P2);
+        const int h = rem / Wp - 1, w = rem % Wp - 1;
+        float v[8];
 #pragma unroll
-        for (int j = 0; j < V; ++j) m[j] = -INFINITY;
-        for (int r = 0; r < R; ++r) {
-            const int ih = p * stride + r - pad;
-            if (ih < 0 || ih >= H) continue;
-            for (int s = 0; s < R; ++s) {
-                const int iw = q * stride + s - pad;
-                if (iw < 0 || iw >= W) continue;
-                const size_t off = ((n * H + ih) * W + iw) * C_pad + (size_t)c * V;
-                const uint4 raw = *reinterpret_cast<const uint4*>(
-                    BF16 ? (const void*)((const __nv_bfloat16*)x + off) : (const void*)((const float*)x + off));
-                if constexpr (BF16) {
-                    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+        for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+        if (h >= 0 && h < H && w >= 0 && w < W) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 f = __bfloat1622float2(h2[j]);
-                        m[2 * j] = fmaxf(m[2 * j], f.x);
-                        m[2 * j + 1] = fmaxf(m[2 * j + 1], f.y);
-                    }
-                } else {
-                    const float* f = reinterpret_cast<const float*>(&raw);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) m[j] = fmaxf(m[j], f[j]);
+            for (int e = 0; e < 8; ++e) {
+                const int c = j * 8 + e;
+                if (c < C) {
+                    const size_t src = ((n * C + c) * H + h) * W + w;
+                    v[e] = in_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)in)[src]) : ((const float*)in)[src];
                 }
             }
         }
-        const size_t o = ((n * P + p) * Q + q) * C_pad + (size_t)c * V;
-        if constexpr (BF16) {
-            uint4 outv;
-            __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&outv);
+        store_vec8<OUT_BF16>(out, i, v);
+    }
+}
+
+// Max pooling; padded positions never win.  Output border positions are written as zeros.
+template <bool BF16>
+__global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y, int N, int H, int W, int chunks, int P,
+                               int Q, int R, int stride, int pad) {
+    const int Wp = W + 2, P2i = (H + 2) * Wp, Qp = Q + 2, P2o = (P + 2) * Qp;
+    const size_t plane_o = (size_t)N * P2o, plane_i = (size_t)N * P2i;
+    const size_t total = plane_o * chunks;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int j = (int)(i / plane_o);
+        const size_t f = i - (size_t)j * plane_o;
+        const size_t n = f / P2o;
+        const int rem = (int)(f - n * P2o);
+        const int p = rem / Qp - 1, q = rem % Qp - 1;
+        float m[8];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) h2[j] = __floats2bfloat162_rn(m[2 * j], m[2 * j + 1]);
-            *reinterpret_cast<uint4*>((__nv_bfloat16*)y + o) = outv;
-        } else {
-            *reinterpret_cast<float4*>((float*)y + o) = make_float4(m[0], m[1], m[2], m[3]);
+        for (int e = 0; e < 8; ++e) m[e] = 0.0f;
+        if (p >= 0 && p < P && q >= 0 && q < Q) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) m[e] = -INFINITY;
+            for (int r = 0; r < R; ++r) {
+                const int ih = p * stride + r - pad;
+                if (ih < 0 || ih >= H) continue;
+                for (int s = 0; s < R; ++s) {
+                    const int iw = q * stride + s - pad;
+                    if (iw < 0 || iw >= W) continue;
+                    float v[8];
+                    load_vec8<BF16>(x, (size_t)j * plane_i + n * P2i + (size_t)(ih + 1) * Wp + (iw + 1), v);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) m[e] = fmaxf(m[e], v[e]);
+                }
+            }
         }
+        store_vec8<BF16>(y, i, m);
     }
 }
 
 // Head: spatial sum per channel (fp32), then logits[k] = sum_c s[c] * Wfc[k][c] + b[k] with the
-// 1/(H*W) of the average already folded into Wfc.  One block per image; the channel sums live in
-// shared memory; one warp per class row with a shuffle reduction.
-__global__ void head_kernel(const void* __restrict__ x, int is_bf16, int HW, int C_pad, const float* __restrict__ fcw,
+// 1/(H*W) of the average already folded into Wfc.  One block per image; channel sums are reduced
+// through shuffles into shared memory; one warp per class row with a shuffle reduction.
+template <bool BF16>
+__global__ void head_kernel(const void* __restrict__ x, int N, int H, int W, int chunks, const float* __restrict__ fcw,
                             const float* __restrict__ fcb, int n_classes, float* __restrict__ logits) {
-    extern __shared__ float sums[];
+    extern __shared__ float sums[];          // chunks * 8
+    const int Wp = W + 2, P2 = (H + 2) * Wp, HW = H * W;
     const size_t n = blockIdx.x;
-    for (int c = threadIdx.x; c < C_pad; c += blockDim.x) {
-        float s = 0.0f;
-        for (int i = 0; i < HW; ++i) s += ld_act(x, (n * HW + i) * C_pad + c, is_bf16);
-        sums[c] = s;
+    const size_t plane = (size_t)N * P2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int j = warp; j < chunks; j += nwarps) {
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+        for (int i = lane; i < HW; i += 32) {
+            const int h = i / W, w = i - h * W;
+            float v[8];
+            load_vec8<BF16>(x, (size_t)j * plane + n * P2 + (size_t)(h + 1) * Wp + (w + 1), v);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += v[e];
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], d);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sums[j * 8 + e] = acc[e];
+        }
     }
     __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int C_pad = chunks * 8;
     for (int k = warp; k < n_classes; k += nwarps) {
         const float* wr = fcw + (size_t)k * C_pad;
         float s = 0.0f;
         for (int c = lane; c < C_pad; c += 32) s = fmaf(sums[c], wr[c], s);
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-        if (lane == 0) logits[n * n_classes + k] = s + fcb[k];
+        if (lane == 0) logits[n * n_classes + k] = s + (fcb ? fcb[k] : 0.0f);
     }
 }
 
-__global__ void nhwc_to_nchw_f32_kernel(const void* __restrict__ x, int is_bf16, float* __restrict__ out, int N, int HW,
-                                        int C_pad, const int32_t* __restrict__ chan_dst, int C_out) {
-    const size_t total = (size_t)N * HW * C_pad;
+template <bool BF16>
+__global__ void planar_to_nchw_f32_kernel(const void* __restrict__ x, float* __restrict__ out, int N, int H, int W,
+                                          int chunks, int C_out) {
+    const int Wp = W + 2, P2 = (H + 2) * Wp;
+    const size_t plane = (size_t)N * P2;
+    const size_t total = (size_t)N * chunks * H * W;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % C_pad);
-        const size_t pix = i / C_pad;
-        const size_t n = pix / HW, hw = pix - n * HW;
-        const int cd = chan_dst[c];
-        if (cd >= 0) out[(n * C_out + cd) * HW + hw] = ld_act(x, i, is_bf16);
+        const int w = (int)(i % W);
+        size_t t = i / W;
+        const int h = (int)(t % H); t /= H;
+        const int j = (int)(t % chunks);
+        const size_t n = t / chunks;
+        float v[8];
+        load_vec8<BF16>(x, (size_t)j * plane + n * P2 + (size_t)(h + 1) * Wp + (w + 1), v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int c = j * 8 + e;
+            if (c < C_out) out[((n * C_out + c) * H + h) * W + w] = v[e];
+        }
     }
 }
 
-static inline int grid_for(size_t n, int threads) {
+inline int grid_for(size_t n, int threads) {
     size_t b = (n + threads - 1) / threads;
     const size_t cap = 148 * 16;
     if (b < 1) b = 1;
     return (int)(b > cap ? cap : b);
 }
 
-void launch_input_to_nhwc(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
-                          int C_pad, cudaStream_t st) {
-    const int HW = H * W;
-    const size_t pix = (size_t)N * HW;
-    if (C_pad == 16 && out_is_bf16) {
-        input_to_nhwc_kernel<__nv_bfloat16, 16><<<grid_for(pix, 256), 256, 0, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, HW);
-    } else if (C_pad == 16) {
-        input_to_nhwc_kernel<float, 16><<<grid_for(pix, 256), 256, 0, st>>>(in, in_is_bf16, (float*)out, N, C, HW);
-    } else {
-        input_to_nhwc_generic_kernel<<<grid_for(pix * C_pad, 256), 256, 0, st>>>(in, in_is_bf16, out, out_is_bf16, N, C, HW, C_pad);
-    }
+}  // namespace
+
+void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
+                            int C_pad, cudaStream_t st) {
+    const size_t n = (size_t)N * (H + 2) * (W + 2) * (C_pad / 8);
+    if (out_is_bf16) input_to_planar_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8);
+    else input_to_planar_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8);
 }
 
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
                     int stride, int pad, cudaStream_t st) {
-    const size_t n = (size_t)N * P * Q * (C_pad / (is_bf16 ? 8 : 4));
-    if (is_bf16) maxpool_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(x, y, N, H, W, C_pad, P, Q, R, stride, pad);
-    else maxpool_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(x, y, N, H, W, C_pad, P, Q, R, stride, pad);
+    const size_t n = (size_t)N * (P + 2) * (Q + 2) * (C_pad / 8);
+    if (is_bf16) maxpool_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
+    else maxpool_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
 }
 
-void launch_head(const void* x, int is_bf16, int N, int HW, int C_pad, const float* fcw, const float* fcb,
+void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
                  int n_classes, float* logits, cudaStream_t st) {
-    head_kernel<<<N, 256, (size_t)C_pad * sizeof(float), st>>>(x, is_bf16, HW, C_pad, fcw, fcb, n_classes, logits);
+    const size_t smem = (size_t)C_pad * sizeof(float);
+    if (is_bf16) head_kernel<true><<<N, 256, smem, st>>>(x, N, H, W, C_pad / 8, fcw, fcb, n_classes, logits);
+    else head_kernel<false><<<N, 256, smem, st>>>(x, N, H, W, C_pad / 8, fcw, fcb, n_classes, logits);
 }
 
-void launch_nhwc_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad,
-                             const int32_t* chan_dst, int C_out, cudaStream_t st) {
-    const size_t n = (size_t)N * H * W * C_pad;
-    nhwc_to_nchw_f32_kernel<<<grid_for(n, 256), 256, 0, st>>>(x, is_bf16, out, N, H * W, C_pad, chan_dst, C_out);
+void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
+                               cudaStream_t st) {
+    const size_t n = (size_t)N * (C_pad / 8) * H * W;
+    if (is_bf16) planar_to_nchw_f32_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(x, out, N, H, W, C_pad / 8, C_out);
+    else planar_to_nchw_f32_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(x, out, N, H, W, C_pad / 8, C_out);
 }
 
 }  // namespace fp

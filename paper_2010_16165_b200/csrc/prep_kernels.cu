@@ -92,20 +92,36 @@ __global__ void rank_mask_kernel(const double* __restrict__ scores, int K, int q
     }
 }
 
-__global__ void repack_kernel(const float* __restrict__ w, int C, int RS, const int32_t* __restrict__ row_src,
-                              int K_pad, const int32_t* __restrict__ chan_src, int C_pad, float scale,
-                              __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32) {
-    const size_t total = (size_t)K_pad * RS * C_pad;
+// Filters of one convolution in the order the MMA wants them: tap-major, then chunks of 8 input
+// channels, then the filter, then the channel within the chunk.  For a fixed tap and chunk the
+// K_pad x 8 block is a stack of 16-byte rows - the canonical K-major operand layout without swizzle.
+__global__ void repack_conv_kernel(const float* __restrict__ w, int C, int RS, const int32_t* __restrict__ row_src,
+                                   int K_pad, const int32_t* __restrict__ chan_src, int C_pad,
+                                   __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32) {
+    const size_t total = (size_t)RS * C_pad * K_pad;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int cp = (int)(i % C_pad);
-        const size_t t = i / C_pad;
-        const int rs = (int)(t % RS);
-        const int kr = (int)(t / RS);
+        const int e = (int)(i % 8);
+        size_t t = i / 8;
+        const int kr = (int)(t % K_pad); t /= K_pad;
+        const int chunk = (int)(t % (C_pad / 8));
+        const int rs = (int)(t / (C_pad / 8));
+        const int cp = chunk * 8 + e;
         const int ks = row_src[kr], cs = chan_src[cp];
         float v = 0.0f;
-        if (ks >= 0 && cs >= 0) v = w[((size_t)ks * C + cs) * RS + rs] * scale;
+        if (ks >= 0 && cs >= 0) v = w[((size_t)ks * C + cs) * RS + rs];
         if (out_bf16) out_bf16[i] = __float2bfloat16_rn(v);
         if (out_f32) out_f32[i] = v;
+    }
+}
+
+__global__ void repack_fc_kernel(const float* __restrict__ w, int C, int K, const int32_t* __restrict__ chan_src,
+                                 int C_pad, float scale, float* __restrict__ out) {
+    const size_t total = (size_t)K * C_pad;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int cp = (int)(i % C_pad);
+        const int k = (int)(i / C_pad);
+        const int cs = chan_src[cp];
+        out[i] = cs >= 0 ? w[(size_t)k * C + cs] * scale : 0.0f;
     }
 }
 
@@ -151,10 +167,15 @@ void launch_rank_mask(const double* scores, int K, int q, int32_t* rank, uint8_t
     rank_mask_kernel<<<1, 256, (size_t)K * sizeof(double), st>>>(scores, K, q, rank, mask);
 }
 
-void launch_repack(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
-                   int C_pad, float scale, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st) {
+void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
+                        int C_pad, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st) {
     const size_t n = (size_t)K_pad * RS * C_pad;
-    repack_kernel<<<blocks_for(n, 256), 256, 0, st>>>(w, C, RS, row_src, K_pad, chan_src, C_pad, scale, out_bf16, out_f32);
+    repack_conv_kernel<<<blocks_for(n, 256), 256, 0, st>>>(w, C, RS, row_src, K_pad, chan_src, C_pad, out_bf16, out_f32);
+}
+
+void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int C_pad, float scale, float* out,
+                      cudaStream_t st) {
+    repack_fc_kernel<<<blocks_for((size_t)K * C_pad, 256), 256, 0, st>>>(w, C, K, chan_src, C_pad, scale, out);
 }
 
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st) {
