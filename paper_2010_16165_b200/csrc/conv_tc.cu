@@ -108,6 +108,17 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same, with both descriptors given by their low words; the high word (stride offset 128 B,
+// descriptor version 1, no swizzle) is the same constant for every operand block of this kernel.
+__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0x4008u) : "memory");
+}
 // Arrives on the mbarrier once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -196,18 +207,24 @@ conv_tc_kernel(const TcParams p) {
     const uint4* __restrict__ xv = reinterpret_cast<const uint4*>(p.a.x);
     const uint4* __restrict__ wv = reinterpret_cast<const uint4*>(p.a.w);
 
+    // Programmatic dependent launch: everything above, and the filter-bank copy below, touches
+    // nothing the previous kernel in the stream writes, so it may overlap that kernel's tail.  The
+    // next kernel is allowed to start its own prologue now; activations (and every global write) wait
+    // until the previous kernel has completed and its writes are visible.
+    if (MODE == MODE_FLAT_RESIDENT && threadIdx.x == 0) {
+        mbar_expect_tx(b_full0, (uint32_t)p.b_bank_bytes);
+        for (int off = 0; off < p.b_bank_bytes; off += 32768) {
+            const int n = p.b_bank_bytes - off < 32768 ? p.b_bank_bytes - off : 32768;
+            bulk_copy(b_base + off, reinterpret_cast<const uint8_t*>(p.a.w) + off, (uint32_t)n, b_full0);
+        }
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     if (warp == 0) {
         // ------------------------------ bulk-copy producer ------------------------------
         if (lane == 0) {
             bool ok = true;
-            if (MODE == MODE_FLAT_RESIDENT) {
-                // the whole filter bank, once
-                mbar_expect_tx(b_full0, (uint32_t)p.b_bank_bytes);
-                for (int off = 0; off < p.b_bank_bytes; off += 32768) {
-                    const int n = p.b_bank_bytes - off < 32768 ? p.b_bank_bytes - off : 32768;
-                    bulk_copy(b_base + off, reinterpret_cast<const uint8_t*>(p.a.w) + off, (uint32_t)n, b_full0);
-                }
-            }
             uint32_t stage = 0, phase = 0;
             if (MODE != MODE_GATHER) {
                 for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
@@ -270,36 +287,44 @@ conv_tc_kernel(const TcParams p) {
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.n_tile);
                 uint32_t accumulate = 0;
                 if (MODE != MODE_GATHER) {
+                    // Descriptors differ only in their 16-byte start-address field, so the inner loops
+                    // just add row counts to the low word (rows are 16 bytes: one row = one address unit).
                     for (int g = 0; g < p.groups && ok; ++g) {
                         if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         int cgg = p.cchunks - g * p.cg;
                         if (cgg > p.cg) cgg = p.cg;
-                        const uint32_t sa = a_base + a_stage * p.a_stage_bytes;
-                        for (int tap = 0; tap < p.taps; ++tap) {
-                            const int r = tap / p.a.S, s = tap - r * p.a.S;
-                            const int row_off = p.halo + (r - p.a.pad) * p.Wp_in + (s - p.a.pad);
-                            uint32_t sb, lbo_b;
-                            if (MODE == MODE_FLAT_RESIDENT) {
-                                sb = b_base + (uint32_t)((((tap * p.cchunks) + g * p.cg) * p.a.K_pad + nt * p.n_tile) * 16);
-                                lbo_b = (uint32_t)(p.a.K_pad * 16);
-                            } else {
-                                if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag)) { ok = false; break; }
-                                tc_fence_after();
-                                sb = b_base + b_stage * p.b_stage_bytes;
-                                lbo_b = (uint32_t)(p.n_tile * 16);
+                        const int ksteps = cgg >> 1;
+                        uint32_t a_row = ((a_base + a_stage * p.a_stage_bytes) >> 4) | ((uint32_t)p.rows_a << 16);
+                        uint32_t b_tap = 0;
+                        if (MODE == MODE_FLAT_RESIDENT)
+                            b_tap = ((b_base >> 4) + (uint32_t)(g * p.cg * p.a.K_pad + nt * p.n_tile)) | ((uint32_t)p.a.K_pad << 16);
+                        const uint32_t a_ks = 2u * (uint32_t)p.rows_a;
+                        const uint32_t b_ks = 2u * (uint32_t)(MODE == MODE_FLAT_RESIDENT ? p.a.K_pad : p.n_tile);
+                        const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.a.K_pad);
+                        for (int r = 0; r < p.a.R && ok; ++r) {
+                            for (int sx = 0; sx < p.a.S; ++sx) {
+                                uint32_t a_lo = a_row + (uint32_t)sx;
+                                uint32_t b_lo = b_tap;
+                                if (MODE == MODE_FLAT_STREAM) {
+                                    if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag)) { ok = false; break; }
+                                    tc_fence_after();
+                                    b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
+                                }
+                                for (int ks = 0; ks < ksteps; ++ks) {
+                                    umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
+                                    accumulate = 1;
+                                    a_lo += a_ks;
+                                    b_lo += b_ks;
+                                }
+                                if (MODE == MODE_FLAT_STREAM) {
+                                    umma_commit(b_empty0 + 8 * b_stage);
+                                    if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
+                                } else {
+                                    b_tap += b_tap_step;
+                                }
                             }
-                            for (int ks = 0; ks < cgg / 2; ++ks) {
-                                const uint64_t da = make_smem_desc(sa + (uint32_t)((2 * ks * p.rows_a + row_off) * 16),
-                                                                   (uint32_t)(p.rows_a * 16));
-                                const uint64_t db = make_smem_desc(sb + (uint32_t)(2 * ks) * lbo_b, lbo_b);
-                                umma_bf16(d_tmem, da, db, idesc, accumulate);
-                                accumulate = 1;
-                            }
-                            if (MODE == MODE_FLAT_STREAM) {
-                                umma_commit(b_empty0 + 8 * b_stage);
-                                if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
-                            }
+                            a_row += (uint32_t)p.Wp_in;
                         }
                         if (!ok) break;
                         umma_commit(a_empty0 + 8 * a_stage);     // releases the stage once these MMAs have read it
@@ -350,14 +375,26 @@ conv_tc_kernel(const TcParams p) {
             const bool interior = exists && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
             const int acc = local & 1;
             const uint32_t ph = acc ? acc_phase1 : acc_phase0;
+            const int k_base = nt * p.n_tile;
+            int cols = p.a.K_pad - k_base;
+            if (cols > p.n_tile) cols = p.n_tile;
+            const long long vec0 = (long long)(k_base >> 3) * p.plane_out + f;     // vector of columns 0..7
+            // the same-shape residual of the first 64 columns is requested before the accumulator is
+            // waited for; later columns are requested four 16-column chunks ahead
+            uint4 rq[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) rq[i] = make_uint4(0, 0, 0, 0);
+            const bool res1 = interior && p.a.res_mode == 1;
+            if (res1) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i * 8 < cols) rq[i] = __ldg(res + vec0 + (long long)i * p.plane_out);
+            }
             ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
             tc_fence_after();
-            const int k_base = nt * p.n_tile;
-            int cols = p.a.K_pad - k_base;
-            if (cols > p.n_tile) cols = p.n_tile;
             long long res_vec = 0;
             if (p.a.res_mode == 2) {
                 const int rWp = p.a.res_W + 2, rP2 = (p.a.res_H + 2) * rWp;
@@ -370,7 +407,7 @@ conv_tc_kernel(const TcParams p) {
                 tmem_ld16(taddr + c0, v);
                 tmem_ld_wait();
                 if (exists) {
-                const long long out_vec = (long long)((k_base + c0) >> 3) * p.plane_out + f;
+                const long long out_vec = vec0 + (long long)(c0 >> 3) * p.plane_out;
                 uint4 o[2];
                 o[0] = make_uint4(0, 0, 0, 0);
                 o[1] = o[0];
@@ -388,8 +425,7 @@ conv_tc_kernel(const TcParams p) {
                     if (p.a.res_mode == 1) {
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
-                            const uint4 raw = __ldg(res + out_vec + hh * p.plane_out);
-                            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+                            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&rq[hh]);
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const float2 g = __bfloat1622float2(h2[i]);
@@ -432,6 +468,14 @@ conv_tc_kernel(const TcParams p) {
                 }
                 y[out_vec] = o[0];
                 y[out_vec + p.plane_out] = o[1];
+                }
+                // rotate the residual queue and refill its tail
+#pragma unroll
+                for (int i = 0; i < 6; ++i) rq[i] = rq[i + 2];
+                if (res1 && c0 + 64 < cols) {
+                    const long long vn = vec0 + (long long)((c0 + 64) >> 3) * p.plane_out;
+                    rq[6] = __ldg(res + vn);
+                    rq[7] = __ldg(res + vn + p.plane_out);
                 }
             }
             tc_fence_before();
@@ -597,8 +641,6 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (ctas > tmem_ctas) ctas = tmem_ctas;
     if (ctas > want_ctas) ctas = want_ctas;
     if (ctas < 1) ctas = 1;
-    plan->ctas_per_sm = ctas;
-
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e0 = cudaFuncSetAttribute(conv_tc_kernel<MODE_FLAT_RESIDENT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
@@ -611,6 +653,20 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         }
         attr_set = true;
     }
+    // persistent grid: exactly as many CTAs as can be resident at once (registers, threads, shared memory)
+    cudaFuncAttributes fa;
+    cudaError_t oe;
+    if (!plan->flat) oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_GATHER>);
+    else if (plan->b_resident) oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_FLAT_RESIDENT>);
+    else oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_FLAT_STREAM>);
+    if (oe != cudaSuccess) { snprintf(err, err_len, "cudaFuncGetAttributes: %s", cudaGetErrorString(oe)); cudaGetLastError(); return 1; }
+    const int threads = plan->flat ? 224 : 320;
+    const int regs_per_warp = round_up_i(fa.numRegs * 32, 256);
+    int occ = 65536 / (regs_per_warp * (threads / 32));
+    if (occ > 2048 / threads) occ = 2048 / threads;
+    if (occ < 1) occ = 1;
+    if (ctas > occ) ctas = occ;
+    plan->ctas_per_sm = ctas;
     plan->valid = 1;
     return 0;
 }
@@ -636,9 +692,20 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     int grid = 148 * plan.ctas_per_sm;
     if (grid > p.total_tiles) grid = p.total_tiles;
     if (grid < 1) grid = 1;
-    if (!plan.flat) conv_tc_kernel<MODE_GATHER><<<grid, 320, plan.smem_bytes, st>>>(p);
-    else if (plan.b_resident) conv_tc_kernel<MODE_FLAT_RESIDENT><<<grid, 224, plan.smem_bytes, st>>>(p);
-    else conv_tc_kernel<MODE_FLAT_STREAM><<<grid, 224, plan.smem_bytes, st>>>(p);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(plan.flat ? 224u : 320u);
+    cfg.dynamicSmemBytes = plan.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (!plan.flat) cudaLaunchKernelEx(&cfg, conv_tc_kernel<MODE_GATHER>, p);
+    else if (plan.b_resident) cudaLaunchKernelEx(&cfg, conv_tc_kernel<MODE_FLAT_RESIDENT>, p);
+    else cudaLaunchKernelEx(&cfg, conv_tc_kernel<MODE_FLAT_STREAM>, p);
 }
 
 }  // namespace fp
