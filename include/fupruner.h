@@ -188,6 +188,37 @@ typedef struct {
 
 fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_out, size_t bytes);
 
+/*
+ * fp_rank_filters_static - score, rank and mask the filters of ONE filter bank without allocating.
+ * (No counterpart in the paper: it is the selection step of fp_prune offered in a form for callers
+ * that must not allocate.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - a serving loop that has handed
+ * all device memory to its own pool, a real-time path that cannot afford cudaMalloc's implicit
+ * device synchronisation, a plug-in that is only given buffers.  fp_fuse/fp_prune allocate (packed
+ * banks, score buffers); this call does not: it calls no cudaMalloc/cudaFree and no allocating
+ * library routine.  Its one intermediate, an fp64 score per filter, lives in a fixed array inside the
+ * library image (32 KB, present on every GPU that loads the library, until the process exits).
+ *
+ *   d_filters   device fp32, K filters of per_filter elements each, filter-major (a K x C x R x S bank).
+ *   norm        FP_NORM_L1 or FP_NORM_L2; scores and order exactly as fp_score / fp_prune define them.
+ *   q           number of filters to mask: the q lowest by (score, index) get mask 0.  0 <= q <= K.
+ *   d_rank      device int32[K]  out: position of each filter in ascending (score, index) order.
+ *   d_mask      device uint8[K]  out: 1 keep, 0 pruned.
+ *   stream      cudaStream_t as void*, NULL = default stream.  Asynchronous.
+ *
+ * Limit: K <= FP_STATIC_RANK_MAX_FILTERS (4096); larger banks are rejected with FP_ERR_BOUNDS.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and keeps it;
+ * make that first call outside any stream capture.  All calls on a device share the array: two calls
+ * whose kernels overlap on the GPU (different streams, no ordering between them) race on it - order
+ * them.  The array keeps the previous call's scores; every call overwrites the part it reads, so
+ * nothing needs clearing.
+ * Errors: FP_ERR_ARG, FP_ERR_BOUNDS, FP_ERR_CUDA.
+ */
+#define FP_STATIC_RANK_MAX_FILTERS 4096
+fp_status fp_rank_filters_static(const float* d_filters, int32_t K, int32_t per_filter, int32_t norm, int32_t q,
+                                 int32_t* d_rank, uint8_t* d_mask, void* stream);
+
 fp_status fp_destroy(fp_handle h);
 
 const char* fp_last_error(void);

@@ -25,7 +25,8 @@ FP_NORM_L1, FP_NORM_L2 = 0, 1
  FP_Q_OP_TIMES) = range(15)
 
 EXPORTS = ["fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_score", "fp_query", "fp_destroy",
-           "fp_last_error"]
+           "fp_last_error", "fp_rank_filters_static"]
+FP_STATIC_RANK_MAX_FILTERS = 4096
 
 
 class fp_node(ctypes.Structure):
@@ -75,6 +76,8 @@ def lib():
         L.fp_score.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
         L.fp_query.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t]
         L.fp_destroy.argtypes = [ctypes.c_void_p]
+        L.fp_rank_filters_static.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                             ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -162,6 +165,13 @@ def fp_query_op(h, index):
     o = fp_op_info()
     _check(lib().fp_query(h, FP_Q_OP_INFO, index, ctypes.byref(o), ctypes.sizeof(o)))
     return o
+
+
+def fp_rank_filters_static(d_filters, K, per_filter, norm, q, d_rank, d_mask, stream=None):
+    """Allocation-free selection for one bank: d_filters fp32 CUDA tensor (K*per_filter), d_rank int32[K] and
+    d_mask uint8[K] CUDA tensors provided by the caller.  Asynchronous on `stream`."""
+    _check(lib().fp_rank_filters_static(d_filters.data_ptr(), K, per_filter, norm, q, d_rank.data_ptr(),
+                                        d_mask.data_ptr(), stream.cuda_stream if stream is not None else None))
 
 
 def fp_destroy(h):

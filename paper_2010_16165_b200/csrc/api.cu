@@ -649,6 +649,10 @@ fp_status all_ones_masks(fp_handle h) {
 
 extern "C" const char* fp_last_error(void) { return g_err.c_str(); }
 
+namespace fp_detail {
+fp_status set_error(fp_status st, const char* msg) { return fail(st, "%s", msg); }
+}
+
 extern "C" fp_status fp_destroy(fp_handle h) {
     if (!h) return FP_OK;
     cudaDeviceSynchronize();
