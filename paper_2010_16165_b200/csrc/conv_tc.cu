@@ -145,6 +145,40 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo) 
     return d;
 }
 
+// Issues the MMAs of one K block of a FLAT-mode tile: R*R filter taps x KSTEPS K=16 steps, fully
+// unrolled so that the single issuing thread spends a handful of instructions per MMA.  Operand
+// descriptors differ only in their low words: one address unit is one 16-byte row, so a tap's
+// activation operand is `a_lo + r*Wp + s` and a K step advances both operands by two planes.
+template <int R, int KSTEPS>
+__device__ __forceinline__ void issue_flat_resident(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t Wp,
+                                                    uint32_t a_ks, uint32_t b_ks, uint32_t b_tap, uint32_t idesc,
+                                                    uint32_t accumulate) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+        for (int sx = 0; sx < R; ++sx) {
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                umma_bf16_lo(d_tmem, a_lo + (uint32_t)r * Wp + (uint32_t)sx + (uint32_t)ks * a_ks,
+                             b_lo + (uint32_t)(r * R + sx) * b_tap + (uint32_t)ks * b_ks, idesc,
+                             (r | sx | ks) ? 1u : accumulate);
+            }
+        }
+    }
+}
+
+template <int R>
+__device__ __forceinline__ void issue_flat_resident_k(int ksteps, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                                      uint32_t Wp, uint32_t a_ks, uint32_t b_ks, uint32_t b_tap,
+                                                      uint32_t idesc, uint32_t accumulate) {
+    switch (ksteps) {
+        case 1: issue_flat_resident<R, 1>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        case 2: issue_flat_resident<R, 2>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        case 3: issue_flat_resident<R, 3>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        default: issue_flat_resident<R, 4>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+    }
+}
+
 // Shared-memory control block at the start of dynamic shared memory.
 struct Ctrl {
     uint64_t a_full[kMaxStages];
@@ -302,6 +336,13 @@ conv_tc_kernel(const TcParams p) {
                         const uint32_t a_ks = 2u * (uint32_t)p.rows_a;
                         const uint32_t b_ks = 2u * (uint32_t)(MODE == MODE_FLAT_RESIDENT ? p.a.K_pad : p.n_tile);
                         const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.a.K_pad);
+                        if (MODE == MODE_FLAT_RESIDENT) {
+                            if (p.a.R == 3)
+                                issue_flat_resident_k<3>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
+                            else
+                                issue_flat_resident_k<1>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
+                            accumulate = 1;
+                        } else
                         for (int r = 0; r < p.a.R && ok; ++r) {
                             for (int sx = 0; sx < p.a.S; ++sx) {
                                 uint32_t a_lo = a_row + (uint32_t)sx;
