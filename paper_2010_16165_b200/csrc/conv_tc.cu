@@ -20,7 +20,7 @@
 //   GATHER mode   any other geometry (stride 2, 7x7, ...): 128 loader threads fetch the vectors of
 //                 their output position for each (tap, K block) with 16-byte loads, zero where the
 //                 window leaves the image.
-//   Warp roles    warp 0 lane 0: bulk-copy producer.  warp 1: tensor-memory allocation, lane 0 issues
+//   Warp roles    warp 0: bulk-copy producer (one lane per chunk copy).  warp 1: tensor-memory allocation, lane 0 issues
 //                 the MMAs.  warps 2-5: epilogue, one thread per accumulator row.  warp 6 lane 0:
 //                 filter producer when filters are streamed in a FLAT mode.  warps 6-9: loader
 //                 threads in GATHER mode.
@@ -189,7 +189,9 @@ struct Ctrl {
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
+    int pad_[2];          // keeps sizeof(Ctrl) a multiple of 16: the bias table follows
 };
+static_assert(sizeof(Ctrl) % 16 == 0, "bias table must stay 16-byte aligned");
 
 __device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
     atomicExch(&ctrl->abort_flag, 1);
@@ -199,10 +201,11 @@ __device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
 template <int MODE>
 __global__ void __launch_bounds__(MODE == MODE_GATHER ? 320 : 224)
 conv_tc_kernel(const TcParams p) {
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(128) uint8_t smem_raw[];
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
     const uint32_t ctrl_addr = smem_u32(smem_raw);
-    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + 1023u) & ~1023u;
+    float* bias_s = reinterpret_cast<float*>(smem_raw + sizeof(Ctrl));            // K_pad floats
+    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + (uint32_t)p.a.K_pad * 4u + 1023u) & ~1023u;
     const uint32_t b_region = MODE == MODE_FLAT_RESIDENT ? (uint32_t)p.b_bank_bytes
                               : MODE == MODE_FLAT_STREAM ? (uint32_t)(p.b_stages * p.b_stage_bytes) : 0u;
     const uint32_t a_base = b_base + ((b_region + 127u) & ~127u);
@@ -228,6 +231,7 @@ conv_tc_kernel(const TcParams p) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    for (int i = threadIdx.x; i < p.a.K_pad; i += blockDim.x) bias_s[i] = p.a.bias[i];   // filters' data: safe before the dependency wait
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_base)), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -257,26 +261,35 @@ conv_tc_kernel(const TcParams p) {
 
     if (warp == 0) {
         // ------------------------------ bulk-copy producer ------------------------------
-        if (lane == 0) {
+        if (MODE != MODE_GATHER) {
+            // One lane per channel chunk issues that chunk's copy, so the copies of a K block are issued
+            // side by side instead of one after the other.
             bool ok = true;
             uint32_t stage = 0, phase = 0;
-            if (MODE != MODE_GATHER) {
-                for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                    const long long f0 = (long long)(tile / p.n_tiles) * 128;
-                    for (int g = 0; g < p.groups; ++g) {
-                        if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                        int cgg = p.cchunks - g * p.cg;
-                        if (cgg > p.cg) cgg = p.cg;
-                        const uint32_t fb = a_full0 + 8 * stage;
-                        const uint32_t dst = a_base + stage * p.a_stage_bytes;
-                        mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
-                        for (int c = 0; c < cgg; ++c)
-                            bulk_copy(dst + c * p.rows_a * 16, xv + (long long)(g * p.cg + c) * p.plane_in + f0 - p.halo,
-                                      (uint32_t)(p.rows_a * 16), fb);
-                        if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
-                    }
+            for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+                const long long f0 = (long long)(tile / p.n_tiles) * 128;
+                for (int g = 0; g < p.groups; ++g) {
+                    bool w = true;
+                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w) { ok = false; break; }
+                    int cgg = p.cchunks - g * p.cg;
+                    if (cgg > p.cg) cgg = p.cg;
+                    const uint32_t fb = a_full0 + 8 * stage;
+                    const uint32_t dst = a_base + stage * p.a_stage_bytes;
+                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
+                    __syncwarp();
+                    if (lane < cgg)
+                        bulk_copy(dst + lane * p.rows_a * 16, xv + (long long)(g * p.cg + lane) * p.plane_in + f0 - p.halo,
+                                  (uint32_t)(p.rows_a * 16), fb);
+                    if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
                 }
-            } else {
+            }
+            if (!ok && lane == 0) raise(ctrl, p.status, 1);
+        } else if (lane == 0) {
+            bool ok = true;
+            uint32_t stage = 0, phase = 0;
+            {
                 // GATHER: filters of each (tap, K block) into the stage the loader threads fill
                 for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
                     const int nt = tile % p.n_tiles;
@@ -454,10 +467,10 @@ conv_tc_kernel(const TcParams p) {
                 o[1] = o[0];
                 if (interior) {
                     float fv[16];
-                    const float4* b4 = reinterpret_cast<const float4*>(p.a.bias + k_base + c0);
+                    const float4* b4 = reinterpret_cast<const float4*>(bias_s + k_base + c0);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const float4 b = __ldg(b4 + i);
+                        const float4 b = b4[i];
                         fv[4 * i + 0] = __uint_as_float(v[4 * i + 0]) + b.x;
                         fv[4 * i + 1] = __uint_as_float(v[4 * i + 1]) + b.y;
                         fv[4 * i + 2] = __uint_as_float(v[4 * i + 2]) + b.z;
@@ -642,7 +655,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     plan->tmem_cols = pow2_at_least(2 * n_tile < 32 ? 32 : 2 * n_tile);
     const int tmem_ctas = 512 / plan->tmem_cols;
 
-    unsigned smem = (unsigned)sizeof(Ctrl) + 1024u;
+    unsigned smem = (unsigned)sizeof(Ctrl) + (unsigned)a.K_pad * 4u + 1024u;
     int want_ctas = 1;
     if (plan->flat) {
         plan->halo = a.pad * (a.W + 3);
