@@ -44,8 +44,13 @@ constexpr long long kWaitCycles = 2000000000LL;    // SM clock cycles per wait (
 
 enum { MODE_FLAT_RESIDENT = 0, MODE_FLAT_STREAM = 1, MODE_GATHER = 2 };
 
+// Division by a run-time constant as multiply-high + shift (n < 2^31, d >= 1).
+struct FastDiv { uint32_t mul, shift, d; };
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f) { return (__umulhi(n, f.mul) + n) >> f.shift; }
+
 struct TcParams {
     ConvArgs a;
+    FastDiv div_ntiles, div_p2out, div_qp;
     int Wp_in, P2_in, Qp, P2_out;
     long long plane_in, plane_out;      // vectors per chunk plane (N * P2)
     long long m_total;                  // flat output positions
@@ -199,7 +204,7 @@ __device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(MODE == MODE_GATHER ? 320 : 224)
+__global__ void __launch_bounds__(MODE == MODE_GATHER ? 320 : MODE == MODE_FLAT_STREAM ? 224 : 192)
 conv_tc_kernel(const TcParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
@@ -267,7 +272,7 @@ conv_tc_kernel(const TcParams p) {
             bool ok = true;
             uint32_t stage = 0, phase = 0;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                const long long f0 = (long long)(tile / p.n_tiles) * 128;
+                const long long f0 = (long long)fdiv((uint32_t)tile, p.div_ntiles) * 128;
                 for (int g = 0; g < p.groups; ++g) {
                     bool w = true;
                     if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
@@ -292,7 +297,7 @@ conv_tc_kernel(const TcParams p) {
             {
                 // GATHER: filters of each (tap, K block) into the stage the loader threads fill
                 for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                    const int nt = tile % p.n_tiles;
+                    const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
                     int nrows = p.a.K_pad - nt * p.n_tile;
                     if (nrows > p.n_tile) nrows = p.n_tile;
                     for (int tap = 0; tap < p.taps && ok; ++tap) {
@@ -330,7 +335,7 @@ conv_tc_kernel(const TcParams p) {
                 if (!mbar_wait(tempty0 + 8 * acc, ph ^ 1, abort_flag)) { ok = false; break; }
                 if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
                 tc_fence_after();
-                const int nt = tile % p.n_tiles;
+                const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.n_tile);
                 uint32_t accumulate = 0;
                 if (MODE != MODE_GATHER) {
@@ -420,12 +425,13 @@ conv_tc_kernel(const TcParams p) {
         const __nv_bfloat16* __restrict__ res_s = reinterpret_cast<const __nv_bfloat16*>(p.a.res);
         uint4* __restrict__ y = reinterpret_cast<uint4*>(p.a.y);
         for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++local) {
-            const int nt = tile % p.n_tiles;
-            const long long f = (long long)(tile / p.n_tiles) * 128 + row;
+            const int mt = (int)fdiv((uint32_t)tile, p.div_ntiles);
+            const int nt = tile - mt * p.n_tiles;
+            const long long f = (long long)mt * 128 + row;
             const bool exists = f < p.m_total;
-            const int n = (int)(f / p.P2_out);
-            const int rem = (int)(f - (long long)n * p.P2_out);
-            const int hp = rem / p.Qp, wq = rem - hp * p.Qp;
+            const int n = (int)fdiv((uint32_t)f, p.div_p2out);
+            const int rem = (int)f - n * p.P2_out;
+            const int hp = (int)fdiv((uint32_t)rem, p.div_qp), wq = rem - hp * p.Qp;
             const bool interior = exists && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
             const int acc = local & 1;
             const uint32_t ph = acc ? acc_phase1 : acc_phase0;
@@ -542,7 +548,7 @@ conv_tc_kernel(const TcParams p) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                const int nt = tile % p.n_tiles;
+                const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
                 int nrows = p.a.K_pad - nt * p.n_tile;
                 if (nrows > p.n_tile) nrows = p.n_tile;
                 for (int g = 0; g < p.groups && ok; ++g) {
@@ -570,10 +576,10 @@ conv_tc_kernel(const TcParams p) {
         bool ok = true;
         const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
         for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-            const long long f = (long long)(tile / p.n_tiles) * 128 + m;
-            const int n = (int)(f / p.P2_out);
-            const int rem = (int)(f - (long long)n * p.P2_out);
-            const int hp = rem / p.Qp, wq = rem - hp * p.Qp;
+            const long long f = (long long)fdiv((uint32_t)tile, p.div_ntiles) * 128 + m;
+            const int n = (int)fdiv((uint32_t)f, p.div_p2out);
+            const int rem = (int)f - n * p.P2_out;
+            const int hp = (int)fdiv((uint32_t)rem, p.div_qp), wq = rem - hp * p.Qp;
             const bool interior = f < p.m_total && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
             const int ih0 = (hp - 1) * p.a.stride - p.a.pad, iw0 = (wq - 1) * p.a.stride - p.a.pad;
             for (int tap = 0; tap < p.taps && ok; ++tap) {
@@ -619,6 +625,15 @@ conv_tc_kernel(const TcParams p) {
 }
 
 int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    uint32_t shift = 0;
+    while ((1ull << shift) < d) ++shift;
+    f.shift = shift;
+    f.mul = (uint32_t)((((1ull << 32) * ((1ull << shift) - d)) / d) + 1);
+    f.d = d;
+    return f;
+}
 int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
 constexpr unsigned kSmemMax = 232448u - 1024u;     // opt-in dynamic shared memory per CTA
@@ -638,6 +653,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     plan->groups = (cchunks + plan->cg - 1) / plan->cg;
     const long long m_total = (long long)a.N * (a.P + 2) * (a.Q + 2);
     const long long m_tiles = (m_total + 127) / 128;
+    if (m_total + 128 >= (1ll << 31)) { snprintf(err, err_len, "more than 2^31 output positions"); return 1; }
 
     // --- filter tile ---
     int n_tiles = (a.K_pad + 255) / 256;
@@ -714,7 +730,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     else if (plan->b_resident) oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_FLAT_RESIDENT>);
     else oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_FLAT_STREAM>);
     if (oe != cudaSuccess) { snprintf(err, err_len, "cudaFuncGetAttributes: %s", cudaGetErrorString(oe)); cudaGetLastError(); return 1; }
-    const int threads = plan->flat ? 224 : 320;
+    const int threads = !plan->flat ? 320 : plan->b_resident ? 192 : 224;
     const int regs_per_warp = round_up_i(fa.numRegs * 32, 256);
     int occ = 65536 / (regs_per_warp * (threads / 32));
     if (occ > 2048 / threads) occ = 2048 / threads;
@@ -743,13 +759,16 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.b_stage_bytes = plan.cg * plan.n_tile * 16;
     p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
     p.status = d_status;
+    p.div_ntiles = make_fastdiv((uint32_t)plan.n_tiles);
+    p.div_p2out = make_fastdiv((uint32_t)p.P2_out);
+    p.div_qp = make_fastdiv((uint32_t)p.Qp);
     int grid = 148 * plan.ctas_per_sm;
     if (grid > p.total_tiles) grid = p.total_tiles;
     if (grid < 1) grid = 1;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(plan.flat ? 224u : 320u);
+    cfg.blockDim = dim3(!plan.flat ? 320u : plan.b_resident ? 192u : 224u);
     cfg.dynamicSmemBytes = plan.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
