@@ -114,6 +114,7 @@ struct fp_handle_s {
     const float* d_fcw = nullptr;          // classes x fc_C (copy of the description's FC weights)
     const float* d_fcb = nullptr;
     float* d_fcw_packed = nullptr;         // classes x C_pad, scaled by 1/(H*W)
+    float* d_pool = nullptr;               // max_batch x C_pad channel sums (between the two head kernels)
     // buffers
     std::vector<void*> act_buffers;        // activation storage (re-planned by fp_prune)
     std::vector<void*> pack_buffers;       // packed filters / biases / index arrays
@@ -534,6 +535,7 @@ fp_status replan(fp_handle h) {
             int32_t* d_chan;
             TRY(upload_i32(h, chan_src, &d_chan));
             TRY(dev_alloc(h->pack_buffers, (void**)&h->d_fcw_packed, (size_t)h->n_classes * src.C_pad * sizeof(float)));
+            TRY(dev_alloc(h->pack_buffers, (void**)&h->d_pool, (size_t)h->max_batch * src.C_pad * sizeof(float)));
             // the average's 1/(H*W) is folded into the FC weights
             fp::launch_repack_fc(h->d_fcw, h->fc_C, h->n_classes, d_chan, src.C_pad, 1.0f / (float)(src.H * src.W),
                                  h->d_fcw_packed, st);
@@ -624,7 +626,7 @@ void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float*
         fp::launch_maxpool(s.d, o.d, bf16, batch, s.H, s.W, s.C_pad, o.H, o.W, p.R, p.stride, p.pad, st);
     } else {
         const Tensor& s = h->tensors[h->head_src];
-        fp::launch_head(s.d, bf16, batch, s.H, s.W, s.C_pad, h->d_fcw_packed, h->d_fcb, h->n_classes, d_logits, st);
+        fp::launch_head(s.d, bf16, batch, s.H, s.W, s.C_pad, h->d_fcw_packed, h->d_fcb, h->n_classes, d_logits, h->d_pool, st);
     }
 }
 
@@ -891,7 +893,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
         case FP_Q_N_CONVS: TRY(need(4)); *(int32_t*)h_out = h->n_desc_convs; return FP_OK;
         case FP_Q_N_CLASSES: TRY(need(4)); *(int32_t*)h_out = h->n_classes; return FP_OK;
         case FP_Q_N_OPS: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size(); return FP_OK;
-        case FP_Q_N_LAUNCHES: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size(); return FP_OK;
+        case FP_Q_N_LAUNCHES: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size() + 1; return FP_OK;   // the head is two kernels
         case FP_Q_CONV_K_FUSED: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K : 0; return FP_OK;
         case FP_Q_CONV_K_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K_kept : 0; return FP_OK;
         case FP_Q_CONV_C_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->C_kept : 0; return FP_OK;

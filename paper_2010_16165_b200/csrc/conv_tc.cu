@@ -56,6 +56,7 @@ struct TcParams {
     long long m_total;                  // flat output positions
     int taps, cchunks, cg, groups, halo, rows_a, a_stages, b_stages;
     int n_tile, n_tiles, tmem_cols, total_tiles;
+    int tpk, kblocks;                   // gather: taps per K block, K blocks per tile
     int a_stage_bytes, b_stage_bytes, b_bank_bytes;
     int* status;
 };
@@ -300,20 +301,21 @@ conv_tc_kernel(const TcParams p) {
                     const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
                     int nrows = p.a.K_pad - nt * p.n_tile;
                     if (nrows > p.n_tile) nrows = p.n_tile;
-                    for (int tap = 0; tap < p.taps && ok; ++tap) {
-                        for (int g = 0; g < p.groups; ++g) {
-                            if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                            int cgg = p.cchunks - g * p.cg;
-                            if (cgg > p.cg) cgg = p.cg;
-                            const uint32_t fb = a_full0 + 8 * stage;
-                            const uint32_t dst = a_base + stage * (p.a_stage_bytes + p.b_stage_bytes) + p.a_stage_bytes;
-                            mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
+                    for (int kb = 0; kb < p.kblocks; ++kb) {
+                        // a K block is either one tap x one channel group, or (few channels) several whole taps
+                        int tap0, g, ntap, cgg;
+                        if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
+                        else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
+                        if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        const uint32_t fb = a_full0 + 8 * stage;
+                        const uint32_t dst = a_base + stage * (p.a_stage_bytes + p.b_stage_bytes) + p.a_stage_bytes;
+                        mbar_expect_tx(fb, (uint32_t)(ntap * cgg * nrows * 16));
+                        for (int tt = 0; tt < ntap; ++tt)
                             for (int c = 0; c < cgg; ++c)
-                                bulk_copy(dst + c * p.n_tile * 16,
-                                          wv + ((long long)tap * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
+                                bulk_copy(dst + (tt * cgg + c) * p.n_tile * 16,
+                                          wv + ((long long)(tap0 + tt) * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
                                           (uint32_t)(nrows * 16), fb);
-                            if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
-                        }
+                        if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
                     }
                 }
             }
@@ -390,21 +392,22 @@ conv_tc_kernel(const TcParams p) {
                         if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
                     }
                 } else {
-                    const int kblocks = p.taps * p.groups;
                     const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-                    for (int kb = 0; kb < kblocks; ++kb) {
+                    for (int kb = 0; kb < p.kblocks; ++kb) {
                         if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const int g = kb % p.groups;
-                        int cgg = p.cchunks - g * p.cg;
-                        if (cgg > p.cg) cgg = p.cg;
+                        int planes;
+                        if (p.groups > 1) { const int g = kb % p.groups; planes = p.cchunks - g * p.cg; if (planes > p.cg) planes = p.cg; }
+                        else { const int tap0 = kb * p.tpk; planes = (p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk) * p.cchunks; }
                         const uint32_t sa = a_base + a_stage * stage_bytes;
                         const uint32_t sb = sa + p.a_stage_bytes;
-                        for (int ks = 0; ks < cgg / 2; ++ks) {
-                            const uint64_t da = make_smem_desc(sa + (uint32_t)(2 * ks * 128 * 16), 128 * 16);
-                            const uint64_t db = make_smem_desc(sb + (uint32_t)(2 * ks * p.n_tile * 16), (uint32_t)(p.n_tile * 16));
-                            umma_bf16(d_tmem, da, db, idesc, accumulate);
+                        uint32_t a_lo = (sa >> 4) | (128u << 16);
+                        uint32_t b_lo = (sb >> 4) | ((uint32_t)p.n_tile << 16);
+                        for (int ks = 0; ks < planes / 2; ++ks) {
+                            umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
                             accumulate = 1;
+                            a_lo += 256u;
+                            b_lo += 2u * (uint32_t)p.n_tile;
                         }
                         umma_commit(a_empty0 + 8 * a_stage);
                         if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
@@ -582,29 +585,34 @@ conv_tc_kernel(const TcParams p) {
             const int hp = (int)fdiv((uint32_t)rem, p.div_qp), wq = rem - hp * p.Qp;
             const bool interior = f < p.m_total && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
             const int ih0 = (hp - 1) * p.a.stride - p.a.pad, iw0 = (wq - 1) * p.a.stride - p.a.pad;
-            for (int tap = 0; tap < p.taps && ok; ++tap) {
-                const int r = tap / p.a.S, s = tap - r * p.a.S;
-                const int ih = ih0 + r, iw = iw0 + s;
-                const bool valid = interior && ih >= 0 && ih < p.a.H && iw >= 0 && iw < p.a.W;
-                const long long src = (long long)n * p.P2_in + (long long)(ih + 1) * p.Wp_in + (iw + 1);
-                for (int g = 0; g < p.groups; ++g) {
-                    int cgg = p.cchunks - g * p.cg;
-                    if (cgg > p.cg) cgg = p.cg;
-                    uint4 v[8];
+            for (int kb = 0; kb < p.kblocks && ok; ++kb) {
+                int tap0, g, ntap, cgg;
+                if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
+                else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
+                uint4 v[8];
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        v[c] = make_uint4(0, 0, 0, 0);
-                        if (valid && c < cgg) v[c] = __ldg(xv + (long long)(g * p.cg + c) * p.plane_in + src);
+                for (int i = 0; i < 8; ++i) v[i] = make_uint4(0, 0, 0, 0);
+                int r = tap0 / p.a.S, s = tap0 - r * p.a.S;
+                for (int tt = 0; tt < ntap; ++tt) {
+                    const int ih = ih0 + r, iw = iw0 + s;
+                    const bool valid = interior && ih >= 0 && ih < p.a.H && iw >= 0 && iw < p.a.W;
+                    const long long src = (long long)n * p.P2_in + (long long)(ih + 1) * p.Wp_in + (iw + 1);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int c = i - tt * cgg;          // plane i holds chunk c of tap tap0+tt
+                        if (valid && c >= 0 && c < cgg) v[i] = __ldg(xv + (long long)(g * p.cg + c) * p.plane_in + src);
                     }
-                    if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                    uint8_t* dst = smem_raw + (a_base - ctrl_addr) + stage * stage_bytes + m * 16;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        if (c < cgg) *reinterpret_cast<uint4*>(dst + c * 128 * 16) = v[c];
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> MMA reads
-                    mbar_arrive(a_full0 + 8 * stage);
-                    if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
+                    if (++s == p.a.S) { s = 0; ++r; }
                 }
+                if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                uint8_t* dst = smem_raw + (a_base - ctrl_addr) + stage * stage_bytes + m * 16;
+                const int planes = ntap * cgg;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i < planes) *reinterpret_cast<uint4*>(dst + i * 128 * 16) = v[i];
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> MMA reads
+                mbar_arrive(a_full0 + 8 * stage);
+                if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
             }
         }
         if (!ok) raise(ctrl, p.status, 5);
@@ -695,7 +703,11 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         }
         want_ctas = 4;
     } else {
-        const unsigned stage = (unsigned)(plan->cg * 128 * 16 + plan->cg * n_tile * 16);
+        plan->tpk = plan->groups > 1 ? 1 : 8 / cchunks;
+        if (plan->tpk > taps) plan->tpk = taps;
+        if (plan->tpk < 1) plan->tpk = 1;
+        const int planes = plan->groups > 1 ? plan->cg : plan->tpk * cchunks;
+        const unsigned stage = (unsigned)(planes * 128 * 16 + planes * n_tile * 16);
         plan->a_stages = 6;
         while (plan->a_stages > 2 && smem + plan->a_stages * stage > 120 * 1024) --plan->a_stages;
         plan->b_stages = plan->a_stages;
@@ -755,8 +767,11 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.n_tile = plan.n_tile; p.n_tiles = plan.n_tiles; p.tmem_cols = plan.tmem_cols;
     const long long m_tiles = (p.m_total + 127) / 128;
     p.total_tiles = (int)(m_tiles * plan.n_tiles);
-    p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : plan.cg * 128 * 16;
-    p.b_stage_bytes = plan.cg * plan.n_tile * 16;
+    const int gplanes = plan.groups > 1 ? plan.cg : plan.tpk * p.cchunks;      // gather: planes per stage
+    p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : gplanes * 128 * 16;
+    p.b_stage_bytes = plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
+    p.tpk = plan.tpk > 0 ? plan.tpk : 1;
+    p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
     p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
     p.status = d_status;
     p.div_ntiles = make_fastdiv((uint32_t)plan.n_tiles);

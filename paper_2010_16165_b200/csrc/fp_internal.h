@@ -66,7 +66,7 @@ void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_i
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
                     int stride, int pad, cudaStream_t st);
 void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
-                 int n_classes, float* logits, cudaStream_t st);
+                 int n_classes, float* logits, float* pool_scratch, cudaStream_t st);
 void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
                                cudaStream_t st);
 
@@ -86,6 +86,7 @@ struct ConvPlanTC {
     int halo;             // flat: vectors fetched before and after the 128 positions of a tile
     int rows_a;           // flat: vectors per chunk per tile (128 + 2*halo, rounded up to 8)
     int a_stages, b_stages;
+    int tpk;              // gather: filter taps per K block (several when the channel count is small)
     int n_tile, n_tiles;  // filters per CTA tile (multiple of 16, <= 256)
     int tmem_cols;
     unsigned smem_bytes;

@@ -106,47 +106,75 @@ __global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y,
     }
 }
 
-// Head: spatial sum per channel (fp32), then logits[k] = sum_c s[c] * Wfc[k][c] + b[k] with the
-// 1/(H*W) of the average already folded into Wfc.  One block per image; channel sums are reduced
-// through shuffles into shared memory; one warp per class row with a shuffle reduction.
+// Head, step 1: spatial sum per channel in fp32.  One warp per (image, chunk of 8 channels): lanes
+// stride over the interior positions with 16-byte loads, shuffle-reduce, and write 8 sums.
 template <bool BF16>
-__global__ void head_kernel(const void* __restrict__ x, int N, int H, int W, int chunks, const float* __restrict__ fcw,
-                            const float* __restrict__ fcb, int n_classes, float* __restrict__ logits) {
-    extern __shared__ float sums[];          // chunks * 8
+__global__ void pool_sum_kernel(const void* __restrict__ x, int N, int H, int W, int chunks, float* __restrict__ sums) {
     const int Wp = W + 2, P2 = (H + 2) * Wp, HW = H * W;
-    const size_t n = blockIdx.x;
     const size_t plane = (size_t)N * P2;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int j = warp; j < chunks; j += nwarps) {
-        float acc[8];
+    const int lane = threadIdx.x & 31;
+    const size_t warp = (blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5;
+    if (warp >= (size_t)N * chunks) return;
+    const int j = (int)(warp % chunks);
+    const size_t n = warp / chunks;
+    float acc[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
-        for (int i = lane; i < HW; i += 32) {
-            const int h = i / W, w = i - h * W;
-            float v[8];
-            load_vec8<BF16>(x, (size_t)j * plane + n * P2 + (size_t)(h + 1) * Wp + (w + 1), v);
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
+    for (int i = lane; i < HW; i += 32) {
+        const int h = i / W, w = i - h * W;
+        float v[8];
+        load_vec8<BF16>(x, (size_t)j * plane + n * P2 + (size_t)(h + 1) * Wp + (w + 1), v);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] += v[e];
-        }
+        for (int e = 0; e < 8; ++e) acc[e] += v[e];
+    }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+    for (int e = 0; e < 8; ++e) {
 #pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], d);
-        }
-        if (lane == 0) {
+        for (int d = 16; d >= 1; d >>= 1) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], d);
+    }
+    if (lane == 0) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) sums[j * 8 + e] = acc[e];
-        }
+        for (int e = 0; e < 8; ++e) sums[n * (size_t)chunks * 8 + j * 8 + e] = acc[e];
+    }
+}
+
+// Head, step 2: logits[n][k] = sum_c sums[n][c] * Wfc[k][c] + b[k]; the 1/(H*W) of the average is
+// already folded into Wfc.  A block handles 4 images x 32 classes: the channel sums of its images sit
+// in shared memory and every FC row it reads serves all four images.
+constexpr int kFcImages = 4, kFcClasses = 32;
+__global__ void fc_kernel(const float* __restrict__ sums, int N, int C_pad, const float* __restrict__ fcw,
+                          const float* __restrict__ fcb, int n_classes, float* __restrict__ logits) {
+    extern __shared__ float sh[];          // kFcImages * C_pad
+    const int n0 = blockIdx.x * kFcImages, k0 = blockIdx.y * kFcClasses;
+    for (int i = threadIdx.x; i < kFcImages * C_pad; i += blockDim.x) {
+        const int img = i / C_pad;
+        sh[i] = (n0 + img < N) ? sums[(size_t)(n0 + img) * C_pad + (i - img * C_pad)] : 0.0f;
     }
     __syncthreads();
-    const int C_pad = chunks * 8;
-    for (int k = warp; k < n_classes; k += nwarps) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int kk = warp; kk < kFcClasses; kk += nwarps) {
+        const int k = k0 + kk;
+        if (k >= n_classes) break;
         const float* wr = fcw + (size_t)k * C_pad;
-        float s = 0.0f;
-        for (int c = lane; c < C_pad; c += 32) s = fmaf(sums[c], wr[c], s);
+        float acc[kFcImages];
 #pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-        if (lane == 0) logits[n * n_classes + k] = s + (fcb ? fcb[k] : 0.0f);
+        for (int i = 0; i < kFcImages; ++i) acc[i] = 0.0f;
+        for (int c = lane; c < C_pad; c += 32) {
+            const float wv = wr[c];
+#pragma unroll
+            for (int i = 0; i < kFcImages; ++i) acc[i] = fmaf(sh[i * C_pad + c], wv, acc[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < kFcImages; ++i) {
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], d);
+        }
+        if (lane == 0) {
+            const float b = fcb ? fcb[k] : 0.0f;
+#pragma unroll
+            for (int i = 0; i < kFcImages; ++i)
+                if (n0 + i < N) logits[(size_t)(n0 + i) * n_classes + k] = acc[i] + b;
+        }
     }
 }
 
@@ -196,10 +224,13 @@ void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, in
 }
 
 void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
-                 int n_classes, float* logits, cudaStream_t st) {
-    const size_t smem = (size_t)C_pad * sizeof(float);
-    if (is_bf16) head_kernel<true><<<N, 256, smem, st>>>(x, N, H, W, C_pad / 8, fcw, fcb, n_classes, logits);
-    else head_kernel<false><<<N, 256, smem, st>>>(x, N, H, W, C_pad / 8, fcw, fcb, n_classes, logits);
+                 int n_classes, float* logits, float* pool_scratch, cudaStream_t st) {
+    const size_t warps = (size_t)N * (C_pad / 8);
+    const int blocks = (int)((warps * 32 + 255) / 256);
+    if (is_bf16) pool_sum_kernel<true><<<blocks, 256, 0, st>>>(x, N, H, W, C_pad / 8, pool_scratch);
+    else pool_sum_kernel<false><<<blocks, 256, 0, st>>>(x, N, H, W, C_pad / 8, pool_scratch);
+    dim3 grid((N + kFcImages - 1) / kFcImages, (n_classes + kFcClasses - 1) / kFcClasses);
+    fc_kernel<<<grid, 256, (size_t)kFcImages * C_pad * sizeof(float), st>>>(pool_scratch, N, C_pad, fcw, fcb, n_classes, logits);
 }
 
 void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
