@@ -30,6 +30,22 @@ UNIT = "images/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def recorded_traffic(workload):
+    """DRAM bytes per conv launch from the committed ncu summary, or None when the kernel source has changed
+    since the counters were taken (or the summary is for another workload)."""
+    import hashlib
+    rec = os.path.join(ROOT, "profiles", "conv_tc_kernel_resnet56_b256.traffic.txt")
+    src = os.path.join(ROOT, "paper_2010_16165_b200", "csrc", "conv_tc.cu")
+    try:
+        kv = dict(l.split(":", 1) for l in open(rec) if ":" in l and not l.startswith("#"))
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+        if kv["workload"].strip() != workload or not sha.startswith(kv["kernel_sha256_prefix"].strip()):
+            return None
+        return float(kv["traffic_bytes_per_launch"])
+    except Exception:
+        return None
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -259,7 +275,7 @@ def run_gpu(args):
         roof = {"bound": "tensor", "achieved": conv_flops / (conv_ms * 1e-3) / 1e12,
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    roof["traffic"] = recorded_traffic(w.name)
     roof["peak_source"] = peak_kind
     roof["kernel"] = "conv_tc_kernel"
     roof["launches_per_step"] = n_conv
