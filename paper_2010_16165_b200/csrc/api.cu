@@ -125,6 +125,7 @@ struct fp_handle_s {
     double* d_scores = nullptr; int32_t* d_rank = nullptr; uint8_t* d_mask = nullptr;
     std::map<GraphKey, cudaGraphExec_t> graphs;
     const void* last_input = nullptr; int last_batch = 0;
+    int stem_packed = 0;                   // network input stored in the packed form of a 7x7/2 first convolution
     int act_is_bf16() const { return compute != FP_COMPUTE_FP32; }
     size_t act_elem() const { return act_is_bf16() ? 2 : 4; }
     size_t in_elem() const { return in_dtype == FP_DTYPE_BF16 ? 2 : 4; }
@@ -488,6 +489,13 @@ fp_status replan(fp_handle h) {
         t.keep.resize(t.C);
         for (int c = 0; c < t.C; ++c) t.keep[c] = c;
     }
+    // A 7x7 / stride-2 / pad-3 first convolution on <= 3 channels runs as a 3x1 convolution over a packed
+    // copy of the input (tensor-core path only; the validation paths keep the plain form).
+    h->stem_packed = 0;
+    for (const FConv& f : h->convs)
+        if (f.src == 0 && h->compute == FP_COMPUTE_BF16_TC && uses[0].size() == 1 && f.R == 7 && f.S == 7 &&
+            f.stride == 2 && f.pad == 3 && f.C <= 3 && h->in_H % 2 == 0 && h->in_W % 2 == 0)
+            h->stem_packed = 1;
     for (const Op& op : h->ops) {
         if (op.kind == 0) {
             FConv& f = h->convs[op.idx];
@@ -517,10 +525,12 @@ fp_status replan(fp_handle h) {
             int32_t *d_row, *d_chan;
             TRY(upload_i32(h, row_src, &d_row));
             TRY(upload_i32(h, chan_src, &d_chan));
-            const size_t cnt = (size_t)f.K_pad * f.R * f.S * f.C_pad;
+            const bool packed_stem = h->stem_packed && f.src == 0;
+            const size_t cnt = packed_stem ? (size_t)f.K_pad * 3 * 80 : (size_t)f.K_pad * f.R * f.S * f.C_pad;
             TRY(dev_alloc(h->pack_buffers, &f.d_wp, cnt * h->act_elem()));
             TRY(dev_alloc(h->pack_buffers, (void**)&f.d_bp, (size_t)f.K_pad * sizeof(float)));
-            fp::launch_repack_conv(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad,
+            if (packed_stem) fp::launch_repack_stem(f.d_w32, f.C, d_row, f.K_pad, (__nv_bfloat16*)f.d_wp, st);
+            else fp::launch_repack_conv(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad,
                                    bf16 ? (__nv_bfloat16*)f.d_wp : nullptr, bf16 ? nullptr : (float*)f.d_wp, st);
             fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);
         } else if (op.kind == 1) {
@@ -562,6 +572,8 @@ fp_status replan(fp_handle h) {
             // planar-8 with border, plus guard vectors before and after (halo reads of the first/last tiles)
             const size_t vec_bytes = 8 * h->act_elem();
             t.bytes = ((size_t)(t.C_pad / 8) * h->max_batch * (t.H + 2) * (t.W + 2) + 2 * (size_t)fp::kGuardVectors) * vec_bytes;
+            if (tid == 0 && h->stem_packed)
+                t.bytes = ((size_t)10 * h->max_batch * (t.H / 2 + 2) * (t.W / 2 + 2) + 2 * (size_t)fp::kGuardVectors) * vec_bytes;
             int best = -1;
             if (!h->keep_outputs)
                 for (int b = 0; b < (int)bufs.size(); ++b)
@@ -587,6 +599,9 @@ fp_status replan(fp_handle h) {
         a.x = src.d; a.y = out.d; a.w = f.d_wp; a.bias = f.d_bp;
         a.N = h->max_batch; a.H = src.H; a.W = src.W; a.C_pad = f.C_pad; a.P = out.H; a.Q = out.W;
         a.K_pad = f.K_pad; a.R = f.R; a.S = f.S; a.stride = f.stride; a.pad = f.pad; a.relu = f.relu;
+        if (h->stem_packed && f.src == 0) {      // 3x1 stride-1 convolution over the packed input, at the output resolution
+            a.H = out.H; a.W = out.W; a.C_pad = 80; a.R = 3; a.S = 1; a.stride = 1; a.pad = 1;
+        }
         a.res_mode = f.res_mode;
         if (f.res_mode) {
             const Tensor& r = h->tensors[f.res_tid];
@@ -612,7 +627,8 @@ void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float*
     const int bf16 = h->act_is_bf16();
     if (op.kind == 3) {
         const Tensor& t = h->tensors[0];
-        fp::launch_input_to_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, st);
+        if (h->stem_packed) fp::launch_input_to_stem_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, batch, t.C, t.H, t.W, st);
+        else fp::launch_input_to_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, st);
     } else if (op.kind == 0) {
         FConv& f = h->convs[op.idx];
         fp::ConvArgs a = f.args;
@@ -926,6 +942,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             if (index < 0 || index >= (int)h->ops.size() || h->ops[index].kind == 2)
                 return fail(FP_ERR_ARG, "fp_query: operator %d has no activation output", index);
             if (h->last_batch <= 0) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
+            if (h->ops[index].kind == 3 && h->stem_packed) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is stored in packed form");
             const Op& op = h->ops[index];
             const int tid = op.kind == 0 ? h->convs[op.idx].out : op.kind == 1 ? h->pools[op.idx].out : 0;
             const Tensor& t = h->tensors[tid];

@@ -9,9 +9,9 @@
 //   Operands      K-major, no swizzle: an operand block is a stack of 16-byte rows (8 channels of
 //                 one position / one filter); the two 8-channel halves of a K=16 MMA step live in
 //                 two such stacks ("planes"), `LBO` apart.
-//   FLAT modes    stride-1 "same" convolutions (3x3 pad 1, 1x1 pad 0).  Because every chunk plane
+//   FLAT modes    stride-1 "same" convolutions (3x3 pad 1, 3x1 pad 1x0, 1x1 pad 0).  Because every chunk plane
 //                 is contiguous over flat positions, the activations a tile needs - its 128
-//                 positions plus a halo of (W+3) before and after - are ONE contiguous run per
+//                 positions plus a halo of (W+3) before and after (3x3) - are ONE contiguous run per
 //                 chunk, fetched with one bulk copy.  The operand of filter tap (r,s) is the same
 //                 shared-memory block read from a start address shifted by (r-1)*(W+2)+(s-1) rows,
 //                 so each activation is fetched once per tile, not once per tap.  The zero border
@@ -155,33 +155,33 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo) 
 // unrolled so that the single issuing thread spends a handful of instructions per MMA.  Operand
 // descriptors differ only in their low words: one address unit is one 16-byte row, so a tap's
 // activation operand is `a_lo + r*Wp + s` and a K step advances both operands by two planes.
-template <int R, int KSTEPS>
+template <int R, int S, int KSTEPS>
 __device__ __forceinline__ void issue_flat_resident(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t Wp,
                                                     uint32_t a_ks, uint32_t b_ks, uint32_t b_tap, uint32_t idesc,
                                                     uint32_t accumulate) {
 #pragma unroll
     for (int r = 0; r < R; ++r) {
 #pragma unroll
-        for (int sx = 0; sx < R; ++sx) {
+        for (int sx = 0; sx < S; ++sx) {
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
                 umma_bf16_lo(d_tmem, a_lo + (uint32_t)r * Wp + (uint32_t)sx + (uint32_t)ks * a_ks,
-                             b_lo + (uint32_t)(r * R + sx) * b_tap + (uint32_t)ks * b_ks, idesc,
+                             b_lo + (uint32_t)(r * S + sx) * b_tap + (uint32_t)ks * b_ks, idesc,
                              (r | sx | ks) ? 1u : accumulate);
             }
         }
     }
 }
 
-template <int R>
+template <int R, int S>
 __device__ __forceinline__ void issue_flat_resident_k(int ksteps, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
                                                       uint32_t Wp, uint32_t a_ks, uint32_t b_ks, uint32_t b_tap,
                                                       uint32_t idesc, uint32_t accumulate) {
     switch (ksteps) {
-        case 1: issue_flat_resident<R, 1>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
-        case 2: issue_flat_resident<R, 2>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
-        case 3: issue_flat_resident<R, 3>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
-        default: issue_flat_resident<R, 4>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        case 1: issue_flat_resident<R, S, 1>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        case 2: issue_flat_resident<R, S, 2>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        case 3: issue_flat_resident<R, S, 3>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
+        default: issue_flat_resident<R, S, 4>(d_tmem, a_lo, b_lo, Wp, a_ks, b_ks, b_tap, idesc, accumulate); break;
     }
 }
 
@@ -357,10 +357,12 @@ conv_tc_kernel(const TcParams p) {
                         const uint32_t b_ks = 2u * (uint32_t)(MODE == MODE_FLAT_RESIDENT ? p.a.K_pad : p.n_tile);
                         const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.a.K_pad);
                         if (MODE == MODE_FLAT_RESIDENT) {
-                            if (p.a.R == 3)
-                                issue_flat_resident_k<3>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
+                            if (p.a.R == 3 && p.a.S == 3)
+                                issue_flat_resident_k<3, 3>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
+                            else if (p.a.R == 3)
+                                issue_flat_resident_k<3, 1>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
                             else
-                                issue_flat_resident_k<1>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
+                                issue_flat_resident_k<1, 1>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
                             accumulate = 1;
                         } else
                         for (int r = 0; r < p.a.R && ok; ++r) {
@@ -655,8 +657,8 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (a.W > kMaxWidth || a.Q > kMaxWidth) { snprintf(err, err_len, "images wider than %d are not supported", kMaxWidth); return 1; }
     const int cchunks = a.C_pad / 8;
     const int taps = a.R * a.S;
-    plan->flat = (a.stride == 1 && a.R == a.S && a.P == a.H && a.Q == a.W &&
-                  ((a.R == 1 && a.pad == 0) || (a.R == 3 && a.pad == 1))) ? 1 : 0;
+    plan->flat = (a.stride == 1 && a.P == a.H && a.Q == a.W &&
+                  ((a.R == 1 && a.S == 1 && a.pad == 0) || (a.R == 3 && (a.S == 3 || a.S == 1) && a.pad == 1))) ? 1 : 0;
     plan->cg = cchunks < 8 ? cchunks : 8;
     plan->groups = (cchunks + plan->cg - 1) / plan->cg;
     const long long m_total = (long long)a.N * (a.P + 2) * (a.Q + 2);
@@ -682,7 +684,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     unsigned smem = (unsigned)sizeof(Ctrl) + (unsigned)a.K_pad * 4u + 1024u;
     int want_ctas = 1;
     if (plan->flat) {
-        plan->halo = a.pad * (a.W + 3);
+        plan->halo = ((a.R - 1) / 2) * (a.W + 2) + (a.S - 1) / 2;      // rows above + columns to the left
         plan->rows_a = round_up_i(128 + 2 * plan->halo, 8);
         const unsigned a_stage = (unsigned)(plan->cg * plan->rows_a * 16);
         if (bank_fits) {

@@ -33,7 +33,7 @@ struct ConvArgs {
     const void* res;      // residual operand or nullptr
     const void* w;        // packed filters [R*S][C_pad/8][K_pad][8]
     const float* bias;    // [K_pad]
-    int N, H, W, C_pad, P, Q, K_pad, R, S, stride, pad;
+    int N, H, W, C_pad, P, Q, K_pad, R, S, stride, pad;   // pad: rows; columns are padded by pad when S == R, by (S-1)/2 otherwise
     int relu;
     int res_mode;         // 0 none, 1 same shape as y, 2 subsample + zero-channel pad
     int res_H, res_W, res_C_pad, res_C, res_pad_lo, res_stride;
@@ -58,11 +58,14 @@ void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, i
 // FC matrix: packed[k][cp] = w[k][chan_src[cp]] * scale
 void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int C_pad, float scale, float* out,
                       cudaStream_t st);
+// 7x7 first convolution as a 3x1 convolution over the packed network input (80 channels)
+void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st);
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st);
 
 // Memory-bound operators ------------------------------------------------------------------
 void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
                             int C_pad, cudaStream_t st);
+void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, cudaStream_t st);
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
                     int stride, int pad, cudaStream_t st);
 void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,

@@ -70,6 +70,49 @@ __global__ void input_to_planar_kernel(const void* __restrict__ in, int in_is_bf
     }
 }
 
+// Network input for a 7x7 / stride-2 / pad-3 first convolution with at most 3 input channels, packed so
+// that the convolution becomes a stride-1 3x1 convolution at the output resolution (P = H/2, Q = W/2):
+// the 7 horizontal taps and the input channels become 24 packed channels j = s*C + c, and the input
+// rows are split by parity into three 24-channel groups
+//     E (chunks 0-2):  E [p][q][j] = x[c][2p    ][2q + s - 3]
+//     O'(chunks 3-5):  O'[p][q][j] = x[c][2p - 1][2q + s - 3]      (odd rows, shifted down by one)
+//     O (chunks 6-8):  O [p][q][j] = x[c][2p + 1][2q + s - 3]
+// (chunk 9 is zero padding to an even chunk count).  Output row p needs input rows 2p-3 .. 2p+3, which
+// are O'(p-1), E(p-1), O'(p), E(p), O'(p+1), E(p+1), O(p+1): vertical offsets -1, 0, +1 only.
+__global__ void input_to_stem_planar_kernel(const void* __restrict__ in, int in_is_bf16, __nv_bfloat16* __restrict__ out,
+                                            int N, int C, int H, int W) {
+    const int P = H / 2, Q = W / 2, Qp = Q + 2, P2 = (P + 2) * Qp;
+    const size_t plane = (size_t)N * P2;
+    const size_t total = plane * 10;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int j8 = (int)(i / plane);             // chunk 0..9
+        const size_t f = i - (size_t)j8 * plane;
+        const size_t n = f / P2;
+        const int rem = (int)(f - n * P2);
+        const int p = rem / Qp - 1, q = rem % Qp - 1;
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+        if (j8 < 9 && p >= 0 && p < P && q >= 0 && q < Q) {
+            const int group = j8 / 3;                // 0 = E, 1 = O', 2 = O
+            const int ih = group == 0 ? 2 * p : group == 1 ? 2 * p - 1 : 2 * p + 1;
+            if (ih >= 0 && ih < H) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int j = (j8 % 3) * 8 + e;  // packed channel s*C + c
+                    const int sx = j / C, c = j - sx * C;
+                    const int iw = 2 * q + sx - 3;
+                    if (sx < 7 && iw >= 0 && iw < W) {
+                        const size_t src = ((n * C + c) * H + ih) * W + iw;
+                        v[e] = in_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)in)[src]) : ((const float*)in)[src];
+                    }
+                }
+            }
+        }
+        store_vec8<true>(out, i, v);
+    }
+}
+
 // Max pooling; padded positions never win.  Output border positions are written as zeros.
 template <bool BF16>
 __global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y, int N, int H, int W, int chunks, int P,
@@ -214,6 +257,11 @@ void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_i
     const size_t n = (size_t)N * (H + 2) * (W + 2) * (C_pad / 8);
     if (out_is_bf16) input_to_planar_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8);
     else input_to_planar_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8);
+}
+
+void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, cudaStream_t st) {
+    const size_t n = (size_t)N * (H / 2 + 2) * (W / 2 + 2) * 10;
+    input_to_stem_planar_kernel<<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W);
 }
 
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,

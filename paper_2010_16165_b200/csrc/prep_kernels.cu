@@ -114,6 +114,35 @@ __global__ void repack_conv_kernel(const float* __restrict__ w, int C, int RS, c
     }
 }
 
+// Filters of a 7x7 first convolution in the order the packed network input wants them (see
+// input_to_stem_planar_kernel): a 3x1 convolution over 80 packed channels.  Tap dr (0..2 = offsets
+// -1,0,+1), chunk 0-2 (group E) take filter row r = 2*dr + 1, chunks 3-5 (O') take r = 2*dr, chunks
+// 6-8 (O) take r = 6 at dr = 2 only; packed channel j = s*C + c within a group; everything else zero.
+__global__ void repack_stem_kernel(const float* __restrict__ w, int C, const int32_t* __restrict__ row_src, int K_pad,
+                                   __nv_bfloat16* __restrict__ out) {
+    const size_t total = (size_t)3 * 10 * K_pad * 8;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int e = (int)(i % 8);
+        size_t t = i / 8;
+        const int kr = (int)(t % K_pad); t /= K_pad;
+        const int chunk = (int)(t % 10);
+        const int dr = (int)(t / 10);
+        float v = 0.0f;
+        const int ks = row_src[kr];
+        if (ks >= 0 && chunk < 9) {
+            const int group = chunk / 3;
+            const int j = (chunk % 3) * 8 + e;
+            const int sx = j / C, c = j - sx * C;
+            int r = -1;
+            if (group == 0) r = 2 * dr + 1;
+            else if (group == 1) r = 2 * dr;
+            else if (dr == 2) r = 6;
+            if (r >= 0 && sx < 7) v = w[(((size_t)ks * C + c) * 7 + r) * 7 + sx];
+        }
+        out[i] = __float2bfloat16_rn(v);
+    }
+}
+
 __global__ void repack_fc_kernel(const float* __restrict__ w, int C, int K, const int32_t* __restrict__ chan_src,
                                  int C_pad, float scale, float* __restrict__ out) {
     const size_t total = (size_t)K * C_pad;
@@ -171,6 +200,10 @@ void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, i
                         int C_pad, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st) {
     const size_t n = (size_t)K_pad * RS * C_pad;
     repack_conv_kernel<<<blocks_for(n, 256), 256, 0, st>>>(w, C, RS, row_src, K_pad, chan_src, C_pad, out_bf16, out_f32);
+}
+
+void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st) {
+    repack_stem_kernel<<<blocks_for((size_t)240 * K_pad, 256), 256, 0, st>>>(w, C, row_src, K_pad, out);
 }
 
 void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int C_pad, float scale, float* out,
