@@ -204,8 +204,11 @@ __device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
     atomicExch(status, code);
 }
 
-template <int MODE>
-__global__ void __launch_bounds__(MODE == MODE_GATHER ? 320 : MODE == MODE_FLAT_STREAM ? 224 : 192)
+// Threads: warp 0 producer, warp 1 MMA, EPI epilogue warps (4, or 8 for wide filter tiles: two warps per
+// TMEM lane quarter, each taking half of the columns), then 1 filter-producer warp (FLAT_STREAM) or 4
+// loader warps (GATHER).
+template <int MODE, int EPI>
+__global__ void __launch_bounds__(64 + 32 * EPI + (MODE == MODE_GATHER ? 128 : MODE == MODE_FLAT_STREAM ? 32 : 0))
 conv_tc_kernel(const TcParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
@@ -232,7 +235,7 @@ conv_tc_kernel(const TcParams p) {
             mbar_init(b_full0 + 8 * s, 1);
             mbar_init(b_empty0 + 8 * s, 1);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 128); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 32 * EPI); }
         ctrl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -419,9 +422,10 @@ conv_tc_kernel(const TcParams p) {
             }
             if (!ok) raise(ctrl, p.status, 2);
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + EPI) {
         // ------------------------------ epilogue ----------------------------------
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int half = (warp - 2) >> 2;             // with 8 epilogue warps: which half of the columns
         const int row = quarter * 32 + lane;          // accumulator row = position within the tile
         uint32_t acc_phase0 = 0, acc_phase1 = 0;
         int local = 0;
@@ -444,8 +448,13 @@ conv_tc_kernel(const TcParams p) {
             int cols = p.a.K_pad - k_base;
             if (cols > p.n_tile) cols = p.n_tile;
             const long long vec0 = (long long)(k_base >> 3) * p.plane_out + f;     // vector of columns 0..7
-            // the same-shape residual of the first 64 columns is requested before the accumulator is
-            // waited for; later columns are requested four 16-column chunks ahead
+            int c_begin = 0, c_end = cols;
+            if (EPI == 8) {
+                const int first = ((cols >> 4) + 1) / 2 * 16;                      // columns of the first half
+                if (half) c_begin = first; else c_end = first;
+            }
+            // the same-shape residual of this warp's first 64 columns is requested before the accumulator
+            // is waited for; later columns are requested four 16-column chunks ahead
             uint4 rq[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) rq[i] = make_uint4(0, 0, 0, 0);
@@ -453,7 +462,7 @@ conv_tc_kernel(const TcParams p) {
             if (res1) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                    if (i * 8 < cols) rq[i] = __ldg(res + vec0 + (long long)i * p.plane_out);
+                    if (c_begin + i * 8 < c_end) rq[i] = __ldg(res + vec0 + (long long)((c_begin >> 3) + i) * p.plane_out);
             }
             ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
@@ -466,7 +475,7 @@ conv_tc_kernel(const TcParams p) {
                 res_vec = (long long)n * rP2 + (long long)((hp - 1) * p.a.res_stride + 1) * rWp + ((wq - 1) * p.a.res_stride + 1);
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.n_tile);
-            for (int c0 = 0; c0 < cols; c0 += 16) {
+            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 uint32_t v[16];
                 __syncwarp();
                 tmem_ld16(taddr + c0, v);
@@ -537,7 +546,7 @@ conv_tc_kernel(const TcParams p) {
                 // rotate the residual queue and refill its tail
 #pragma unroll
                 for (int i = 0; i < 6; ++i) rq[i] = rq[i + 2];
-                if (res1 && c0 + 64 < cols) {
+                if (res1 && c0 + 64 < c_end) {
                     const long long vn = vec0 + (long long)((c0 + 64) >> 3) * p.plane_out;
                     rq[6] = __ldg(res + vn);
                     rq[7] = __ldg(res + vn + p.plane_out);
@@ -549,7 +558,7 @@ conv_tc_kernel(const TcParams p) {
         if (!ok && lane == 0) raise(ctrl, p.status, 3);
     } else if (MODE == MODE_FLAT_STREAM) {
         // ------------------------------ filter producer (streamed filters) --------------
-        if (warp == 6 && lane == 0) {
+        if (warp == 2 + EPI && lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
@@ -576,7 +585,7 @@ conv_tc_kernel(const TcParams p) {
         }
     } else if (MODE == MODE_GATHER) {
         // ------------------------------ loader threads (gathered activations) -----------
-        const int m = threadIdx.x - 192;             // 0..127: row of the tile this thread fills
+        const int m = threadIdx.x - 32 * (2 + EPI);  // 0..127: row of the tile this thread fills
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
@@ -646,6 +655,12 @@ FastDiv make_fastdiv(uint32_t d) {
 }
 int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
+const void* kernel_for(int mode, int epi) {
+    if (mode == MODE_FLAT_RESIDENT) return epi == 8 ? (const void*)conv_tc_kernel<MODE_FLAT_RESIDENT, 8> : (const void*)conv_tc_kernel<MODE_FLAT_RESIDENT, 4>;
+    if (mode == MODE_FLAT_STREAM) return epi == 8 ? (const void*)conv_tc_kernel<MODE_FLAT_STREAM, 8> : (const void*)conv_tc_kernel<MODE_FLAT_STREAM, 4>;
+    return epi == 8 ? (const void*)conv_tc_kernel<MODE_GATHER, 8> : (const void*)conv_tc_kernel<MODE_GATHER, 4>;
+}
+
 constexpr unsigned kSmemMax = 232448u - 1024u;     // opt-in dynamic shared memory per CTA
 constexpr unsigned kSmemPerSm = 233472u;           // 228 KB per SM
 
@@ -666,10 +681,12 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (m_total + 128 >= (1ll << 31)) { snprintf(err, err_len, "more than 2^31 output positions"); return 1; }
 
     // --- filter tile ---
-    int n_tiles = (a.K_pad + 255) / 256;
+    // at most 128 filters per tile: two CTAs then share an SM's 512 tensor-memory columns, which doubles the
+    // epilogue warps and the loads in flight; a 128-wide MMA already runs at the full tensor rate
+    int n_tiles = (a.K_pad + 127) / 128;
     int n_tile = round_up_i((a.K_pad + n_tiles - 1) / n_tiles, 16);
     const long long bank = (long long)taps * a.C_pad * a.K_pad * 2;
-    const bool bank_fits = plan->flat && n_tiles == 1 && bank <= 100 * 1024;
+    const bool bank_fits = plan->flat && bank <= 100 * 1024;
     if (!bank_fits) {
         while (m_tiles * n_tiles < 148 && n_tile > 64) {      // few position tiles: split the filters to fill the SMs
             n_tiles *= 2;
@@ -725,26 +742,25 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (ctas > tmem_ctas) ctas = tmem_ctas;
     if (ctas > want_ctas) ctas = want_ctas;
     if (ctas < 1) ctas = 1;
+    const int epi = n_tile >= 64 ? 8 : 4;
+    plan->epi_warps = epi;
+    const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
+    const void* fn = kernel_for(mode, epi);
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e0 = cudaFuncSetAttribute(conv_tc_kernel<MODE_FLAT_RESIDENT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
-        cudaError_t e1 = cudaFuncSetAttribute(conv_tc_kernel<MODE_FLAT_STREAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
-        cudaError_t e2 = cudaFuncSetAttribute(conv_tc_kernel<MODE_GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax);
-        if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess) {
-            snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
-            cudaGetLastError();
-            return 1;
-        }
+        for (int m = 0; m < 3; ++m)
+            for (int e = 4; e <= 8; e += 4)
+                if (cudaFuncSetAttribute(kernel_for(m, e), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
+                    snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
+                    cudaGetLastError();
+                    return 1;
+                }
         attr_set = true;
     }
-    // persistent grid: exactly as many CTAs as can be resident at once (registers, threads, shared memory)
     cudaFuncAttributes fa;
-    cudaError_t oe;
-    if (!plan->flat) oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_GATHER>);
-    else if (plan->b_resident) oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_FLAT_RESIDENT>);
-    else oe = cudaFuncGetAttributes(&fa, conv_tc_kernel<MODE_FLAT_STREAM>);
+    cudaError_t oe = cudaFuncGetAttributes(&fa, fn);
     if (oe != cudaSuccess) { snprintf(err, err_len, "cudaFuncGetAttributes: %s", cudaGetErrorString(oe)); cudaGetLastError(); return 1; }
-    const int threads = !plan->flat ? 320 : plan->b_resident ? 192 : 224;
+    const int threads = 64 + 32 * epi + (mode == MODE_GATHER ? 128 : mode == MODE_FLAT_STREAM ? 32 : 0);
     const int regs_per_warp = round_up_i(fa.numRegs * 32, 256);
     int occ = 65536 / (regs_per_warp * (threads / 32));
     if (occ > 2048 / threads) occ = 2048 / threads;
@@ -785,7 +801,8 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(!plan.flat ? 320u : plan.b_resident ? 192u : 224u);
+    const int mode = !plan.flat ? MODE_GATHER : plan.b_resident ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
+    cfg.blockDim = dim3((unsigned)(64 + 32 * plan.epi_warps + (mode == MODE_GATHER ? 128 : mode == MODE_FLAT_STREAM ? 32 : 0)));
     cfg.dynamicSmemBytes = plan.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -793,9 +810,8 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (!plan.flat) cudaLaunchKernelEx(&cfg, conv_tc_kernel<MODE_GATHER>, p);
-    else if (plan.b_resident) cudaLaunchKernelEx(&cfg, conv_tc_kernel<MODE_FLAT_RESIDENT>, p);
-    else cudaLaunchKernelEx(&cfg, conv_tc_kernel<MODE_FLAT_STREAM>, p);
+    void* args[1] = {(void*)&p};
+    cudaLaunchKernelExC(&cfg, kernel_for(mode, plan.epi_warps), args);
 }
 
 }  // namespace fp
