@@ -57,6 +57,7 @@ struct TcParams {
     int taps, cchunks, cg, groups, halo, rows_a, a_stages, b_stages;
     int n_tile, n_tiles, tmem_cols, total_tiles;
     int tpk, kblocks;                   // gather: taps per K block, K blocks per tile
+    int tps;                            // streamed filters: 128-position tiles per pipeline step (share each filter block)
     int a_stage_bytes, b_stage_bytes, b_bank_bytes;
     int* status;
 };
@@ -276,7 +277,7 @@ conv_tc_kernel(const TcParams p) {
             bool ok = true;
             uint32_t stage = 0, phase = 0;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                const long long f0 = (long long)fdiv((uint32_t)tile, p.div_ntiles) * 128;
+                const long long f0 = (long long)fdiv((uint32_t)tile, p.div_ntiles) * p.tps * 128;
                 for (int g = 0; g < p.groups; ++g) {
                     bool w = true;
                     if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
@@ -295,34 +296,37 @@ conv_tc_kernel(const TcParams p) {
                 }
             }
             if (!ok && lane == 0) raise(ctrl, p.status, 1);
-        } else if (lane == 0) {
+        } else {
+            // GATHER: filters of each K block into the stage the loader threads fill, one lane per plane
             bool ok = true;
             uint32_t stage = 0, phase = 0;
-            {
-                // GATHER: filters of each (tap, K block) into the stage the loader threads fill
-                for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-                    const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
-                    int nrows = p.a.K_pad - nt * p.n_tile;
-                    if (nrows > p.n_tile) nrows = p.n_tile;
-                    for (int kb = 0; kb < p.kblocks; ++kb) {
-                        // a K block is either one tap x one channel group, or (few channels) several whole taps
-                        int tap0, g, ntap, cgg;
-                        if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
-                        else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
-                        if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                        const uint32_t fb = a_full0 + 8 * stage;
-                        const uint32_t dst = a_base + stage * (p.a_stage_bytes + p.b_stage_bytes) + p.a_stage_bytes;
-                        mbar_expect_tx(fb, (uint32_t)(ntap * cgg * nrows * 16));
-                        for (int tt = 0; tt < ntap; ++tt)
-                            for (int c = 0; c < cgg; ++c)
-                                bulk_copy(dst + (tt * cgg + c) * p.n_tile * 16,
-                                          wv + ((long long)(tap0 + tt) * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
-                                          (uint32_t)(nrows * 16), fb);
-                        if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
+            for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+                const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
+                int nrows = p.a.K_pad - nt * p.n_tile;
+                if (nrows > p.n_tile) nrows = p.n_tile;
+                for (int kb = 0; kb < p.kblocks; ++kb) {
+                    // a K block is either one tap x one channel group, or (few channels) several whole taps
+                    int tap0, g, ntap, cgg;
+                    if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
+                    else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
+                    bool w = true;
+                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w) { ok = false; break; }
+                    const uint32_t fb = a_full0 + 8 * stage;
+                    const uint32_t dst = a_base + stage * (p.a_stage_bytes + p.b_stage_bytes) + p.a_stage_bytes;
+                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(ntap * cgg * nrows * 16));
+                    __syncwarp();
+                    if (lane < ntap * cgg) {
+                        const int tt = lane / cgg, c = lane - tt * cgg;
+                        bulk_copy(dst + lane * p.n_tile * 16,
+                                  wv + ((long long)(tap0 + tt) * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
+                                  (uint32_t)(nrows * 16), fb);
                     }
+                    if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
                 }
             }
-            if (!ok) raise(ctrl, p.status, 1);
+            if (!ok && lane == 0) raise(ctrl, p.status, 1);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer --------------------------------
@@ -341,7 +345,7 @@ conv_tc_kernel(const TcParams p) {
                 if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
                 tc_fence_after();
                 const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.n_tile);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.tps * p.n_tile);
                 uint32_t accumulate = 0;
                 if (MODE != MODE_GATHER) {
                     // Descriptors differ only in their 16-byte start-address field, so the inner loops
@@ -377,12 +381,18 @@ conv_tc_kernel(const TcParams p) {
                                     tc_fence_after();
                                     b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
                                 }
-                                for (int ks = 0; ks < ksteps; ++ks) {
-                                    umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
-                                    accumulate = 1;
-                                    a_lo += a_ks;
-                                    b_lo += b_ks;
+                                // every 128-position tile of the step uses this filter block: its own accumulator,
+                                // its activation rows 128 further on
+                                for (int t = 0; t < p.tps; ++t) {
+                                    uint32_t a_t = a_lo + (uint32_t)(t * 128), b_t = b_lo;
+                                    const uint32_t d_t = d_tmem + (uint32_t)(t * p.n_tile);
+                                    for (int ks = 0; ks < ksteps; ++ks) {
+                                        umma_bf16_lo(d_t, a_t, b_t, idesc, accumulate | (uint32_t)(ks > 0));
+                                        a_t += a_ks;
+                                        b_t += b_ks;
+                                    }
                                 }
+                                accumulate = 1;
                                 if (MODE == MODE_FLAT_STREAM) {
                                     umma_commit(b_empty0 + 8 * b_stage);
                                     if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
@@ -436,14 +446,15 @@ conv_tc_kernel(const TcParams p) {
         for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++local) {
             const int mt = (int)fdiv((uint32_t)tile, p.div_ntiles);
             const int nt = tile - mt * p.n_tiles;
-            const long long f = (long long)mt * 128 + row;
+            const int acc = local & 1;
+            const uint32_t ph = acc ? acc_phase1 : acc_phase0;
+            for (int t = 0; t < p.tps; ++t) {
+            const long long f = ((long long)mt * p.tps + t) * 128 + row;
             const bool exists = f < p.m_total;
             const int n = (int)fdiv((uint32_t)f, p.div_p2out);
             const int rem = (int)f - n * p.P2_out;
             const int hp = (int)fdiv((uint32_t)rem, p.div_qp), wq = rem - hp * p.Qp;
             const bool interior = exists && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
-            const int acc = local & 1;
-            const uint32_t ph = acc ? acc_phase1 : acc_phase0;
             const int k_base = nt * p.n_tile;
             int cols = p.a.K_pad - k_base;
             if (cols > p.n_tile) cols = p.n_tile;
@@ -464,17 +475,19 @@ conv_tc_kernel(const TcParams p) {
                 for (int i = 0; i < 8; ++i)
                     if (c_begin + i * 8 < c_end) rq[i] = __ldg(res + vec0 + (long long)((c_begin >> 3) + i) * p.plane_out);
             }
-            ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
-            tc_fence_after();
+            if (t == 0) {
+                ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
+                tc_fence_after();
+            }
             long long res_vec = 0;
             if (p.a.res_mode == 2) {
                 const int rWp = p.a.res_W + 2, rP2 = (p.a.res_H + 2) * rWp;
                 res_vec = (long long)n * rP2 + (long long)((hp - 1) * p.a.res_stride + 1) * rWp + ((wq - 1) * p.a.res_stride + 1);
             }
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.n_tile);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((acc * p.tps + t) * p.n_tile);
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 uint32_t v[16];
                 __syncwarp();
@@ -552,15 +565,20 @@ conv_tc_kernel(const TcParams p) {
                     rq[7] = __ldg(res + vn + p.plane_out);
                 }
             }
+            }   // tiles of the step
+            if (!ok) break;
             tc_fence_before();
             mbar_arrive(tempty0 + 8 * acc);
         }
         if (!ok && lane == 0) raise(ctrl, p.status, 3);
     } else if (MODE == MODE_FLAT_STREAM) {
         // ------------------------------ filter producer (streamed filters) --------------
-        if (warp == 2 + EPI && lane == 0) {
+        if (warp == 2 + EPI) {
+            // One filter block per (K group, tap).  When a tile takes all filters the block's chunks are one
+            // contiguous run of the packed bank: a single copy; otherwise one lane per chunk copies its rows.
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            const bool whole = p.n_tiles == 1;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
                 const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
                 int nrows = p.a.K_pad - nt * p.n_tile;
@@ -569,19 +587,25 @@ conv_tc_kernel(const TcParams p) {
                     int cgg = p.cchunks - g * p.cg;
                     if (cgg > p.cg) cgg = p.cg;
                     for (int tap = 0; tap < p.taps; ++tap) {
-                        if (!mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                        bool w = true;
+                        if (lane == 0) w = mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                        w = __shfl_sync(0xffffffffu, w, 0);
+                        if (!w) { ok = false; break; }
                         const uint32_t fb = b_full0 + 8 * stage;
                         const uint32_t dst = b_base + stage * p.b_stage_bytes;
-                        mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
-                        for (int c = 0; c < cgg; ++c)
-                            bulk_copy(dst + c * p.n_tile * 16,
-                                      wv + ((long long)tap * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
-                                      (uint32_t)(nrows * 16), fb);
+                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
+                        __syncwarp();
+                        const uint4* src = wv + ((long long)tap * p.cchunks + g * p.cg) * p.a.K_pad + nt * p.n_tile;
+                        if (whole) {
+                            if (lane == 0) bulk_copy(dst, src, (uint32_t)(cgg * nrows * 16), fb);
+                        } else if (lane < cgg) {
+                            bulk_copy(dst + lane * p.n_tile * 16, src + (long long)lane * p.a.K_pad, (uint32_t)(nrows * 16), fb);
+                        }
                         if (++stage == (uint32_t)p.b_stages) { stage = 0; phase ^= 1; }
                     }
                 }
             }
-            if (!ok) raise(ctrl, p.status, 4);
+            if (!ok && lane == 0) raise(ctrl, p.status, 4);
         }
     } else if (MODE == MODE_GATHER) {
         // ------------------------------ loader threads (gathered activations) -----------
@@ -695,14 +719,22 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     }
     n_tiles = (a.K_pad + n_tile - 1) / n_tile;
     plan->n_tile = n_tile; plan->n_tiles = n_tiles;
-    plan->tmem_cols = pow2_at_least(2 * n_tile < 32 ? 32 : 2 * n_tile);
-    const int tmem_ctas = 512 / plan->tmem_cols;
 
     unsigned smem = (unsigned)sizeof(Ctrl) + (unsigned)a.K_pad * 4u + 1024u;
     int want_ctas = 1;
     if (plan->flat) {
         plan->halo = ((a.R - 1) / 2) * (a.W + 2) + (a.S - 1) / 2;      // rows above + columns to the left
-        plan->rows_a = round_up_i(128 + 2 * plan->halo, 8);
+        plan->tps = 1;
+        if (!bank_fits) {
+            // several 128-position tiles per step share every streamed filter block (less filter traffic)
+            for (int tps = 4; tps > 1; tps >>= 1) {
+                const unsigned a_try = (unsigned)(plan->cg * round_up_i(tps * 128 + 2 * plan->halo, 8) * 16);
+                if (2 * tps * n_tile <= 512 && tps * 128 + plan->halo + 8 <= kGuardVectors &&
+                    ((m_tiles + tps - 1) / tps) * n_tiles >= 148 &&
+                    smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * a_try <= kSmemMax) { plan->tps = tps; break; }
+            }
+        }
+        plan->rows_a = round_up_i(plan->tps * 128 + 2 * plan->halo, 8);
         const unsigned a_stage = (unsigned)(plan->cg * plan->rows_a * 16);
         if (bank_fits) {
             plan->b_resident = 1;
@@ -715,7 +747,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             plan->b_resident = 0;
             plan->b_stages = 4;
             const unsigned b_stage = (unsigned)(plan->cg * n_tile * 16);
-            plan->a_stages = 3;
+            plan->a_stages = plan->tps > 1 ? 2 : 3;
             while (plan->a_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->a_stages;
             while (plan->b_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->b_stages;
             smem += (unsigned)round_up_i((int)(plan->b_stages * b_stage), 128) + plan->a_stages * a_stage;
@@ -733,6 +765,9 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         smem += plan->a_stages * stage;
         want_ctas = 2;
     }
+    if (plan->tps < 1) plan->tps = 1;
+    plan->tmem_cols = pow2_at_least(2 * plan->tps * n_tile < 32 ? 32 : 2 * plan->tps * n_tile);
+    const int tmem_ctas = 512 / plan->tmem_cols;
     if (smem > kSmemMax) { snprintf(err, err_len, "tile does not fit shared memory (%u bytes)", smem); return 1; }
     // co-resident CTAs must not ask for more than the 512 tensor-memory columns of an SM
     const unsigned min_smem = kSmemPerSm / (unsigned)(tmem_ctas + 1) + 1u;
@@ -784,7 +819,8 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.halo = plan.halo; p.rows_a = plan.rows_a; p.a_stages = plan.a_stages; p.b_stages = plan.b_stages;
     p.n_tile = plan.n_tile; p.n_tiles = plan.n_tiles; p.tmem_cols = plan.tmem_cols;
     const long long m_tiles = (p.m_total + 127) / 128;
-    p.total_tiles = (int)(m_tiles * plan.n_tiles);
+    p.tps = plan.tps > 0 ? plan.tps : 1;
+    p.total_tiles = (int)(((m_tiles + p.tps - 1) / p.tps) * plan.n_tiles);
     const int gplanes = plan.groups > 1 ? plan.cg : plan.tpk * p.cchunks;      // gather: planes per stage
     p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : gplanes * 128 * 16;
     p.b_stage_bytes = plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;

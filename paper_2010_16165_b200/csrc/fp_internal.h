@@ -92,6 +92,7 @@ struct ConvPlanTC {
     int tpk;              // gather: filter taps per K block (several when the channel count is small)
     int n_tile, n_tiles;  // filters per CTA tile (multiple of 16, <= 256)
     int epi_warps;        // 4, or 8 for wide filter tiles
+    int tps;              // streamed filters: 128-position tiles per pipeline step
     int tmem_cols;
     unsigned smem_bytes;
     int ctas_per_sm;
