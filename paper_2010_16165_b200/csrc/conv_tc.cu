@@ -186,6 +186,24 @@ __device__ __forceinline__ void issue_flat_resident_k(int ksteps, uint32_t d_tme
     }
 }
 
+// The K=16 steps of one (tap, K group) block for one accumulator, unrolled.
+template <int KSTEPS>
+__device__ __forceinline__ void issue_ksteps_n(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_ks, uint32_t b_ks,
+                                               uint32_t idesc, uint32_t accumulate) {
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks)
+        umma_bf16_lo(d_tmem, a_lo + (uint32_t)ks * a_ks, b_lo + (uint32_t)ks * b_ks, idesc, ks ? 1u : accumulate);
+}
+__device__ __forceinline__ void issue_ksteps(int ksteps, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_ks,
+                                             uint32_t b_ks, uint32_t idesc, uint32_t accumulate) {
+    switch (ksteps) {
+        case 1: issue_ksteps_n<1>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
+        case 2: issue_ksteps_n<2>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
+        case 3: issue_ksteps_n<3>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
+        default: issue_ksteps_n<4>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
+    }
+}
+
 // Shared-memory control block at the start of dynamic shared memory.
 struct Ctrl {
     uint64_t a_full[kMaxStages];
@@ -206,10 +224,12 @@ __device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
 }
 
 // Threads: warp 0 producer, warp 1 MMA, EPI epilogue warps (4, or 8 for wide filter tiles: two warps per
-// TMEM lane quarter, each taking half of the columns), then 1 filter-producer warp (FLAT_STREAM) or 4
-// loader warps (GATHER).
+// TMEM lane quarter, each taking half of the columns), then either 4 loader warps (GATHER) or 1 filter-producer
+// warp and 3 more MMA warps (FLAT_STREAM).  A single thread cannot issue MMAs as fast as the tensor pipe
+// retires them (measured: 75-110 cycles per issued MMA against 56-64 of execution at N = 96-128), so in
+// FLAT_STREAM, where one CTA owns the SM, each 128-position tile of a step has an issuing warp of its own.
 template <int MODE, int EPI>
-__global__ void __launch_bounds__(64 + 32 * EPI + (MODE == MODE_GATHER ? 128 : MODE == MODE_FLAT_STREAM ? 32 : 0))
+__global__ void __launch_bounds__(64 + 32 * EPI + (MODE == MODE_FLAT_RESIDENT ? 0 : 128))
 conv_tc_kernel(const TcParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
@@ -229,14 +249,17 @@ conv_tc_kernel(const TcParams p) {
     const uint32_t tfull0 = ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_full);
     const uint32_t tempty0 = ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_empty);
 
+    // MMA-issuing warps: warp 1, plus (streamed filters) the last three warps, one per tile of a step
+    const uint32_t n_issuers = MODE == MODE_FLAT_STREAM ? (uint32_t)p.tps : 1u;
+    const int issuer = warp == 1 ? 0 : (MODE == MODE_FLAT_STREAM && warp >= 3 + EPI) ? warp - (2 + EPI) : -1;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(a_full0 + 8 * s, MODE == MODE_GATHER ? 129 : 1);   // gather: 128 loaders + the filter producer
-            mbar_init(a_empty0 + 8 * s, 1);
+            mbar_init(a_empty0 + 8 * s, n_issuers);
             mbar_init(b_full0 + 8 * s, 1);
-            mbar_init(b_empty0 + 8 * s, 1);
+            mbar_init(b_empty0 + 8 * s, n_issuers);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, 1); mbar_init(tempty0 + 8 * s, 32 * EPI); }
+        for (int s = 0; s < 2; ++s) { mbar_init(tfull0 + 8 * s, n_issuers); mbar_init(tempty0 + 8 * s, 32 * EPI); }
         ctrl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -328,9 +351,9 @@ conv_tc_kernel(const TcParams p) {
             }
             if (!ok && lane == 0) raise(ctrl, p.status, 1);
         }
-    } else if (warp == 1) {
+    } else if (issuer >= 0) {
         // ------------------------------ MMA issuer --------------------------------
-        if (lane == 0) {
+        if (lane == 0 && issuer < (int)n_issuers) {
             // instruction descriptor: D = f32, A = B = bf16, both K-major, N = n_tile, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
             uint32_t a_stage = 0, a_phase = 0, b_stage = 0, b_phase = 0;
@@ -381,17 +404,10 @@ conv_tc_kernel(const TcParams p) {
                                     tc_fence_after();
                                     b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
                                 }
-                                // every 128-position tile of the step uses this filter block: its own accumulator,
-                                // its activation rows 128 further on
-                                for (int t = 0; t < p.tps; ++t) {
-                                    uint32_t a_t = a_lo + (uint32_t)(t * 128), b_t = b_lo;
-                                    const uint32_t d_t = d_tmem + (uint32_t)(t * p.n_tile);
-                                    for (int ks = 0; ks < ksteps; ++ks) {
-                                        umma_bf16_lo(d_t, a_t, b_t, idesc, accumulate | (uint32_t)(ks > 0));
-                                        a_t += a_ks;
-                                        b_t += b_ks;
-                                    }
-                                }
+                                // every 128-position tile of the step uses this filter block: its own accumulator
+                                // and issuing warp, its activation rows 128 further on
+                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_lo + (uint32_t)(issuer * 128), b_lo,
+                                             a_ks, b_ks, idesc, accumulate);
                                 accumulate = 1;
                                 if (MODE == MODE_FLAT_STREAM) {
                                     umma_commit(b_empty0 + 8 * b_stage);
@@ -745,7 +761,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             smem = fixed + plan->a_stages * a_stage;
         } else {
             plan->b_resident = 0;
-            plan->b_stages = 4;
+            plan->b_stages = 8;      // filter blocks are small next to the copy latency: keep many in flight
             const unsigned b_stage = (unsigned)(plan->cg * n_tile * 16);
             plan->a_stages = plan->tps > 1 ? 2 : 3;
             while (plan->a_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->a_stages;
@@ -795,7 +811,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     cudaFuncAttributes fa;
     cudaError_t oe = cudaFuncGetAttributes(&fa, fn);
     if (oe != cudaSuccess) { snprintf(err, err_len, "cudaFuncGetAttributes: %s", cudaGetErrorString(oe)); cudaGetLastError(); return 1; }
-    const int threads = 64 + 32 * epi + (mode == MODE_GATHER ? 128 : mode == MODE_FLAT_STREAM ? 32 : 0);
+    const int threads = 64 + 32 * epi + (mode == MODE_FLAT_RESIDENT ? 0 : 128);
     const int regs_per_warp = round_up_i(fa.numRegs * 32, 256);
     int occ = 65536 / (regs_per_warp * (threads / 32));
     if (occ > 2048 / threads) occ = 2048 / threads;
@@ -838,7 +854,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
     const int mode = !plan.flat ? MODE_GATHER : plan.b_resident ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
-    cfg.blockDim = dim3((unsigned)(64 + 32 * plan.epi_warps + (mode == MODE_GATHER ? 128 : mode == MODE_FLAT_STREAM ? 32 : 0)));
+    cfg.blockDim = dim3((unsigned)(64 + 32 * plan.epi_warps + (mode == MODE_FLAT_RESIDENT ? 0 : 128)));
     cfg.dynamicSmemBytes = plan.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
