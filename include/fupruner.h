@@ -184,6 +184,10 @@ typedef struct {
     double flops_per_image;  /* 2*MACs, unpadded                                                    */
     double bytes_per_image;  /* algorithmic activation bytes (in + residual + out)                   */
     double bytes_fixed;      /* weight + bias bytes                                                  */
+    int32_t chain;           /* >= 0: the operator is a layer of fused run number `chain` (one kernel for the
+                                whole run, activations in shared memory; FP_Q_OP_TIMES reports the run's time
+                                at its first layer and 0 at the others); -1: launched on its own          */
+    int32_t reserved;
 } fp_op_info;
 
 fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_out, size_t bytes);

@@ -48,7 +48,7 @@ class fp_op_info(ctypes.Structure):
                 ("kind", "conv_index", "K", "C", "R", "S", "stride", "pad", "K_pad", "C_pad", "H", "W", "P", "Q",
                  "res_mode", "relu")] + \
                [("flops_per_image", ctypes.c_double), ("bytes_per_image", ctypes.c_double),
-                ("bytes_fixed", ctypes.c_double)]
+                ("bytes_fixed", ctypes.c_double), ("chain", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class FpError(RuntimeError):

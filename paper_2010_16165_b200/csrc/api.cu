@@ -78,11 +78,22 @@ struct FConv {
     int K_kept = 0, K_rows = 0, K_pad = 0, C_kept = 0, C_pad = 0;
     void* d_wp = nullptr;      // packed filters in the compute type, K_pad x R x S x C_pad
     float* d_bp = nullptr;
+    int32_t* d_row = nullptr;  // packed filter row -> fused filter (-1 = zero row)
+    int32_t* d_chan = nullptr; // packed input channel -> fused input channel (-1 = zero channel)
     fp::ConvArgs args;
     fp::ConvPlanTC tc;
 };
 
 struct Pool { int src, out, R, stride, pad; };
+
+// Consecutive stride-1 3x3 convolutions that one kernel runs with the activations in shared memory.
+struct Chain {
+    int first_op = -1, last_op = -1;
+    std::vector<int> convs;    // indices into the handle's convs, in execution order
+    fp::ChainArgs args;
+    fp::ChainPlan plan;
+    uint8_t* d_blob = nullptr;
+};
 
 struct Op { int kind; int idx; };   // kind: 0 conv, 1 pool, 2 head, 3 input conversion
 
@@ -109,6 +120,8 @@ struct fp_handle_s {
     std::vector<Pool> pools;
     std::vector<Tensor> tensors;           // tensor 0 = network input (after layout conversion)
     std::vector<Op> ops;
+    std::vector<Chain> chains;             // re-derived by fp_prune
+    std::vector<int> op_chain;             // operator -> chain number, -1 = launched on its own
     // head
     int head_src = -1, n_classes = 0, fc_C = 0;
     const float* d_fcw = nullptr;          // classes x fc_C (copy of the description's FC weights)
@@ -473,6 +486,91 @@ fp_status upload_i32(fp_handle h, const std::vector<int32_t>& v, int32_t** out) 
     return FP_OK;
 }
 
+bool chain_candidate(fp_handle h, const FConv& f) {
+    if (h->compute != FP_COMPUTE_BF16_TC || h->keep_outputs) return false;
+    if (f.R != 3 || f.S != 3 || f.stride != 1 || f.pad != 1) return false;
+    if (h->stem_packed && f.src == 0) return false;
+    const Tensor& s = h->tensors[f.src];
+    return fp::chain_layer_supported(s.H, s.W, f.K_pad, f.C_pad);
+}
+
+// Finds runs of consecutive operators that are stride-1 3x3 convolutions where each reads the previous
+// one's output, a shortcut operand (other than the first layer's) is the tensor two layers back, and no
+// tensor inside the run is read from outside it; packs their filters for the fused kernel.
+fp_status find_chains(fp_handle h, const std::vector<std::vector<Use>>& uses) {
+    h->chains.clear();
+    h->op_chain.assign(h->ops.size(), -1);
+    const int n_ops = (int)h->ops.size();
+    int i = 0;
+    while (i < n_ops) {
+        if (h->ops[i].kind != 0 || !chain_candidate(h, h->convs[h->ops[i].idx])) { ++i; continue; }
+        // longest candidate run starting at operator i
+        int len = 1;
+        while (i + len < n_ops && len < fp::kChainMaxLayers && h->ops[i + len].kind == 0) {
+            const FConv& f = h->convs[h->ops[i + len].idx];
+            const FConv& prev = h->convs[h->ops[i + len - 1].idx];
+            if (!chain_candidate(h, f) || f.src != prev.out) break;
+            if (f.res_mode != 0 && !(f.res_mode == 1 && f.res_tid == prev.src)) break;
+            ++len;
+        }
+        // shorten until every tensor inside the run is read only inside it, and the run fits the kernel
+        fp::ChainArgs a;
+        fp::ChainPlan plan;
+        for (; len >= 2; --len) {
+            bool ok = true;
+            for (int j = 0; j + 1 < len && ok; ++j) {
+                const int tid = h->convs[h->ops[i + j].idx].out;
+                for (const Use& u : uses[tid]) {
+                    const bool main_next = u.how == 0 && u.op == i + j + 1;
+                    const bool res_after = u.how == 1 && u.op == i + j + 2 && j + 2 < len;
+                    if (!main_next && !res_after) { ok = false; break; }
+                }
+            }
+            if (!ok) continue;
+            memset(&a, 0, sizeof(a));
+            const FConv& f0 = h->convs[h->ops[i].idx];
+            const Tensor& s0 = h->tensors[f0.src];
+            a.N = h->max_batch; a.H = s0.H; a.W = s0.W; a.n_layers = len;
+            a.res_mode = f0.res_mode;
+            if (f0.res_mode) {
+                const Tensor& r = h->tensors[f0.res_tid];
+                a.res_H = r.H; a.res_W = r.W; a.res_C_pad = r.C_pad; a.res_C = r.C;
+                a.res_pad_lo = f0.res_pad_lo; a.res_stride = f0.res_stride;
+            }
+            int off = 0;
+            for (int j = 0; j < len; ++j) {
+                const FConv& f = h->convs[h->ops[i + j].idx];
+                fp::ChainLayer& ly = a.layers[j];
+                ly.cchunks = f.C_pad / 8; ly.K_pad = f.K_pad; ly.relu = f.relu;
+                ly.res = j == 0 ? (f.res_mode != 0) : (f.res_mode == 1);
+                ly.blob_off = off;
+                ly.blob_bytes = fp::chain_layer_blob_bytes(ly.cchunks, ly.K_pad);
+                off += (ly.blob_bytes + 127) / 128 * 128;
+            }
+            char msg[256];
+            if (fp::plan_chain_tc(a, &plan, msg, sizeof(msg)) != 0) continue;
+            Chain ch;
+            ch.first_op = i; ch.last_op = i + len - 1; ch.args = a; ch.plan = plan;
+            for (int j = 0; j < len; ++j) ch.convs.push_back(h->ops[i + j].idx);
+            TRY(dev_alloc(h->pack_buffers, (void**)&ch.d_blob, (size_t)off));
+            for (int j = 0; j < len; ++j) {
+                const FConv& f = h->convs[ch.convs[j]];
+                const fp::ChainLayer& ly = a.layers[j];
+                fp::launch_repack_chain(f.d_w32, f.C, f.d_row, f.K_pad, f.d_chan, f.C_pad,
+                                        (__nv_bfloat16*)(ch.d_blob + ly.blob_off), 0);
+                fp::launch_pack_bias(f.d_b32, f.d_row, f.K_pad,
+                                     (float*)(ch.d_blob + ly.blob_off + (size_t)9 * f.C_pad * f.K_pad * 2), 0);
+            }
+            CK(cudaGetLastError());
+            for (int j = 0; j < len; ++j) h->op_chain[i + j] = (int)h->chains.size();
+            h->chains.push_back(ch);
+            break;
+        }
+        i += len >= 2 ? len : 1;
+    }
+    return FP_OK;
+}
+
 fp_status replan(fp_handle h) {
     drop_graphs(h);
     CK(cudaDeviceSynchronize());
@@ -525,6 +623,7 @@ fp_status replan(fp_handle h) {
             int32_t *d_row, *d_chan;
             TRY(upload_i32(h, row_src, &d_row));
             TRY(upload_i32(h, chan_src, &d_chan));
+            f.d_row = d_row; f.d_chan = d_chan;
             const bool packed_stem = h->stem_packed && f.src == 0;
             const size_t cnt = packed_stem ? (size_t)f.K_pad * 3 * 80 : (size_t)f.K_pad * f.R * f.S * f.C_pad;
             TRY(dev_alloc(h->pack_buffers, &f.d_wp, cnt * h->act_elem()));
@@ -552,6 +651,7 @@ fp_status replan(fp_handle h) {
         }
     }
     CK(cudaGetLastError());
+    TRY(find_chains(h, uses));
 
     // --- activation memory: buffers are reused once their last reader has run ---
     {
@@ -564,7 +664,15 @@ fp_status replan(fp_handle h) {
         for (int i = 0; i < (int)h->ops.size(); ++i) {
             const Op& op = h->ops[i];
             int tid = -1;
-            if (op.kind == 0) tid = h->convs[op.idx].out;
+            if (op.kind == 0 && h->op_chain[i] >= 0) {
+                // a fused run is one kernel: only its last tensor exists in memory, and it must not share
+                // a buffer with the run's inputs, which other CTAs still read while the first ones finish
+                const Chain& ch = h->chains[h->op_chain[i]];
+                if (i != ch.last_op) h->tensors[h->convs[op.idx].out].d = nullptr;
+                if (i != ch.first_op) continue;
+                tid = h->convs[ch.convs.back()].out;
+            }
+            else if (op.kind == 0) tid = h->convs[op.idx].out;
             else if (op.kind == 1) tid = h->pools[op.idx].out;
             else if (op.kind == 3) tid = 0;
             if (tid < 0) continue;
@@ -615,6 +723,11 @@ fp_status replan(fp_handle h) {
                 return fail(FP_ERR_UNSUPPORTED, "convolution %d: %s", f.conv_index, msg);
         }
     }
+    for (Chain& ch : h->chains) {
+        const FConv& f0 = h->convs[ch.convs.front()];
+        const FConv& fl = h->convs[ch.convs.back()];
+        ch.args.x = f0.args.x; ch.args.res = f0.args.res; ch.args.y = fl.args.y; ch.args.w = ch.d_blob;
+    }
     CK(cudaDeviceSynchronize());
     return FP_OK;
 }
@@ -623,8 +736,17 @@ fp_status replan(fp_handle h) {
 // execution
 // ---------------------------------------------------------------------------------------
 
-void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
+void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
+    const Op& op = h->ops[op_index];
     const int bf16 = h->act_is_bf16();
+    if (op.kind == 0 && h->op_chain[op_index] >= 0) {
+        const Chain& ch = h->chains[h->op_chain[op_index]];
+        if (op_index != ch.first_op) return;       // the run's first operator launches all of it
+        fp::ChainArgs a = ch.args;
+        a.N = batch;
+        fp::launch_chain_tc(ch.plan, a, h->d_status, st);
+        return;
+    }
     if (op.kind == 3) {
         const Tensor& t = h->tensors[0];
         if (h->stem_packed) fp::launch_input_to_stem_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, batch, t.C, t.H, t.W, st);
@@ -647,7 +769,7 @@ void launch_op(fp_handle h, const Op& op, const void* d_input, int batch, float*
 }
 
 void launch_all(fp_handle h, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
-    for (const Op& op : h->ops) launch_op(h, op, d_input, batch, d_logits, st);
+    for (int i = 0; i < (int)h->ops.size(); ++i) launch_op(h, i, d_input, batch, d_logits, st);
 }
 
 fp_status all_ones_masks(fp_handle h) {
@@ -859,6 +981,7 @@ static void fill_op_info(fp_handle h, int i, fp_op_info* o) {
     const Op& op = h->ops[i];
     const double e = (double)h->act_elem();
     o->kind = op.kind; o->conv_index = -1;
+    o->chain = h->op_chain[i];
     if (op.kind == 0) {
         const FConv& f = h->convs[op.idx];
         const Tensor& s = h->tensors[f.src];
@@ -909,7 +1032,13 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
         case FP_Q_N_CONVS: TRY(need(4)); *(int32_t*)h_out = h->n_desc_convs; return FP_OK;
         case FP_Q_N_CLASSES: TRY(need(4)); *(int32_t*)h_out = h->n_classes; return FP_OK;
         case FP_Q_N_OPS: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size(); return FP_OK;
-        case FP_Q_N_LAUNCHES: TRY(need(4)); *(int32_t*)h_out = (int32_t)h->ops.size() + 1; return FP_OK;   // the head is two kernels
+        case FP_Q_N_LAUNCHES: {
+            TRY(need(4));
+            int n = (int)h->ops.size() + 1;                                  // the head is two kernels
+            for (const Chain& ch : h->chains) n -= (int)ch.convs.size() - 1; // a fused run is one
+            *(int32_t*)h_out = n;
+            return FP_OK;
+        }
         case FP_Q_CONV_K_FUSED: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K : 0; return FP_OK;
         case FP_Q_CONV_K_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K_kept : 0; return FP_OK;
         case FP_Q_CONV_C_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->C_kept : 0; return FP_OK;
@@ -946,6 +1075,8 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             const Op& op = h->ops[index];
             const int tid = op.kind == 0 ? h->convs[op.idx].out : op.kind == 1 ? h->pools[op.idx].out : 0;
             const Tensor& t = h->tensors[tid];
+            if (!t.d) return fail(FP_ERR_UNSUPPORTED, "fp_query: operator %d runs inside a fused run of layers and its output never "
+                                  "reaches memory (set keep_outputs to run every layer on its own)", index);
             const size_t cnt = (size_t)h->last_batch * t.C * t.H * t.W;
             TRY(need(cnt * sizeof(float)));
             float* d_tmp;
@@ -977,7 +1108,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             for (int r = 0; r < reps + 1; ++r) {
                 CK(cudaEventRecord(ev[0], st));
                 for (int i = 0; i < n; ++i) {
-                    launch_op(h, h->ops[i], h->last_input, h->last_batch, h->d_logits_stage, st);
+                    launch_op(h, i, h->last_input, h->last_batch, h->d_logits_stage, st);
                     CK(cudaEventRecord(ev[i + 1], st));
                 }
                 CK(cudaStreamSynchronize(st));

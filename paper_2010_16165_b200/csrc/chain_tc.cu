@@ -1,0 +1,535 @@
+// A run of consecutive stride-1 3x3 convolutions (the convolutions of a stage of basic residual
+// blocks) as ONE kernel: every CTA carries a group of G whole images through all layers of the run,
+// with the activations in shared memory from the first layer's input to the last layer's output.
+// Only the run's input, the first layer's shortcut operand and the run's output touch global memory;
+// the filters of each layer are streamed into a double buffer while the previous layer computes.
+//
+//   Activation layout in shared memory: planar-8 (one 16-byte vector = 8 channels of one position),
+//   row pitch W with NO column border, one zero row above every image and one below the last:
+//       position f = img*(H+1)*W + hrow*W + w,   hrow = 0 is the zero row, hrow = h + 1 a pixel row.
+//   W divides 32, so a warp of the epilogue always covers whole image rows.
+//
+//   GEMM view of one layer: M = positions (tiles of 128), K = input channels, and the three
+//   HORIZONTAL filter taps are stacked along N:   D[p, (s,k)] = sum_{r,c} x[p + (r-1)*W, c] * W'[k,c,r,s].
+//   The vertical taps are three accumulating MMAs whose A operand is the same shared-memory plane
+//   read from a start address shifted by (r-1)*W rows (the zero rows are the vertical padding).  The
+//   horizontal taps are recombined in the epilogue with two warp shuffles,
+//       y[p, k] = D[p-1, (0,k)] + D[p, (1,k)] + D[p+1, (2,k)],
+//   where the neighbour terms are dropped in the first / last column of an image row (that is the
+//   horizontal padding).  For the narrow layers this path is built for (16..64 channels) one MMA of
+//   N = 3*K_pad replaces three of N = K_pad, and the tensor pipe's time per MMA hardly depends on N there.
+//
+//   Warp roles: warp 0 streams filter blobs (bulk copies), warp 1 owns tensor memory and lane 0
+//   issues the MMAs, warps 2-17 are the epilogue: four groups of four warps (one warp per quarter of
+//   the 128 accumulator rows).  A group takes every (4/split)-th tile and every split-th channel chunk
+//   of it (split = 1, 2 or 4: runs with few tiles per layer spread each tile over more warps).  The
+//   same warps load the run's input and store its output.
+//   Pipelining: the accumulators form a ring of up to 8 stages in tensor memory, so the MMAs of later
+//   tiles run while earlier tiles are in their epilogue (an MMA group completes about a thousand cycles
+//   after it is issued).  Layers overlap too: tile t of a layer needs only tiles t-1, t, t+1 of the
+//   previous layer (the vertical halo is W <= 32 positions), tracked with one mbarrier per tile, so
+//   the next layer's first tiles are issued while the current layer's last tiles are in flight.
+//   Every wait is bounded and raises a status word.
+#include "fp_internal.h"
+#include "tc_common.cuh"
+
+#include <cstdio>
+#include <cstring>
+
+namespace fp {
+
+namespace {
+
+using namespace tc;
+
+struct ChainParams {
+    ChainArgs a;
+    int G, tiles, plane_rows, buf_bytes, wbuf_bytes, tmem_cols, acc_cols, n_groups, stages, split, issuers, ring;
+    int img_pos, w_shift, P2, Wp;
+    FastDiv div_img, div_ring, div_iss;
+    long long plane_in, plane_out, plane_res;
+    int rP2, rWp;
+    int* status;
+};
+
+constexpr int kMaxStages = 8;
+constexpr int kMaxTiles = 64;
+
+struct ChainCtrl {
+    uint64_t w_full[2], w_empty[2], tmem_full[kMaxStages], tmem_empty[kMaxStages], tile_done[2][kMaxTiles], group_sync;
+    uint32_t tmem_base;
+    int abort_flag;
+    int pad_[4];
+};
+static_assert(sizeof(ChainCtrl) % 16 == 0, "buffers behind the control block must stay 16-byte aligned");
+
+constexpr int kEpiThreads = 512;
+constexpr int kIssuers = 4;                        // MMA-issuing warps: warp 1 and the last three
+constexpr int kThreads = 64 + kEpiThreads + 32 * (kIssuers - 1);
+
+__device__ __forceinline__ void raise_chain(ChainCtrl* ctrl, int* status, int code) {
+    atomicExch(&ctrl->abort_flag, 1);
+    atomicExch(status, code);
+}
+
+// 8 channels of one position of the first layer's shortcut operand (read from global memory)
+__device__ __forceinline__ uint4 load_residual_vec(const ChainParams& p, int chunk, int n, int hrow, int wcol) {
+    const uint4* __restrict__ res = reinterpret_cast<const uint4*>(p.a.res);
+    if (p.a.res_mode == 1) {
+        if (chunk * 8 >= p.a.res_C_pad) return make_uint4(0, 0, 0, 0);
+        return __ldg(res + (long long)chunk * p.plane_res + (long long)n * p.rP2 + (long long)hrow * p.rWp + (wcol + 1));
+    }
+    // subsampled input, channel k of the output takes channel k - pad_lo of the operand
+    const long long pos = (long long)n * p.rP2 + (long long)((hrow - 1) * p.a.res_stride + 1) * p.rWp + (wcol * p.a.res_stride + 1);
+    const int cs = chunk * 8 - p.a.res_pad_lo;
+    if (cs >= 0 && cs + 8 <= p.a.res_C_pad && (cs & 7) == 0) return __ldg(res + (long long)(cs >> 3) * p.plane_res + pos);
+    uint4 out = make_uint4(0, 0, 0, 0);
+    if (cs + 8 > 0 && cs < p.a.res_C) {
+        const __nv_bfloat16* __restrict__ rs = reinterpret_cast<const __nv_bfloat16*>(p.a.res);
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(&out);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = cs + i;
+            if (c >= 0 && c < p.a.res_C) o[i] = rs[((long long)(c >> 3) * p.plane_res + pos) * 8 + (c & 7)];
+        }
+    }
+    return out;
+}
+
+// The MMAs of one tile: three vertical taps x KSTEPS K=16 steps, unrolled with every operand address a
+// register + constant, because the issuing thread's own instruction latency is what limits narrow layers.
+template <int KSTEPS>
+__device__ __forceinline__ void issue_tile(uint32_t d_tmem, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t b0, uint32_t b1,
+                                           uint32_t b2, uint32_t a_ks, uint32_t b_ks, uint32_t idesc) {
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a0 + ks * a_ks, b0 + ks * b_ks, idesc, ks ? 1u : 0u);
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a1 + ks * a_ks, b1 + ks * b_ks, idesc, 1u);
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a2 + ks * a_ks, b2 + ks * b_ks, idesc, 1u);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainParams p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    ChainCtrl* ctrl = reinterpret_cast<ChainCtrl*>(smem_raw);
+    const uint32_t ctrl_addr = smem_u32(smem_raw);
+    const uint32_t wbuf0 = (ctrl_addr + (uint32_t)sizeof(ChainCtrl) + 127u) & ~127u;
+    const uint32_t act0 = wbuf0 + 2u * (uint32_t)p.wbuf_bytes;
+    uint8_t* const wbuf_ptr = smem_raw + (wbuf0 - ctrl_addr);
+    uint8_t* const act_ptr = smem_raw + (act0 - ctrl_addr);
+    volatile int* abort_flag = &ctrl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t w_full0 = ctrl_addr + (uint32_t)offsetof(ChainCtrl, w_full);
+    const uint32_t w_empty0 = ctrl_addr + (uint32_t)offsetof(ChainCtrl, w_empty);
+    const uint32_t tfull0 = ctrl_addr + (uint32_t)offsetof(ChainCtrl, tmem_full);
+    const uint32_t tempty0 = ctrl_addr + (uint32_t)offsetof(ChainCtrl, tmem_empty);
+    const uint32_t tdone0 = ctrl_addr + (uint32_t)offsetof(ChainCtrl, tile_done);
+    const uint32_t group_sync = ctrl_addr + (uint32_t)offsetof(ChainCtrl, group_sync);
+    const int split = p.split, units = 4 / p.split;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(w_full0 + 8 * s, 1);
+            mbar_init(w_empty0 + 8 * s, p.issuers + kEpiThreads / 32);    // the MMA issuers + every epilogue warp (bias reads)
+        }
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(tfull0 + 8 * s, 1);
+            mbar_init(tempty0 + 8 * s, 128 * split);               // every thread that reads the stage
+        }
+        for (int t = 0; t < p.tiles; ++t) {
+            mbar_init(tdone0 + 8 * t, 128 * split);
+            mbar_init(tdone0 + 8 * (kMaxTiles + t), 128 * split);
+        }
+        mbar_init(group_sync, kEpiThreads);
+        ctrl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(ctrl_addr + (uint32_t)offsetof(ChainCtrl, tmem_base)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
+
+    // Programmatic dependent launch: the next kernel may begin its prologue now.  The filter producer
+    // reads only filters (never written by a forward) and starts at once; every other role waits until
+    // the previous kernel has completed before it touches activations.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    const int L = p.a.n_layers;
+    const uint32_t plane_bytes = (uint32_t)p.plane_rows * 16u;
+
+    if (warp == 0) {
+        // ------------------------------ filter producer ------------------------------
+        bool ok = true;
+        uint32_t it = 0;
+        for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
+            for (int l = 0; l < L; ++l, ++it) {
+                const uint32_t wb = it & 1, wph = (it >> 1) & 1;
+                bool w = true;
+                if (lane == 0) w = mbar_wait(w_empty0 + 8 * wb, wph ^ 1, abort_flag);
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (!w) { ok = false; break; }
+                const int bytes = p.a.layers[l].blob_bytes;
+                const uint32_t fb = w_full0 + 8 * wb;
+                if (lane == 0) mbar_expect_tx(fb, (uint32_t)bytes);
+                __syncwarp();
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(p.a.w) + p.a.layers[l].blob_off;
+                for (int off = lane * 4096; off < bytes; off += 32 * 4096) {
+                    const int n = bytes - off < 4096 ? bytes - off : 4096;
+                    bulk_copy(wbuf0 + wb * p.wbuf_bytes + off, src + off, (uint32_t)n, fb);
+                }
+            }
+        }
+        if (!ok && lane == 0) raise_chain(ctrl, p.status, 11);
+    } else if (warp == 1 || warp >= 2 + kEpiThreads / 32) {
+        // ------------------------------ MMA issuers -----------------------------------
+        // A single thread issues the handful of MMAs of a narrow tile more slowly than the tensor pipe
+        // executes them (a bounded mbarrier test alone costs about a hundred cycles), so up to four warps take
+        // the tiles round robin; each tile's accumulation chain stays within one thread.  Every issuer owns
+        // the accumulator stages iss, iss + issuers, ...: all uses of a stage are then in one thread's program
+        // order, which the parity waits on the stage's barriers rely on.
+        const int iss = warp == 1 ? 0 : warp - (1 + kEpiThreads / 32);
+        if (lane == 0 && iss < p.issuers) {
+            const uint32_t my_tiles = iss < p.tiles ? (uint32_t)((p.tiles - iss + p.issuers - 1) / p.issuers) : 0u;
+            bool ok = true;
+            uint32_t it = 0;
+            for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
+                for (int l = 0; l < L && ok; ++l, ++it) {
+                    const ChainLayer& ly = p.a.layers[l];
+                    const uint32_t wb = it & 1, wph = (it >> 1) & 1;
+                    // Tile t's input is complete when its barrier has completed `it` + 1 times (once per group load
+                    // and per layer).  Completions alternate between two barriers per tile, so that a parity test
+                    // cannot mistake "two completions ahead" for "not yet": a tile is never two layers ahead of a
+                    // neighbour that still waits for it.
+                    const uint32_t td = tdone0 + 8u * (uint32_t)kMaxTiles * (it & 1), tdp = (it >> 1) & 1;
+                    if (!mbar_wait(w_full0 + 8 * wb, wph, abort_flag)) { ok = false; break; }
+                    const uint32_t N = 3u * (uint32_t)ly.K_pad;
+                    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((128u >> 4) << 24);
+                    const int ksteps = ly.cchunks >> 1;
+                    const uint32_t src = act0 + (uint32_t)(l & 1) * (uint32_t)p.buf_bytes;
+                    // low descriptor words: start address / 16 | (bytes between the two K halves / 16) << 16
+                    const uint32_t a_r0 = (src >> 4) | ((uint32_t)p.plane_rows << 16);     // tap row r = 0 starts W rows before the tile
+                    const uint32_t a_r1 = a_r0 + (uint32_t)p.a.W, a_r2 = a_r1 + (uint32_t)p.a.W;
+                    const uint32_t b_r0 = ((wbuf0 + wb * (uint32_t)p.wbuf_bytes) >> 4) | (N << 16);
+                    const uint32_t b_r1 = b_r0 + (uint32_t)ly.cchunks * N, b_r2 = b_r1 + (uint32_t)ly.cchunks * N;
+                    const uint32_t a_ks = 2u * (uint32_t)p.plane_rows, b_ks = 2u * N;
+                    uint32_t m = it * my_tiles;          // this issuer's tiles so far
+                    for (int t = iss; t < p.tiles; t += p.issuers, ++m) {
+                        const uint32_t round = fdiv(m, p.div_ring);
+                        const uint32_t stage = (uint32_t)iss + (uint32_t)p.issuers * (m - round * (uint32_t)p.ring), sph = round & 1;
+                        if (!mbar_wait(tempty0 + 8 * stage, sph ^ 1, abort_flag)) { ok = false; break; }
+                        // the tile reads positions t*128 - W .. t*128 + 127 + W of the previous layer's output
+                        if (t > 0 && !mbar_wait(td + 8 * (t - 1), tdp, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(td + 8 * t, tdp, abort_flag)) { ok = false; break; }
+                        if (t + 1 < p.tiles && !mbar_wait(td + 8 * (t + 1), tdp, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t d_tmem = tmem_base + stage * (uint32_t)p.acc_cols;
+                        const uint32_t to = (uint32_t)(t * 128);
+                        switch (ksteps) {
+                            case 1: issue_tile<1>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 2: issue_tile<2>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 3: issue_tile<3>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 4: issue_tile<4>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            default: {
+                                uint32_t accumulate = 0;
+                                for (int r = 0; r < 3; ++r) {
+                                    uint32_t a_lo = (r == 0 ? a_r0 : r == 1 ? a_r1 : a_r2) + to, b_lo = r == 0 ? b_r0 : r == 1 ? b_r1 : b_r2;
+                                    for (int ks = 0; ks < ksteps; ++ks) {
+                                        umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
+                                        accumulate = 1;
+                                        a_lo += a_ks; b_lo += b_ks;
+                                    }
+                                }
+                            }
+                        }
+                        umma_commit(tfull0 + 8 * stage);
+                    }
+                    if (ok) umma_commit(w_empty0 + 8 * wb);     // the filter buffer is free once this warp's MMAs have read it
+                }
+            }
+            if (!ok) raise_chain(ctrl, p.status, 12);
+        }
+    } else {
+        // ------------------------------ load / epilogue / store ------------------------
+        const int etid = threadIdx.x - 64;
+        const int grp = (warp - 2) >> 2;
+        const int unit = grp / split;                 // takes tiles unit, unit + units, ...
+        const int part = grp - unit * split;          // takes channel chunks part, part + split, ...
+        const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+        const int W = p.a.W, H = p.a.H;
+        const uint4* __restrict__ xv = reinterpret_cast<const uint4*>(p.a.x);
+        uint4* __restrict__ yv = reinterpret_cast<uint4*>(p.a.y);
+        bool ok = true;
+        uint32_t it = 0, gs_it = 0;
+        for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
+            if (gs_it) {
+                // every MMA and every epilogue of the previous group has finished before its buffers are overwritten
+                mbar_arrive(group_sync);
+                if (!mbar_wait(group_sync, (gs_it - 1) & 1, abort_flag)) { ok = false; break; }
+            }
+            ++gs_it;
+            // ---- load the group's images (and the first layer's shortcut operand); each thread loads the
+            //      positions and channel chunks it will later own in the epilogues ----
+            {
+                const int in_chunks = p.a.layers[0].cchunks;
+                const int out_chunks = p.a.layers[0].K_pad >> 3;
+                uint8_t* b0 = act_ptr + (size_t)W * 16;
+                uint8_t* b1 = b0 + p.buf_bytes;
+                for (int t = unit; t < p.tiles; t += units) {
+                    const int f = t * 128 + quarter * 32 + lane;
+                    const int img = (int)fdiv((uint32_t)f, p.div_img);
+                    const int rem = f - img * p.img_pos;
+                    const int hrow = rem >> p.w_shift, wcol = rem & (W - 1);
+                    const int n = g * p.G + img;
+                    const bool pixel = hrow >= 1 && img < p.G && n < p.a.N;
+                    const long long gpos = (long long)n * p.P2 + (long long)hrow * p.Wp + (wcol + 1);
+                    for (int c = part; c < in_chunks; c += split) {
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (pixel) v = __ldg(xv + (long long)c * p.plane_in + gpos);
+                        *reinterpret_cast<uint4*>(b0 + (size_t)c * plane_bytes + (size_t)f * 16) = v;
+                    }
+                    if (p.a.res_mode) {
+                        for (int c = part; c < out_chunks; c += split) {
+                            uint4 v = make_uint4(0, 0, 0, 0);
+                            if (pixel) v = load_residual_vec(p, c, n, hrow, wcol);
+                            *reinterpret_cast<uint4*>(b1 + (size_t)c * plane_bytes + (size_t)f * 16) = v;
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic stores -> MMA operand reads
+                    mbar_arrive(tdone0 + 8 * ((it & 1) * kMaxTiles + t));
+                }
+            }
+            // ---- layers ----
+            for (int l = 0; l < L && ok; ++l, ++it) {
+                const ChainLayer& ly = p.a.layers[l];
+                const uint32_t wb = it & 1, wph = (it >> 1) & 1;
+                const bool last = l == L - 1;
+                if (!mbar_wait(w_full0 + 8 * wb, wph, abort_flag)) { ok = false; break; }     // the bias is in the blob
+                const int K_pad = ly.K_pad;
+                const float* bias = reinterpret_cast<const float*>(wbuf_ptr + (size_t)wb * p.wbuf_bytes +
+                                                                   (size_t)(3 * ly.cchunks * 3 * K_pad) * 16);
+                uint8_t* dst = act_ptr + (size_t)((l + 1) & 1) * p.buf_bytes + (size_t)W * 16;
+                for (int t = unit; t < p.tiles; t += units) {
+                    const int f = t * 128 + quarter * 32 + lane;
+                    const int img = (int)fdiv((uint32_t)f, p.div_img);
+                    const int rem = f - img * p.img_pos;
+                    const int hrow = rem >> p.w_shift, wcol = rem & (W - 1);
+                    const int n = g * p.G + img;
+                    const bool pixel = hrow >= 1 && img < p.G && n < p.a.N;
+                    const bool has_left = wcol > 0, has_right = wcol < W - 1;
+                    // the accumulator stage: tile t is the (t / issuers)-th tile of issuer t % issuers in this layer
+                    const uint32_t ti = fdiv((uint32_t)t, p.div_iss), is = (uint32_t)t - ti * (uint32_t)p.issuers;
+                    const uint32_t m = it * (uint32_t)((p.tiles - (int)is + p.issuers - 1) / p.issuers) + ti;
+                    const uint32_t round = fdiv(m, p.div_ring);
+                    const uint32_t stage = is + (uint32_t)p.issuers * (m - round * (uint32_t)p.ring), sph = round & 1;
+                    bool w = mbar_wait(tfull0 + 8 * stage, sph, abort_flag);
+                    w = __all_sync(0xffffffffu, w);
+                    if (!w) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + stage * (uint32_t)p.acc_cols;
+                    const long long gpos = (long long)n * p.P2 + (long long)hrow * p.Wp + (wcol + 1);
+                    for (int kc = part; kc < (K_pad >> 3); kc += split) {
+                        uint32_t vl[8], vc[8], vr[8];
+                        tmem_ld8(taddr + (uint32_t)(kc * 8), vl);
+                        tmem_ld8(taddr + (uint32_t)(K_pad + kc * 8), vc);
+                        tmem_ld8(taddr + (uint32_t)(2 * K_pad + kc * 8), vr);
+                        uint4* slot = reinterpret_cast<uint4*>(dst + (size_t)kc * plane_bytes + (size_t)f * 16);
+                        uint4 rv = make_uint4(0, 0, 0, 0);
+                        if (ly.res) rv = *slot;
+                        const float4 bA = *reinterpret_cast<const float4*>(bias + kc * 8);
+                        const float4 bB = *reinterpret_cast<const float4*>(bias + kc * 8 + 4);
+                        tmem_ld_wait();
+                        float o[8];
+                        const float bb[8] = {bA.x, bA.y, bA.z, bA.w, bB.x, bB.y, bB.z, bB.w};
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float lf = __shfl_up_sync(0xffffffffu, __uint_as_float(vl[i]), 1);
+                            const float rt = __shfl_down_sync(0xffffffffu, __uint_as_float(vr[i]), 1);
+                            o[i] = __uint_as_float(vc[i]) + (has_left ? lf : 0.0f) + (has_right ? rt : 0.0f) + bb[i];
+                        }
+                        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float2 q = __bfloat1622float2(h2[i]);
+                            o[2 * i] += q.x;
+                            o[2 * i + 1] += q.y;
+                        }
+                        if (ly.relu) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) o[i] = fmaxf(o[i], 0.0f);
+                        }
+                        uint4 ov = make_uint4(0, 0, 0, 0);
+                        if (pixel) {
+                            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) o2[i] = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                        }
+                        if (!last) *slot = ov;
+                        else if (pixel) yv[(long long)kc * p.plane_out + gpos] = ov;
+                    }
+                    tc_fence_before();
+                    mbar_arrive(tempty0 + 8 * stage);
+                    if (!last) {
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        mbar_arrive(tdone0 + 8 * (((it + 1) & 1) * kMaxTiles + t));
+                    }
+                }
+                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(w_empty0 + 8 * wb);       // this warp no longer reads the layer's bias
+            }
+            if (!ok) break;
+            // ---- zero border of the group's output images in global memory ----
+            {
+                const int out_chunks = p.a.layers[L - 1].K_pad >> 3;
+                const int border = 2 * p.Wp + 2 * H;
+                const int total = p.G * border * out_chunks;
+                for (int i = etid; i < total; i += kEpiThreads) {
+                    const int c = i / (p.G * border);
+                    const int r2 = i - c * (p.G * border);
+                    const int img = r2 / border, b = r2 - img * border;
+                    const int n = g * p.G + img;
+                    if (n >= p.a.N) continue;
+                    int row, col;
+                    if (b < p.Wp) { row = 0; col = b; }
+                    else if (b < 2 * p.Wp) { row = H + 1; col = b - p.Wp; }
+                    else { const int s2 = b - 2 * p.Wp; row = 1 + (s2 >> 1); col = (s2 & 1) ? W + 1 : 0; }
+                    yv[(long long)c * p.plane_out + (long long)n * p.P2 + (long long)row * p.Wp + col] = make_uint4(0, 0, 0, 0);
+                }
+            }
+        }
+        if (!ok && lane == 0) raise_chain(ctrl, p.status, 13);
+    }
+
+    // ---- teardown: everyone arrives here, also after a wait that ran out ----
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);     // let copies in flight land before shared memory is released
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+}
+
+constexpr unsigned kSmemMax = 232448u - 1024u;
+constexpr unsigned kSmemMin = 120u * 1024u;        // more than half an SM: one CTA per SM, so tensor memory is never contended
+
+int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+int chain_layer_blob_bytes(int cchunks, int K_pad) { return 3 * cchunks * 3 * K_pad * 16 + K_pad * 4; }
+
+bool chain_layer_supported(int H, int W, int K_pad, int C_pad) {
+    if (!(W == 8 || W == 16 || W == 32)) return false;
+    if (H < 1 || H > 64) return false;
+    if (K_pad % 16 || C_pad % 16 || K_pad > 80 || C_pad > 128) return false;
+    return true;
+}
+
+int plan_chain_tc(const ChainArgs& a, ChainPlan* plan, char* err, size_t err_len) {
+    memset(plan, 0, sizeof(*plan));
+    if (a.n_layers < 1 || a.n_layers > kChainMaxLayers) { snprintf(err, err_len, "bad layer count"); return 1; }
+    int max_chunks = 0, max_blob = 0, max_N = 0;
+    for (int l = 0; l < a.n_layers; ++l) {
+        const ChainLayer& ly = a.layers[l];
+        if (!chain_layer_supported(a.H, a.W, ly.K_pad, ly.cchunks * 8)) { snprintf(err, err_len, "layer %d not supported", l); return 1; }
+        max_chunks = ly.cchunks > max_chunks ? ly.cchunks : max_chunks;
+        max_chunks = (ly.K_pad >> 3) > max_chunks ? (ly.K_pad >> 3) : max_chunks;
+        max_blob = ly.blob_bytes > max_blob ? ly.blob_bytes : max_blob;
+        max_N = 3 * ly.K_pad > max_N ? 3 * ly.K_pad : max_N;
+    }
+    const int wbuf = round_up_i(max_blob, 128);
+    const int img_pos = (a.H + 1) * a.W;
+    int best_G = 0; double best_cost = 0;
+    for (int G = 1; G <= 64 && G <= a.N; ++G) {
+        const int tiles = (G * img_pos + a.W + 127) / 128;
+        const int rows = 2 * a.W + tiles * 128;
+        if (rows > 16383 || tiles > kMaxTiles) break;
+        const unsigned smem = (unsigned)sizeof(ChainCtrl) + 128u + 2u * wbuf + 2u * (unsigned)max_chunks * rows * 16u;
+        if (smem > kSmemMax) break;
+        const int groups = (a.N + G - 1) / G;
+        const int rounds = (groups + 147) / 148;
+        const double cost = rounds * (tiles + 1.5);
+        if (best_G == 0 || cost <= best_cost) { best_G = G; best_cost = cost; }
+    }
+    if (best_G == 0) { snprintf(err, err_len, "one image does not fit shared memory"); return 1; }
+    plan->G = best_G;
+    plan->tiles = (best_G * img_pos + a.W + 127) / 128;
+    plan->plane_rows = 2 * a.W + plan->tiles * 128;
+    plan->buf_bytes = max_chunks * plan->plane_rows * 16;
+    plan->wbuf_bytes = wbuf;
+    plan->acc_cols = max_N;
+    plan->tmem_cols = 512;                              // one CTA per SM: all of tensor memory is the accumulator ring
+    plan->stages = 512 / max_N < kMaxStages ? 512 / max_N : kMaxStages;
+    plan->split = plan->tiles <= 4 ? 4 : plan->tiles <= 8 ? 2 : 1;
+    // issuers: a power of two (1, 2, 4) not above the stage and tile counts; epilogue units (4 / split) must not
+    // outnumber the issuers, so that all tiles of one issuer - all uses of one accumulator stage - go to one unit
+    plan->issuers = kIssuers;
+    while (plan->issuers > 1 && (plan->issuers > plan->stages || plan->issuers > plan->tiles)) plan->issuers >>= 1;
+    if (4 / plan->split > plan->issuers) plan->split = 4 / plan->issuers;
+    unsigned smem = (unsigned)sizeof(ChainCtrl) + 128u + 2u * wbuf + 2u * (unsigned)plan->buf_bytes;
+    if (smem < kSmemMin) smem = kSmemMin;
+    plan->smem_bytes = smem;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
+            snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
+            cudaGetLastError();
+            return 1;
+        }
+        attr_set = true;
+    }
+    plan->valid = 1;
+    return 0;
+}
+
+void launch_chain_tc(const ChainPlan& plan, const ChainArgs& a, int* d_status, cudaStream_t st) {
+    ChainParams p;
+    memset(&p, 0, sizeof(p));
+    p.a = a;
+    // the group size was planned for the largest batch; a smaller batch just has fewer groups
+    p.G = plan.G; p.tiles = plan.tiles; p.plane_rows = plan.plane_rows; p.buf_bytes = plan.buf_bytes;
+    p.wbuf_bytes = plan.wbuf_bytes; p.tmem_cols = plan.tmem_cols; p.acc_cols = plan.acc_cols;
+    p.stages = plan.stages; p.split = plan.split; p.issuers = plan.issuers;
+    p.ring = plan.stages / plan.issuers;
+    p.n_groups = (a.N + plan.G - 1) / plan.G;
+    p.img_pos = (a.H + 1) * a.W;
+    p.w_shift = a.W == 8 ? 3 : a.W == 16 ? 4 : 5;
+    p.Wp = a.W + 2; p.P2 = (a.H + 2) * (a.W + 2);
+    p.div_img = make_fastdiv((uint32_t)p.img_pos);
+    p.div_ring = make_fastdiv((uint32_t)p.ring);
+    p.div_iss = make_fastdiv((uint32_t)p.issuers);
+    p.plane_in = (long long)a.N * p.P2;
+    p.plane_out = p.plane_in;
+    p.rWp = a.res_W + 2; p.rP2 = (a.res_H + 2) * (a.res_W + 2);
+    p.plane_res = (long long)a.N * p.rP2;
+    p.status = d_status;
+    int grid = p.n_groups < 148 ? p.n_groups : 148;
+    if (grid < 1) grid = 1;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)kThreads);
+    cfg.dynamicSmemBytes = plan.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    void* args[1] = {(void*)&p};
+    cudaLaunchKernelExC(&cfg, (const void*)chain_tc_kernel, args);
+}
+
+}  // namespace fp

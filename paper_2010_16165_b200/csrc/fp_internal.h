@@ -61,6 +61,10 @@ void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int
 // 7x7 first convolution as a 3x1 convolution over the packed network input (80 channels)
 void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st);
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st);
+// 3x3 filters of one layer of a fused run: blob[r][cp/8][s*K_pad + kr][cp%8], the three horizontal taps
+// stacked along the filter (N) axis of the MMA (see chain_tc.cu)
+void launch_repack_chain(const float* w, int C, const int32_t* row_src, int K_pad, const int32_t* chan_src, int C_pad,
+                         __nv_bfloat16* out, cudaStream_t st);
 
 // Memory-bound operators ------------------------------------------------------------------
 void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
@@ -100,5 +104,41 @@ struct ConvPlanTC {
 // Returns 0 on success, otherwise writes a message.
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len);
 void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st);
+
+// A run of stride-1 3x3 convolutions executed by one kernel with the activations in shared memory.
+constexpr int kChainMaxLayers = 40;
+struct ChainLayer {
+    int cchunks;          // input channels / 8
+    int K_pad;            // output channels, multiple of 16, <= 80
+    int relu;
+    int res;              // 1: add the tensor two layers back (the one this layer overwrites in place)
+    int blob_off;         // byte offset of the layer's filter blob (filters, then K_pad fp32 biases) in `w`
+    int blob_bytes;
+};
+struct ChainArgs {
+    const void* x;        // input of the first layer, planar-8 with border (global)
+    void* y;              // output of the last layer, same layout
+    const void* res;      // shortcut operand of the FIRST layer (global) or nullptr
+    const void* w;        // filter blobs of all layers
+    int N, H, W, n_layers;
+    int res_mode;         // first layer: 0 none, 1 same shape as its output, 2 subsample + zero-channel pad
+    int res_H, res_W, res_C_pad, res_C, res_pad_lo, res_stride;
+    ChainLayer layers[kChainMaxLayers];
+};
+struct ChainPlan {
+    int valid;
+    int G;                // images per group (per CTA at a time)
+    int tiles;            // 128-position tiles per group
+    int plane_rows;       // vectors per channel chunk of an activation buffer
+    int buf_bytes, wbuf_bytes, acc_cols, tmem_cols;
+    int stages;           // accumulator stages in tensor memory (ring)
+    int issuers;          // MMA-issuing warps (each owns stages/issuers accumulator stages)
+    int split;            // epilogue groups per tile (1, 2, 4): each takes every split-th channel chunk
+    unsigned smem_bytes;
+};
+int chain_layer_blob_bytes(int cchunks, int K_pad);
+bool chain_layer_supported(int H, int W, int K_pad, int C_pad);
+int plan_chain_tc(const ChainArgs& a, ChainPlan* plan, char* err, size_t err_len);
+void launch_chain_tc(const ChainPlan& plan, const ChainArgs& a, int* d_status, cudaStream_t st);
 
 }  // namespace fp

@@ -114,6 +114,25 @@ __global__ void repack_conv_kernel(const float* __restrict__ w, int C, int RS, c
     }
 }
 
+// Filters of a 3x3 convolution for a fused run of layers: for tap row r and channel chunk the operand is
+// a stack of 3*K_pad 16-byte rows, row s*K_pad + kr = filter kr at horizontal tap s.
+__global__ void repack_chain_kernel(const float* __restrict__ w, int C, const int32_t* __restrict__ row_src, int K_pad,
+                                    const int32_t* __restrict__ chan_src, int C_pad, __nv_bfloat16* __restrict__ out) {
+    const size_t total = (size_t)9 * C_pad * K_pad;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int e = (int)(i % 8);
+        size_t t = i / 8;
+        const int kr = (int)(t % K_pad); t /= K_pad;
+        const int s = (int)(t % 3); t /= 3;
+        const int chunk = (int)(t % (C_pad / 8));
+        const int r = (int)(t / (C_pad / 8));
+        const int ks = row_src[kr], cs = chan_src[chunk * 8 + e];
+        float v = 0.0f;
+        if (ks >= 0 && cs >= 0) v = w[((size_t)ks * C + cs) * 9 + r * 3 + s];
+        out[i] = __float2bfloat16_rn(v);
+    }
+}
+
 // Filters of a 7x7 first convolution in the order the packed network input wants them (see
 // input_to_stem_planar_kernel): a 3x1 convolution over 80 packed channels.  Tap dr (0..2 = offsets
 // -1,0,+1), chunk 0-2 (group E) take filter row r = 2*dr + 1, chunks 3-5 (O') take r = 2*dr, chunks
@@ -200,6 +219,11 @@ void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, i
                         int C_pad, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st) {
     const size_t n = (size_t)K_pad * RS * C_pad;
     repack_conv_kernel<<<blocks_for(n, 256), 256, 0, st>>>(w, C, RS, row_src, K_pad, chan_src, C_pad, out_bf16, out_f32);
+}
+
+void launch_repack_chain(const float* w, int C, const int32_t* row_src, int K_pad, const int32_t* chan_src, int C_pad,
+                         __nv_bfloat16* out, cudaStream_t st) {
+    repack_chain_kernel<<<blocks_for((size_t)9 * C_pad * K_pad, 256), 256, 0, st>>>(w, C, row_src, K_pad, chan_src, C_pad, out);
 }
 
 void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st) {
