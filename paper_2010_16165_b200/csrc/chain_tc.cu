@@ -10,7 +10,8 @@
 //   W divides 32, so a warp of the epilogue always covers whole image rows.
 //
 //   GEMM view of one layer: M = positions (tiles of 128), K = input channels, and the three
-//   HORIZONTAL filter taps are stacked along N:   D[p, (s,k)] = sum_{r,c} x[p + (r-1)*W, c] * W'[k,c,r,s].
+//   HORIZONTAL filter taps are stacked along N:   D[p, (s,k)] = sum_{r,c} x[p + (r-1)*W, c] * W'[k,c,r,s]
+//   (column of (s,k) = 48*(k/16) + 16*s + k%16: the 48 values one thread needs for 16 channels are adjacent).
 //   The vertical taps are three accumulating MMAs whose A operand is the same shared-memory plane
 //   read from a start address shifted by (r-1)*W rows (the zero rows are the vertical padding).  The
 //   horizontal taps are recombined in the epilogue with two warp shuffles,
@@ -46,14 +47,14 @@ struct ChainParams {
     ChainArgs a;
     int G, tiles, plane_rows, buf_bytes, wbuf_bytes, tmem_cols, acc_cols, n_groups, stages, split, issuers, ring;
     int img_pos, w_shift, P2, Wp;
-    FastDiv div_img, div_ring, div_iss;
+    FastDiv div_rows;
     long long plane_in, plane_out, plane_res;
     int rP2, rWp;
     int* status;
 };
 
 constexpr int kMaxStages = 8;
-constexpr int kMaxTiles = 64;
+constexpr int kMaxTiles = 64;        // per group; a unit takes at most 32 of them (one bit each in a mask)
 
 struct ChainCtrl {
     uint64_t w_full[2], w_empty[2], tmem_full[kMaxStages], tmem_empty[kMaxStages], tile_done[2][kMaxTiles], group_sync;
@@ -146,6 +147,18 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // The W guard rows before and after each chunk plane are only read for rows whose results are discarded,
+    // but they must hold finite values (the epilogue masks neighbour terms by multiplying with 0): zero them once.
+    {
+        const int planes = 2 * (p.buf_bytes / (p.plane_rows * 16));
+        const int guard = p.a.W;
+        for (int i = threadIdx.x; i < planes * 2 * guard; i += blockDim.x) {
+            const int pl = i / (2 * guard), r = i - pl * 2 * guard;
+            const int row = r < guard ? r : p.plane_rows - 2 * guard + r;
+            *reinterpret_cast<uint4*>(act_ptr + ((size_t)pl * p.plane_rows + row) * 16) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(ctrl_addr + (uint32_t)offsetof(ChainCtrl, tmem_base)), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -197,9 +210,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         // order, which the parity waits on the stage's barriers rely on.
         const int iss = warp == 1 ? 0 : warp - (1 + kEpiThreads / 32);
         if (lane == 0 && iss < p.issuers) {
-            const uint32_t my_tiles = iss < p.tiles ? (uint32_t)((p.tiles - iss + p.issuers - 1) / p.issuers) : 0u;
             bool ok = true;
-            uint32_t it = 0;
+            uint32_t it = 0, ring_pos = 0, ring_phase = 0;     // position in this issuer's ring of accumulator stages
             for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
                 for (int l = 0; l < L && ok; ++l, ++it) {
                     const ChainLayer& ly = p.a.layers[l];
@@ -220,10 +232,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                     const uint32_t b_r0 = ((wbuf0 + wb * (uint32_t)p.wbuf_bytes) >> 4) | (N << 16);
                     const uint32_t b_r1 = b_r0 + (uint32_t)ly.cchunks * N, b_r2 = b_r1 + (uint32_t)ly.cchunks * N;
                     const uint32_t a_ks = 2u * (uint32_t)p.plane_rows, b_ks = 2u * N;
-                    uint32_t m = it * my_tiles;          // this issuer's tiles so far
-                    for (int t = iss; t < p.tiles; t += p.issuers, ++m) {
-                        const uint32_t round = fdiv(m, p.div_ring);
-                        const uint32_t stage = (uint32_t)iss + (uint32_t)p.issuers * (m - round * (uint32_t)p.ring), sph = round & 1;
+                    for (int t = iss; t < p.tiles; t += p.issuers) {
+                        const uint32_t stage = (uint32_t)iss + (uint32_t)p.issuers * ring_pos, sph = ring_phase;
+                        if (++ring_pos == (uint32_t)p.ring) { ring_pos = 0; ring_phase ^= 1; }
                         if (!mbar_wait(tempty0 + 8 * stage, sph ^ 1, abort_flag)) { ok = false; break; }
                         // the tile reads positions t*128 - W .. t*128 + 127 + W of the previous layer's output
                         if (t > 0 && !mbar_wait(td + 8 * (t - 1), tdp, abort_flag)) { ok = false; break; }
@@ -260,14 +271,22 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         // ------------------------------ load / epilogue / store ------------------------
         const int etid = threadIdx.x - 64;
         const int grp = (warp - 2) >> 2;
-        const int unit = grp / split;                 // takes tiles unit, unit + units, ...
-        const int part = grp - unit * split;          // takes channel chunks part, part + split, ...
+        const int unit = grp / split;                 // takes tiles unit, unit + units, ... (the tiles of MMA issuer `unit`)
+        const int part = grp - unit * split;          // takes 16-channel groups part, part + split, ...
         const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
         const int W = p.a.W, H = p.a.H;
+        const int wcol = lane & (W - 1);              // W divides 32: the column of this thread's positions never changes
+        const float m_left = wcol > 0 ? 1.0f : 0.0f, m_right = wcol < W - 1 ? 1.0f : 0.0f;
+        const int tiles = p.tiles;
+        const uint32_t ring = (uint32_t)p.ring, acc_cols = (uint32_t)p.acc_cols;
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int f_first = unit * 128 + quarter * 32 + lane;       // this thread's position in its first tile
+        const size_t tile_step_bytes = (size_t)units * 128 * 16;
         const uint4* __restrict__ xv = reinterpret_cast<const uint4*>(p.a.x);
         uint4* __restrict__ yv = reinterpret_cast<uint4*>(p.a.y);
         bool ok = true;
-        uint32_t it = 0, gs_it = 0;
+        uint32_t it = 0, gs_it = 0, ring_pos = 0, ring_phase = 0;
+        uint32_t pixel_mask = 0;       // bit i: this thread's position in the unit's i-th tile is a pixel of an image of the batch
         for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
             if (gs_it) {
                 // every MMA and every epilogue of the previous group has finished before its buffers are overwritten
@@ -282,13 +301,16 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 const int out_chunks = p.a.layers[0].K_pad >> 3;
                 uint8_t* b0 = act_ptr + (size_t)W * 16;
                 uint8_t* b1 = b0 + p.buf_bytes;
-                for (int t = unit; t < p.tiles; t += units) {
+                pixel_mask = 0;
+                int slot = 0;
+                for (int t = unit; t < p.tiles; t += units, ++slot) {
                     const int f = t * 128 + quarter * 32 + lane;
-                    const int img = (int)fdiv((uint32_t)f, p.div_img);
-                    const int rem = f - img * p.img_pos;
-                    const int hrow = rem >> p.w_shift, wcol = rem & (W - 1);
+                    const int row = f >> p.w_shift;
+                    const int img = (int)fdiv((uint32_t)row, p.div_rows);
+                    const int hrow = row - img * (H + 1);
                     const int n = g * p.G + img;
                     const bool pixel = hrow >= 1 && img < p.G && n < p.a.N;
+                    pixel_mask |= (pixel ? 1u : 0u) << slot;
                     const long long gpos = (long long)n * p.P2 + (long long)hrow * p.Wp + (wcol + 1);
                     for (int c = part; c < in_chunks; c += split) {
                         uint4 v = make_uint4(0, 0, 0, 0);
@@ -312,73 +334,86 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 const uint32_t wb = it & 1, wph = (it >> 1) & 1;
                 const bool last = l == L - 1;
                 if (!mbar_wait(w_full0 + 8 * wb, wph, abort_flag)) { ok = false; break; }     // the bias is in the blob
-                const int K_pad = ly.K_pad;
-                const float* bias = reinterpret_cast<const float*>(wbuf_ptr + (size_t)wb * p.wbuf_bytes +
-                                                                   (size_t)(3 * ly.cchunks * 3 * K_pad) * 16);
-                uint8_t* dst = act_ptr + (size_t)((l + 1) & 1) * p.buf_bytes + (size_t)W * 16;
-                for (int t = unit; t < p.tiles; t += units) {
-                    const int f = t * 128 + quarter * 32 + lane;
-                    const int img = (int)fdiv((uint32_t)f, p.div_img);
-                    const int rem = f - img * p.img_pos;
-                    const int hrow = rem >> p.w_shift, wcol = rem & (W - 1);
-                    const int n = g * p.G + img;
-                    const bool pixel = hrow >= 1 && img < p.G && n < p.a.N;
-                    const bool has_left = wcol > 0, has_right = wcol < W - 1;
-                    // the accumulator stage: tile t is the (t / issuers)-th tile of issuer t % issuers in this layer
-                    const uint32_t ti = fdiv((uint32_t)t, p.div_iss), is = (uint32_t)t - ti * (uint32_t)p.issuers;
-                    const uint32_t m = it * (uint32_t)((p.tiles - (int)is + p.issuers - 1) / p.issuers) + ti;
-                    const uint32_t round = fdiv(m, p.div_ring);
-                    const uint32_t stage = is + (uint32_t)p.issuers * (m - round * (uint32_t)p.ring), sph = round & 1;
+                const int K_pad = ly.K_pad, kgroups = K_pad >> 4;
+                const bool res = ly.res != 0, relu = ly.relu != 0;
+                const float4* bias4 = reinterpret_cast<const float4*>(wbuf_ptr + (size_t)wb * p.wbuf_bytes +
+                                                                      (size_t)(3 * ly.cchunks * 3 * K_pad) * 16);
+                // this thread's vector in chunk plane 0 of the destination buffer, for its first tile
+                uint8_t* dst = act_ptr + (size_t)((l + 1) & 1) * p.buf_bytes + (size_t)(W + f_first) * 16;
+                const uint32_t td_next = tdone0 + 8u * (uint32_t)kMaxTiles * ((it + 1) & 1);
+                uint32_t pm = pixel_mask;
+                for (int t = unit; t < tiles; t += units, pm >>= 1, dst += tile_step_bytes) {
+                    const bool pixel = pm & 1u;
+                    // the accumulator stage: this unit's tiles are the tiles of issuer `unit`, in the same order
+                    const uint32_t stage = (uint32_t)unit + (uint32_t)units * ring_pos, sph = ring_phase;
+                    if (++ring_pos == ring) { ring_pos = 0; ring_phase ^= 1; }
                     bool w = mbar_wait(tfull0 + 8 * stage, sph, abort_flag);
                     w = __all_sync(0xffffffffu, w);
                     if (!w) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + stage * (uint32_t)p.acc_cols;
-                    const long long gpos = (long long)n * p.P2 + (long long)hrow * p.Wp + (wcol + 1);
-                    for (int kc = part; kc < (K_pad >> 3); kc += split) {
-                        uint32_t vl[8], vc[8], vr[8];
-                        tmem_ld8(taddr + (uint32_t)(kc * 8), vl);
-                        tmem_ld8(taddr + (uint32_t)(K_pad + kc * 8), vc);
-                        tmem_ld8(taddr + (uint32_t)(2 * K_pad + kc * 8), vr);
-                        uint4* slot = reinterpret_cast<uint4*>(dst + (size_t)kc * plane_bytes + (size_t)f * 16);
-                        uint4 rv = make_uint4(0, 0, 0, 0);
-                        if (ly.res) rv = *slot;
-                        const float4 bA = *reinterpret_cast<const float4*>(bias + kc * 8);
-                        const float4 bB = *reinterpret_cast<const float4*>(bias + kc * 8 + 4);
-                        tmem_ld_wait();
-                        float o[8];
-                        const float bb[8] = {bA.x, bA.y, bA.z, bA.w, bB.x, bB.y, bB.z, bB.w};
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float lf = __shfl_up_sync(0xffffffffu, __uint_as_float(vl[i]), 1);
-                            const float rt = __shfl_down_sync(0xffffffffu, __uint_as_float(vr[i]), 1);
-                            o[i] = __uint_as_float(vc[i]) + (has_left ? lf : 0.0f) + (has_right ? rt : 0.0f) + bb[i];
-                        }
-                        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&rv);
+                    const uint32_t taddr = tmem_lane + stage * acc_cols;
+                    for (int kq = part; kq < kgroups; kq += split) {
+                        uint32_t vlc[32], vr[16];
+                        tmem_ld32(taddr + (uint32_t)(kq * 48), vlc);
+                        tmem_ld16(taddr + (uint32_t)(kq * 48 + 32), vr);
+                        uint4* slot0 = reinterpret_cast<uint4*>(dst + (size_t)(2 * kq) * plane_bytes);
+                        uint4* slot1 = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(slot0) + plane_bytes);
+                        uint4 rv[2];
+                        rv[0] = make_uint4(0, 0, 0, 0);
+                        rv[1] = rv[0];
+                        if (res) { rv[0] = *slot0; rv[1] = *slot1; }
+                        float bb[16];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const float2 q = __bfloat1622float2(h2[i]);
-                            o[2 * i] += q.x;
-                            o[2 * i + 1] += q.y;
+                            const float4 b = bias4[kq * 4 + i];
+                            bb[4 * i] = b.x; bb[4 * i + 1] = b.y; bb[4 * i + 2] = b.z; bb[4 * i + 3] = b.w;
                         }
-                        if (ly.relu) {
+                        tmem_ld_wait();
+                        // of the 48 columns: [0,16) tap s = 0, wanted by the position on the right; [16,32) the centre
+                        // tap; [32,48) tap s = 2, wanted by the position on the left.  The masks drop the neighbour's
+                        // term in the first / last column of an image row (all values involved are finite).
+                        float o[16];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) o[i] = fmaxf(o[i], 0.0f);
+                        for (int i = 0; i < 16; ++i) {
+                            const float lf = __shfl_up_sync(0xffffffffu, __uint_as_float(vlc[i]), 1);
+                            const float rt = __shfl_down_sync(0xffffffffu, __uint_as_float(vr[i]), 1);
+                            o[i] = fmaf(rt, m_right, fmaf(lf, m_left, __uint_as_float(vlc[16 + i]) + bb[i]));
                         }
-                        uint4 ov = make_uint4(0, 0, 0, 0);
+                        const uint32_t* rw = reinterpret_cast<const uint32_t*>(rv);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {                    // bf16 pair -> two floats
+                            o[2 * i] += __uint_as_float(rw[i] << 16);
+                            o[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                        }
+                        uint4 ov[2];
+                        ov[0] = make_uint4(0, 0, 0, 0);
+                        ov[1] = ov[0];
                         if (pixel) {
-                            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&ov);
+                            uint32_t* ow = reinterpret_cast<uint32_t*>(ov);
+                            if (relu) {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) o2[i] = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                                for (int i = 0; i < 8; ++i) ow[i] = pack_bf16x2_relu(o[2 * i], o[2 * i + 1]);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) ow[i] = pack_bf16x2(o[2 * i], o[2 * i + 1]);
+                            }
                         }
-                        if (!last) *slot = ov;
-                        else if (pixel) yv[(long long)kc * p.plane_out + gpos] = ov;
+                        if (!last) { *slot0 = ov[0]; *slot1 = ov[1]; }
+                        else if (pixel) {
+                            const int f = t * 128 + quarter * 32 + lane;
+                            const int row = f >> p.w_shift;
+                            const int img = (int)fdiv((uint32_t)row, p.div_rows);
+                            const int hrow = row - img * (H + 1);
+                            const long long gpos = (long long)(g * p.G + img) * p.P2 + (long long)hrow * p.Wp + (wcol + 1);
+                            yv[(long long)(2 * kq) * p.plane_out + gpos] = ov[0];
+                            yv[(long long)(2 * kq + 1) * p.plane_out + gpos] = ov[1];
+                        }
                     }
                     tc_fence_before();
                     mbar_arrive(tempty0 + 8 * stage);
                     if (!last) {
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        mbar_arrive(tdone0 + 8 * (((it + 1) & 1) * kMaxTiles + t));
+                        mbar_arrive(td_next + 8 * t);
                     }
                 }
                 if (!ok) break;
@@ -473,11 +508,10 @@ int plan_chain_tc(const ChainArgs& a, ChainPlan* plan, char* err, size_t err_len
     plan->tmem_cols = 512;                              // one CTA per SM: all of tensor memory is the accumulator ring
     plan->stages = 512 / max_N < kMaxStages ? 512 / max_N : kMaxStages;
     plan->split = plan->tiles <= 4 ? 4 : plan->tiles <= 8 ? 2 : 1;
-    // issuers: a power of two (1, 2, 4) not above the stage and tile counts; epilogue units (4 / split) must not
-    // outnumber the issuers, so that all tiles of one issuer - all uses of one accumulator stage - go to one unit
-    plan->issuers = kIssuers;
-    while (plan->issuers > 1 && (plan->issuers > plan->stages || plan->issuers > plan->tiles)) plan->issuers >>= 1;
-    if (4 / plan->split > plan->issuers) plan->split = 4 / plan->issuers;
+    // One MMA issuer per epilogue unit (4 / split of them): the tiles of an issuer, i.e. all uses of its
+    // accumulator stages, then go to one unit in the issuer's own order.  Not more units than stages or tiles.
+    while (4 / plan->split > plan->stages || 4 / plan->split > plan->tiles) plan->split *= 2;
+    plan->issuers = 4 / plan->split;
     unsigned smem = (unsigned)sizeof(ChainCtrl) + 128u + 2u * wbuf + 2u * (unsigned)plan->buf_bytes;
     if (smem < kSmemMin) smem = kSmemMin;
     plan->smem_bytes = smem;
@@ -507,9 +541,7 @@ void launch_chain_tc(const ChainPlan& plan, const ChainArgs& a, int* d_status, c
     p.img_pos = (a.H + 1) * a.W;
     p.w_shift = a.W == 8 ? 3 : a.W == 16 ? 4 : 5;
     p.Wp = a.W + 2; p.P2 = (a.H + 2) * (a.W + 2);
-    p.div_img = make_fastdiv((uint32_t)p.img_pos);
-    p.div_ring = make_fastdiv((uint32_t)p.ring);
-    p.div_iss = make_fastdiv((uint32_t)p.issuers);
+    p.div_rows = make_fastdiv((uint32_t)(a.H + 1));
     p.plane_in = (long long)a.N * p.P2;
     p.plane_out = p.plane_in;
     p.rWp = a.res_W + 2; p.rP2 = (a.res_H + 2) * (a.res_W + 2);

@@ -61,8 +61,8 @@ void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int
 // 7x7 first convolution as a 3x1 convolution over the packed network input (80 channels)
 void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st);
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st);
-// 3x3 filters of one layer of a fused run: blob[r][cp/8][s*K_pad + kr][cp%8], the three horizontal taps
-// stacked along the filter (N) axis of the MMA (see chain_tc.cu)
+// 3x3 filters of one layer of a fused run: blob[r][cp/8][48*(kr/16) + 16*s + kr%16][cp%8], the three
+// horizontal taps stacked along the filter (N) axis of the MMA (see chain_tc.cu)
 void launch_repack_chain(const float* w, int C, const int32_t* row_src, int K_pad, const int32_t* chan_src, int C_pad,
                          __nv_bfloat16* out, cudaStream_t st);
 

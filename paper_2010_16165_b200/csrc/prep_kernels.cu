@@ -115,20 +115,20 @@ __global__ void repack_conv_kernel(const float* __restrict__ w, int C, int RS, c
 }
 
 // Filters of a 3x3 convolution for a fused run of layers: for tap row r and channel chunk the operand is
-// a stack of 3*K_pad 16-byte rows, row s*K_pad + kr = filter kr at horizontal tap s.
+// a stack of 3*K_pad 16-byte rows; filter kr at horizontal tap s is row 48*(kr/16) + 16*s + kr%16.
 __global__ void repack_chain_kernel(const float* __restrict__ w, int C, const int32_t* __restrict__ row_src, int K_pad,
                                     const int32_t* __restrict__ chan_src, int C_pad, __nv_bfloat16* __restrict__ out) {
     const size_t total = (size_t)9 * C_pad * K_pad;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const int e = (int)(i % 8);
         size_t t = i / 8;
-        const int kr = (int)(t % K_pad); t /= K_pad;
-        const int s = (int)(t % 3); t /= 3;
+        const int n = (int)(t % (3 * K_pad)); t /= 3 * K_pad;
         const int chunk = (int)(t % (C_pad / 8));
         const int r = (int)(t / (C_pad / 8));
+        const int kr = (n / 48) * 16 + n % 16, sx = (n % 48) / 16;
         const int ks = row_src[kr], cs = chan_src[chunk * 8 + e];
         float v = 0.0f;
-        if (ks >= 0 && cs >= 0) v = w[((size_t)ks * C + cs) * 9 + r * 3 + s];
+        if (ks >= 0 && cs >= 0) v = w[((size_t)ks * C + cs) * 9 + r * 3 + sx];
         out[i] = __float2bfloat16_rn(v);
     }
 }
