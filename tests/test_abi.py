@@ -32,7 +32,8 @@ def test_struct_layouts_match_header():
     from paper_2010_16165_b200 import binding
     assert ctypes.sizeof(binding.fp_node) == 80
     assert binding.fp_node.w_off.offset == 56
-    assert ctypes.sizeof(binding.fp_op_info) == 16 * 4 + 3 * 8
+    assert ctypes.sizeof(binding.fp_op_info) == 16 * 4 + 3 * 8 + 2 * 4
+    assert binding.fp_op_info.chain.offset == 16 * 4 + 3 * 8
     assert binding.fp_model_desc.nodes.offset == 8
 
 
