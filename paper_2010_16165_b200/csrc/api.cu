@@ -122,6 +122,7 @@ struct fp_handle_s {
     std::vector<Op> ops;
     std::vector<Chain> chains;             // re-derived by fp_prune
     std::vector<int> op_chain;             // operator -> chain number, -1 = launched on its own
+    int input_fused = 0;                   // 1: the first fused run reads the network input directly (no layout conversion launch)
     // head
     int head_src = -1, n_classes = 0, fc_C = 0;
     const float* d_fcw = nullptr;          // classes x fc_C (copy of the description's FC weights)
@@ -568,6 +569,16 @@ fp_status find_chains(fp_handle h, const std::vector<std::vector<Use>>& uses) {
         }
         i += len >= 2 ? len : 1;
     }
+    // A run whose first layer is the only reader of the network input converts the layout while it loads.
+    h->input_fused = 0;
+    for (Chain& ch : h->chains) {
+        const FConv& f0 = h->convs[ch.convs.front()];
+        if (f0.src == 0 && uses[0].size() == 1 && !h->stem_packed) {
+            ch.args.in_mode = h->in_dtype == FP_DTYPE_BF16 ? 2 : 1;
+            ch.args.in_C = h->in_C;
+            h->input_fused = 1;
+        }
+    }
     return FP_OK;
 }
 
@@ -739,11 +750,13 @@ fp_status replan(fp_handle h) {
 void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
     const Op& op = h->ops[op_index];
     const int bf16 = h->act_is_bf16();
+    if (op.kind == 3 && h->input_fused) return;        // the first fused run reads the network input itself
     if (op.kind == 0 && h->op_chain[op_index] >= 0) {
         const Chain& ch = h->chains[h->op_chain[op_index]];
         if (op_index != ch.first_op) return;       // the run's first operator launches all of it
         fp::ChainArgs a = ch.args;
         a.N = batch;
+        if (a.in_mode) a.x = d_input;
         fp::launch_chain_tc(ch.plan, a, h->d_status, st);
         return;
     }
@@ -1036,6 +1049,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             TRY(need(4));
             int n = (int)h->ops.size() + 1;                                  // the head is two kernels
             for (const Chain& ch : h->chains) n -= (int)ch.convs.size() - 1; // a fused run is one
+            n -= h->input_fused;
             *(int32_t*)h_out = n;
             return FP_OK;
         }
@@ -1072,6 +1086,8 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
                 return fail(FP_ERR_ARG, "fp_query: operator %d has no activation output", index);
             if (h->last_batch <= 0) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
             if (h->ops[index].kind == 3 && h->stem_packed) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is stored in packed form");
+            if (h->ops[index].kind == 3 && h->input_fused) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is converted inside the first fused run "
+                                                                        "and never stored (set keep_outputs to run every layer on its own)");
             const Op& op = h->ops[index];
             const int tid = op.kind == 0 ? h->convs[op.idx].out : op.kind == 1 ? h->pools[op.idx].out : 0;
             const Tensor& t = h->tensors[tid];

@@ -65,6 +65,7 @@ struct ChainCtrl {
 static_assert(sizeof(ChainCtrl) % 16 == 0, "buffers behind the control block must stay 16-byte aligned");
 
 constexpr int kEpiThreads = 512;
+constexpr int kLoadBatch = 2;                      // tiles whose global loads a thread keeps in flight together
 constexpr int kIssuers = 4;                        // MMA-issuing warps: warp 1 and the last three
 constexpr int kThreads = 64 + kEpiThreads + 32 * (kIssuers - 1);
 
@@ -295,38 +296,95 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             }
             ++gs_it;
             // ---- load the group's images (and the first layer's shortcut operand); each thread loads the
-            //      positions and channel chunks it will later own in the epilogues ----
+            //      positions and 16-channel groups it will later own in the epilogues.  kLoadBatch tiles at a time,
+            //      all global loads of a batch issued before the first shared-memory store (latencies overlap).
+            //      The input is either a planar-8 tensor or the network input itself (NCHW, fp32 or bf16). ----
             {
-                const int in_chunks = p.a.layers[0].cchunks;
-                const int out_chunks = p.a.layers[0].K_pad >> 3;
+                const int in_groups = p.a.layers[0].cchunks >> 1;
+                const int out_groups = p.a.layers[0].K_pad >> 4;
                 uint8_t* b0 = act_ptr + (size_t)W * 16;
                 uint8_t* b1 = b0 + p.buf_bytes;
                 pixel_mask = 0;
                 int slot = 0;
-                for (int t = unit; t < p.tiles; t += units, ++slot) {
-                    const int f = t * 128 + quarter * 32 + lane;
-                    const int row = f >> p.w_shift;
-                    const int img = (int)fdiv((uint32_t)row, p.div_rows);
-                    const int hrow = row - img * (H + 1);
-                    const int n = g * p.G + img;
-                    const bool pixel = hrow >= 1 && img < p.G && n < p.a.N;
-                    pixel_mask |= (pixel ? 1u : 0u) << slot;
-                    const long long gpos = (long long)n * p.P2 + (long long)hrow * p.Wp + (wcol + 1);
-                    for (int c = part; c < in_chunks; c += split) {
-                        uint4 v = make_uint4(0, 0, 0, 0);
-                        if (pixel) v = __ldg(xv + (long long)c * p.plane_in + gpos);
-                        *reinterpret_cast<uint4*>(b0 + (size_t)c * plane_bytes + (size_t)f * 16) = v;
+                for (int tb = unit; tb < tiles; tb += kLoadBatch * units, slot += kLoadBatch) {
+                    int fq[kLoadBatch], nq[kLoadBatch], hq[kLoadBatch];
+                    bool pq[kLoadBatch];
+#pragma unroll
+                    for (int q = 0; q < kLoadBatch; ++q) {
+                        const int t = tb + q * units;
+                        const int f = t * 128 + quarter * 32 + lane;
+                        const int row = f >> p.w_shift;
+                        const int img = (int)fdiv((uint32_t)row, p.div_rows);
+                        const int hrow = row - img * (H + 1);
+                        const int n = g * p.G + img;
+                        const bool pixel = t < tiles && hrow >= 1 && img < p.G && n < p.a.N;
+                        fq[q] = f; nq[q] = n; hq[q] = hrow; pq[q] = pixel;
+                        if (t < tiles) pixel_mask |= (pixel ? 1u : 0u) << (slot + q);
                     }
-                    if (p.a.res_mode) {
-                        for (int c = part; c < out_chunks; c += split) {
-                            uint4 v = make_uint4(0, 0, 0, 0);
-                            if (pixel) v = load_residual_vec(p, c, n, hrow, wcol);
-                            *reinterpret_cast<uint4*>(b1 + (size_t)c * plane_bytes + (size_t)f * 16) = v;
+                    for (int cq = part; cq < in_groups; cq += split) {
+                        uint4 v[kLoadBatch][2];
+#pragma unroll
+                        for (int q = 0; q < kLoadBatch; ++q) {
+                            v[q][0] = make_uint4(0, 0, 0, 0);
+                            v[q][1] = v[q][0];
+                            if (!pq[q]) continue;
+                            if (p.a.in_mode == 0) {
+                                const long long gpos = (long long)nq[q] * p.P2 + (long long)hq[q] * p.Wp + (wcol + 1);
+                                v[q][0] = __ldg(xv + (long long)(2 * cq) * p.plane_in + gpos);
+                                v[q][1] = __ldg(xv + (long long)(2 * cq + 1) * p.plane_in + gpos);
+                            } else {
+                                // channels 16*cq .. 16*cq+15 of pixel (h, w) of image n, rounded to bf16
+                                const long long e0 = ((long long)nq[q] * p.a.in_C * H + (hq[q] - 1)) * W + wcol;
+                                __nv_bfloat16 tmp[16];
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) {
+                                    const int ch = 16 * cq + i;
+                                    float val = 0.0f;
+                                    if (ch < p.a.in_C) {
+                                        const long long e = e0 + (long long)ch * H * W;
+                                        val = p.a.in_mode == 1 ? __ldg(reinterpret_cast<const float*>(p.a.x) + e)
+                                                               : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.a.x)[e]);
+                                    }
+                                    tmp[i] = __float2bfloat16_rn(val);
+                                }
+                                v[q][0] = *reinterpret_cast<const uint4*>(tmp);
+                                v[q][1] = *reinterpret_cast<const uint4*>(tmp + 8);
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < kLoadBatch; ++q) {
+                            if (tb + q * units < tiles) {
+                                uint8_t* d = b0 + (size_t)(2 * cq) * plane_bytes + (size_t)fq[q] * 16;
+                                *reinterpret_cast<uint4*>(d) = v[q][0];
+                                *reinterpret_cast<uint4*>(d + plane_bytes) = v[q][1];
+                            }
                         }
                     }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic stores -> MMA operand reads
-                    mbar_arrive(tdone0 + 8 * ((it & 1) * kMaxTiles + t));
+                    if (p.a.res_mode) {
+                        for (int cq = part; cq < out_groups; cq += split) {
+                            uint4 v[kLoadBatch][2];
+#pragma unroll
+                            for (int q = 0; q < kLoadBatch; ++q) {
+                                v[q][0] = make_uint4(0, 0, 0, 0);
+                                v[q][1] = v[q][0];
+                                if (pq[q]) {
+                                    v[q][0] = load_residual_vec(p, 2 * cq, nq[q], hq[q], wcol);
+                                    v[q][1] = load_residual_vec(p, 2 * cq + 1, nq[q], hq[q], wcol);
+                                }
+                            }
+#pragma unroll
+                            for (int q = 0; q < kLoadBatch; ++q) {
+                                if (tb + q * units < tiles) {
+                                    uint8_t* d = b1 + (size_t)(2 * cq) * plane_bytes + (size_t)fq[q] * 16;
+                                    *reinterpret_cast<uint4*>(d) = v[q][0];
+                                    *reinterpret_cast<uint4*>(d + plane_bytes) = v[q][1];
+                                }
+                            }
+                        }
+                    }
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic stores -> MMA operand reads
+                for (int t = unit; t < tiles; t += units) mbar_arrive(tdone0 + 8 * ((it & 1) * kMaxTiles + t));
             }
             // ---- layers ----
             for (int l = 0; l < L && ok; ++l, ++it) {

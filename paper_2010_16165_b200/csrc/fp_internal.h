@@ -116,11 +116,13 @@ struct ChainLayer {
     int blob_bytes;
 };
 struct ChainArgs {
-    const void* x;        // input of the first layer, planar-8 with border (global)
+    const void* x;        // input of the first layer (global): planar-8 with border, or, with in_mode 1 / 2, the
+                          // network input itself: N x in_C x H x W, NCHW, fp32 / bf16 (rounded to bf16 on load)
     void* y;              // output of the last layer, same layout
     const void* res;      // shortcut operand of the FIRST layer (global) or nullptr
     const void* w;        // filter blobs of all layers
     int N, H, W, n_layers;
+    int in_mode, in_C;
     int res_mode;         // first layer: 0 none, 1 same shape as its output, 2 subsample + zero-channel pad
     int res_H, res_W, res_C_pad, res_C, res_pad_lo, res_stride;
     ChainLayer layers[kChainMaxLayers];
