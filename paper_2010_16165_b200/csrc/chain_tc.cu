@@ -101,14 +101,16 @@ __device__ __forceinline__ uint4 load_residual_vec(const ChainParams& p, int chu
 // The MMAs of one tile: three vertical taps x KSTEPS K=16 steps, unrolled with every operand address a
 // register + constant, because the issuing thread's own instruction latency is what limits narrow layers.
 template <int KSTEPS>
-__device__ __forceinline__ void issue_tile(uint32_t d_tmem, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t b0, uint32_t b1,
-                                           uint32_t b2, uint32_t a_ks, uint32_t b_ks, uint32_t idesc) {
+__device__ __forceinline__ void issue_tile(bool leader, uint32_t d_tmem, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t b0,
+                                           uint32_t b1, uint32_t b2, uint32_t a_ks, uint32_t b_ks, uint32_t idesc) {
+    if (leader) {
 #pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a0 + ks * a_ks, b0 + ks * b_ks, idesc, ks ? 1u : 0u);
+        for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a0 + ks * a_ks, b0 + ks * b_ks, idesc, ks ? 1u : 0u);
 #pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a1 + ks * a_ks, b1 + ks * b_ks, idesc, 1u);
+        for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a1 + ks * a_ks, b1 + ks * b_ks, idesc, 1u);
 #pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a2 + ks * a_ks, b2 + ks * b_ks, idesc, 1u);
+        for (int ks = 0; ks < KSTEPS; ++ks) umma_bf16_lo(d_tmem, a2 + ks * a_ks, b2 + ks * b_ks, idesc, 1u);
+    }
 }
 
 __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainParams p) {
@@ -210,7 +212,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         // the accumulator stages iss, iss + issuers, ...: all uses of a stage are then in one thread's program
         // order, which the parity waits on the stage's barriers rely on.
         const int iss = warp == 1 ? 0 : warp - (1 + kEpiThreads / 32);
-        if (lane == 0 && iss < p.issuers) {
+        // The whole warp runs the loop in step (one lane issues): operand descriptors are then warp-uniform values.
+        if (iss < p.issuers) {
+            const bool leader = lane == 0;
             bool ok = true;
             uint32_t it = 0, ring_pos = 0, ring_phase = 0;     // position in this issuer's ring of accumulator stages
             for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
@@ -245,28 +249,28 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                         const uint32_t d_tmem = tmem_base + stage * (uint32_t)p.acc_cols;
                         const uint32_t to = (uint32_t)(t * 128);
                         switch (ksteps) {
-                            case 1: issue_tile<1>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
-                            case 2: issue_tile<2>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
-                            case 3: issue_tile<3>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
-                            case 4: issue_tile<4>(d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 1: issue_tile<1>(leader, d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 2: issue_tile<2>(leader, d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 3: issue_tile<3>(leader, d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
+                            case 4: issue_tile<4>(leader, d_tmem, a_r0 + to, a_r1 + to, a_r2 + to, b_r0, b_r1, b_r2, a_ks, b_ks, idesc); break;
                             default: {
                                 uint32_t accumulate = 0;
                                 for (int r = 0; r < 3; ++r) {
                                     uint32_t a_lo = (r == 0 ? a_r0 : r == 1 ? a_r1 : a_r2) + to, b_lo = r == 0 ? b_r0 : r == 1 ? b_r1 : b_r2;
                                     for (int ks = 0; ks < ksteps; ++ks) {
-                                        umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
+                                        if (leader) umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
                                         accumulate = 1;
                                         a_lo += a_ks; b_lo += b_ks;
                                     }
                                 }
                             }
                         }
-                        umma_commit(tfull0 + 8 * stage);
+                        if (leader) umma_commit(tfull0 + 8 * stage);
                     }
-                    if (ok) umma_commit(w_empty0 + 8 * wb);     // the filter buffer is free once this warp's MMAs have read it
+                    if (ok && leader) umma_commit(w_empty0 + 8 * wb);     // the filter buffer is free once this warp's MMAs have read it
                 }
             }
-            if (!ok) raise_chain(ctrl, p.status, 12);
+            if (!ok && leader) raise_chain(ctrl, p.status, 12);
         }
     } else {
         // ------------------------------ load / epilogue / store ------------------------
