@@ -323,7 +323,7 @@ def run_gpu(args):
             "whole_step": {"flops": flops_img * w.batch, "algorithmic_bytes": whole_bytes,
                            "hbm_frac": whole_bytes / (step_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                            "tensor_frac": flops_img * w.batch / (step_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                           "sum_op_ms_no_graph": float(sum(op_ms))},
+                           "sum_op_ms": float(sum(op_ms))},
         }
     if rank == 0 and args.per_op:
         groups = {}
@@ -336,8 +336,8 @@ def run_gpu(args):
             g[2] += o.bytes_per_image * w.batch + o.bytes_fixed; g[3] += o.flops_per_image * w.batch
         out["per_op"] = [{"op": k[0], "C": k[1], "K": k[2], "R": k[3], "stride": k[4], "H": k[5], "res": k[6],
                           "launches": g[0], "us_per_launch": round(g[1] / g[0], 2),
-                          "GBps": round(g[2] / g[0] / (g[1] / g[0] * 1e-6) / 1e9, 1),
-                          "TFLOPs": round(g[3] / g[0] / (g[1] / g[0] * 1e-6) / 1e12, 2)} for k, g in groups.items()]
+                          "GBps": round(g[2] / g[1] * 1e6 / 1e9, 1) if g[1] > 0 else None,
+                          "TFLOPs": round(g[3] / g[1] * 1e6 / 1e12, 2) if g[1] > 0 else None} for k, g in groups.items()]
     B.fp_destroy(h)
     if rank == 0:
         if world == 1 and not args.no_cpu:

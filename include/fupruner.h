@@ -169,8 +169,11 @@ typedef enum {
                                 `index` from the last fp_forward (debug; synchronises the device)  */
     FP_Q_DEVICE_STATUS = 12, /* int32: 0, or FP_ERR_TIMEOUT if a bounded device wait ran out       */
     FP_Q_N_LAUNCHES = 13,    /* int32: kernels one fp_forward launches                             */
-    FP_Q_OP_TIMES = 14       /* float[N_OPS]: milliseconds per fused operator, measured now by running
-                                one forward of the last batch size with CUDA events (synchronises)  */
+    FP_Q_OP_TIMES = 14       /* float[N_OPS]: milliseconds per fused operator of a forward of the last batch size,
+                                measured now as differences of the times of the forward's prefixes (launches 0..i
+                                minus launches 0..i-1), each prefix replayed as a CUDA graph `index` times (0 = 10)
+                                between two events; a layer inside a fused run reports 0 except the run's first;
+                                synchronises */
 } fp_query_what;
 
 typedef struct {

@@ -1115,25 +1115,53 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             const int n = (int)h->ops.size();
             TRY(need((size_t)n * sizeof(float)));
             if (h->last_batch <= 0 || !h->last_input) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
-            const int reps = index > 0 ? index : 5;
-            std::vector<cudaEvent_t> ev(n + 1);
-            for (auto& e : ev) CK(cudaEventCreate(&e));
-            std::vector<float> acc(n, 0.f);
+            // Operator i's time = (time of the launches 0..i) - (time of the launches 0..i-1), each prefix of the forward
+            // captured as a CUDA graph - the way fp_forward runs them, programmatic dependent launch included - and
+            // replayed `reps` times back to back between two events.  An event between two kernels would cost more
+            // than the short kernels it is meant to time.
+            const int reps = index > 0 ? index : 10;
             cudaStream_t st;
             CK(cudaStreamCreate(&st));
-            for (int r = 0; r < reps + 1; ++r) {
-                CK(cudaEventRecord(ev[0], st));
-                for (int i = 0; i < n; ++i) {
-                    launch_op(h, i, h->last_input, h->last_batch, h->d_logits_stage, st);
-                    CK(cudaEventRecord(ev[i + 1], st));
+            cudaEvent_t e0, e1;
+            CK(cudaEventCreate(&e0));
+            CK(cudaEventCreate(&e1));
+            std::vector<float> prefix(n, 0.f);
+            fp_status rc = FP_OK;
+            for (int i = 0; i < n && rc == FP_OK; ++i) {
+                cudaGraph_t g = nullptr;
+                cudaGraphExec_t ge = nullptr;
+                if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { rc = fail(FP_ERR_CUDA, "fp_query: capture failed"); break; }
+                for (int j = 0; j <= i; ++j) launch_op(h, j, h->last_input, h->last_batch, h->d_logits_stage, st);
+                if (cudaStreamEndCapture(st, &g) != cudaSuccess || g == nullptr) { rc = fail(FP_ERR_CUDA, "fp_query: capture failed"); break; }
+                size_t n_nodes = 0;
+                cudaGraphGetNodes(g, nullptr, &n_nodes);
+                if (n_nodes == 0) {                      // nothing launched yet (e.g. a layout conversion done inside the first run)
+                    prefix[i] = i ? prefix[i - 1] : 0.f;
+                    cudaGraphDestroy(g);
+                    continue;
                 }
-                CK(cudaStreamSynchronize(st));
-                if (r == 0) continue;   // warm-up
-                for (int i = 0; i < n; ++i) { float ms; CK(cudaEventElapsedTime(&ms, ev[i], ev[i + 1])); acc[i] += ms; }
+                if (cudaGraphInstantiate(&ge, g, 0) != cudaSuccess) { cudaGraphDestroy(g); rc = fail(FP_ERR_CUDA, "fp_query: graph instantiate failed"); break; }
+                for (int k = 0; k < 3; ++k) cudaGraphLaunch(ge, st);          // warm-up
+                cudaEventRecord(e0, st);
+                for (int k = 0; k < reps; ++k) cudaGraphLaunch(ge, st);
+                cudaEventRecord(e1, st);
+                cudaError_t e = cudaStreamSynchronize(st);
+                float ms = 0.f;
+                if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+                cudaGraphExecDestroy(ge);
+                cudaGraphDestroy(g);
+                if (e != cudaSuccess) { rc = fail(FP_ERR_CUDA, "fp_query: timing failed: %s", cudaGetErrorString(e)); break; }
+                prefix[i] = ms / reps;
             }
-            for (int i = 0; i < n; ++i) ((float*)h_out)[i] = acc[i] / reps;
-            for (auto& e : ev) cudaEventDestroy(e);
+            cudaEventDestroy(e0);
+            cudaEventDestroy(e1);
             cudaStreamDestroy(st);
+            cudaGetLastError();
+            if (rc != FP_OK) return rc;
+            for (int i = 0; i < n; ++i) {
+                const float d = prefix[i] - (i ? prefix[i - 1] : 0.f);
+                ((float*)h_out)[i] = d > 0.f ? d : 0.f;
+            }
             return FP_OK;
         }
         default: return fail(FP_ERR_ARG, "fp_query: unknown query %d", what);
