@@ -1128,6 +1128,12 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             std::vector<float> prefix(n, 0.f);
             fp_status rc = FP_OK;
             for (int i = 0; i < n && rc == FP_OK; ++i) {
+                // an operator without a launch of its own (a layer inside a fused run, a layout conversion done by the
+                // first run) adds nothing to the prefix
+                const Op& op = h->ops[i];
+                const bool silent = (op.kind == 0 && h->op_chain[i] >= 0 && h->chains[h->op_chain[i]].first_op != i) ||
+                                    (op.kind == 3 && h->input_fused);
+                if (silent) { prefix[i] = i ? prefix[i - 1] : 0.f; continue; }
                 cudaGraph_t g = nullptr;
                 cudaGraphExec_t ge = nullptr;
                 if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { rc = fail(FP_ERR_CUDA, "fp_query: capture failed"); break; }

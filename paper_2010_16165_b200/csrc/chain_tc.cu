@@ -441,11 +441,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                             const float rt = __shfl_down_sync(0xffffffffu, __uint_as_float(vr[i]), 1);
                             o[i] = fmaf(rt, m_right, fmaf(lf, m_left, __uint_as_float(vlc[16 + i]) + bb[i]));
                         }
-                        const uint32_t* rw = reinterpret_cast<const uint32_t*>(rv);
+                        if (res) {
+                            const uint32_t* rw = reinterpret_cast<const uint32_t*>(rv);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {                    // bf16 pair -> two floats
-                            o[2 * i] += __uint_as_float(rw[i] << 16);
-                            o[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                            for (int i = 0; i < 8; ++i) {                // bf16 pair -> two floats
+                                o[2 * i] += __uint_as_float(rw[i] << 16);
+                                o[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                            }
                         }
                         uint4 ov[2];
                         ov[0] = make_uint4(0, 0, 0, 0);

@@ -115,3 +115,46 @@ def test_intermediate_output_query_is_refused(B):
         assert e.value.status == B.FP_ERR_UNSUPPORTED
     finally:
         g.close()
+
+
+def test_fused_runs_non_square_images_and_bf16_input(B, fpo):
+    """Images that are not square (24 x 32, then 12 x 16 and 6 x 8), network input given as bf16 NCHW: the first
+    fused run converts the layout while it loads."""
+    net = wl.resnet_cifar(2, (16, 32, 64), in_hw=32, n_classes=5, name="rect_cifar")
+    net.in_H = 24
+    w = wl.Workload("rect_cifar", net, 3, 5, True, wl.uniform_ratios(0.3), "uniform 0.3")
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC)
+    g1 = Gpu(B, w, B.FP_COMPUTE_BF16_TC, keep_outputs=1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        B.fp_prune(g1.h, w.ratios)
+        assert len(_runs(B, g.h)) == 3
+        got = g.forward(w.x)
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        assert err(got, fpo.fused_forward(gp, w.x)) < TOL_BF16
+        assert err(got, g1.forward(w.x)) < 1e-2
+        # no layout-conversion launch: 3 runs + 2 strided convolutions + 2 head kernels
+        assert B.fp_query_int(g.h, B.FP_Q_N_LAUNCHES) == 7
+    finally:
+        g.close()
+        g1.close()
+
+
+def test_operator_times_add_up(B):
+    """FP_Q_OP_TIMES: one non-negative time per operator, layers inside a run report 0 except the run's first."""
+    w = wl.tiny_cifar(widths=(16, 32, 64), in_hw=32, batch=4, n_per_stage=2, p=0.3)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        g.forward(w.x)
+        ops = B.op_infos(g.h)
+        ms = B.fp_query_array(g.h, B.FP_Q_OP_TIMES, 3, np.float32, len(ops))
+        assert (ms >= 0).all() and ms.sum() > 0
+        seen = set()
+        for o, t in zip(ops, ms):
+            if o.kind == 0 and o.chain >= 0:
+                if o.chain in seen:
+                    assert t == 0
+                seen.add(o.chain)
+    finally:
+        g.close()
