@@ -79,53 +79,80 @@ __global__ void input_to_planar_kernel(const void* __restrict__ in, int in_is_bf
 //     O (chunks 6-8):  O [p][q][j] = x[c][2p + 1][2q + s - 3]
 // (chunk 9 is zero padding to an even chunk count).  Output row p needs input rows 2p-3 .. 2p+3, which
 // are O'(p-1), E(p-1), O'(p), E(p), O'(p+1), E(p+1), O(p+1): vertical offsets -1, 0, +1 only.
+// One block per (image, output row incl. the two border rows): the three input rows the output row needs are
+// staged in shared memory (coalesced reads, each input element read once per block), then every thread builds
+// packed vectors from them.  32-bit index arithmetic only.
 __global__ void input_to_stem_planar_kernel(const void* __restrict__ in, int in_is_bf16, __nv_bfloat16* __restrict__ out,
                                             int N, int C, int H, int W) {
+    extern __shared__ float rows[];                  // [3 rows: 2p-1, 2p, 2p+1][C][W + 6], zero where outside the image
+    __shared__ int tap_off[24];                      // packed channel j = s*C + c -> c*(W+6) + s, or -1 (padding)
     const int P = H / 2, Q = W / 2, Qp = Q + 2, P2 = (P + 2) * Qp;
+    const int n = blockIdx.x / (P + 2), pp = blockIdx.x - n * (P + 2);
+    const int p = pp - 1;
     const size_t plane = (size_t)N * P2;
-    const size_t total = plane * 10;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int j8 = (int)(i / plane);             // chunk 0..9
-        const size_t f = i - (size_t)j8 * plane;
-        const size_t n = f / P2;
-        const int rem = (int)(f - n * P2);
-        const int p = rem / Qp - 1, q = rem % Qp - 1;
+    uint4* outv = reinterpret_cast<uint4*>(out) + (size_t)n * P2 + (size_t)pp * Qp;
+    if (p < 0 || p >= P) {                           // border row: zeros in every chunk
+        for (int i = threadIdx.x; i < 10 * Qp; i += blockDim.x) {
+            const int j8 = i / Qp, qq = i - j8 * Qp;
+            outv[(size_t)j8 * plane + qq] = make_uint4(0, 0, 0, 0);
+        }
+        return;
+    }
+    const int Ws = W + 6;
+    if (threadIdx.x < 24) {
+        const int sx = threadIdx.x / C, c = threadIdx.x - sx * C;
+        tap_off[threadIdx.x] = sx < 7 ? c * Ws + sx : -1;
+    }
+    for (int i = threadIdx.x; i < 3 * C * Ws; i += blockDim.x) {
+        const int rc = i / Ws, col = i - rc * Ws;
+        const int r = rc / C, c = rc - r * C;
+        const int ih = 2 * p - 1 + r, iw = col - 3;
+        float v = 0.0f;
+        if (ih >= 0 && ih < H && iw >= 0 && iw < W) {
+            const size_t src = (((size_t)n * C + c) * H + ih) * W + iw;
+            v = in_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)in)[src]) : ((const float*)in)[src];
+        }
+        rows[i] = v;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 10 * Qp; i += blockDim.x) {
+        const int j8 = i / Qp, qq = i - j8 * Qp;
+        const int q = qq - 1;
         float v[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) v[e] = 0.0f;
-        if (j8 < 9 && p >= 0 && p < P && q >= 0 && q < Q) {
-            const int group = j8 / 3;                // 0 = E, 1 = O', 2 = O
-            const int ih = group == 0 ? 2 * p : group == 1 ? 2 * p - 1 : 2 * p + 1;
-            if (ih >= 0 && ih < H) {
+        if (j8 < 9 && q >= 0 && q < Q) {
+            const int group = j8 / 3;                // 0 = E (row 2p), 1 = O' (row 2p-1), 2 = O (row 2p+1)
+            const int r = group == 0 ? 1 : group == 1 ? 0 : 2;
+            const float* base = rows + r * C * Ws + 2 * q;          // input column 2q + s - 3 sits at 2q + s
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int j = (j8 % 3) * 8 + e;  // packed channel s*C + c
-                    const int sx = j / C, c = j - sx * C;
-                    const int iw = 2 * q + sx - 3;
-                    if (sx < 7 && iw >= 0 && iw < W) {
-                        const size_t src = ((n * C + c) * H + ih) * W + iw;
-                        v[e] = in_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)in)[src]) : ((const float*)in)[src];
-                    }
-                }
+            for (int e = 0; e < 8; ++e) {
+                const int off = tap_off[(j8 - group * 3) * 8 + e];
+                if (off >= 0) v[e] = base[off];
             }
         }
-        store_vec8<true>(out, i, v);
+        Vec8h o;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o.v[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+        reinterpret_cast<Vec8h*>(outv)[(size_t)j8 * plane + qq] = o;
     }
 }
 
 // Max pooling; padded positions never win.  Output border positions are written as zeros.
+// blockIdx.x = (chunk, image, output row incl. borders), threads run along the row: no divisions per element,
+// 32-bit arithmetic, and a warp reads runs of neighbouring vectors.
 template <bool BF16>
 __global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y, int N, int H, int W, int chunks, int P,
                                int Q, int R, int stride, int pad) {
     const int Wp = W + 2, P2i = (H + 2) * Wp, Qp = Q + 2, P2o = (P + 2) * Qp;
-    const size_t plane_o = (size_t)N * P2o, plane_i = (size_t)N * P2i;
-    const size_t total = plane_o * chunks;
-    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int j = (int)(i / plane_o);
-        const size_t f = i - (size_t)j * plane_o;
-        const size_t n = f / P2o;
-        const int rem = (int)(f - n * P2o);
-        const int p = rem / Qp - 1, q = rem % Qp - 1;
+    const int rows_per_image = P + 2;
+    const int row = blockIdx.x * blockDim.y + threadIdx.y;
+    if (row >= chunks * N * rows_per_image) return;
+    const int jn = row / rows_per_image, pp = row - jn * rows_per_image;     // jn = chunk * N + image
+    const int p = pp - 1;
+    const size_t in_base = (size_t)jn * P2i, out_base = (size_t)jn * P2o + (size_t)pp * Qp;
+    for (int qq = threadIdx.x; qq < Qp; qq += blockDim.x) {
+        const int q = qq - 1;
         float m[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) m[e] = 0.0f;
@@ -135,17 +162,17 @@ __global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y,
             for (int r = 0; r < R; ++r) {
                 const int ih = p * stride + r - pad;
                 if (ih < 0 || ih >= H) continue;
-                for (int s = 0; s < R; ++s) {
-                    const int iw = q * stride + s - pad;
+                for (int sx = 0; sx < R; ++sx) {
+                    const int iw = q * stride + sx - pad;
                     if (iw < 0 || iw >= W) continue;
                     float v[8];
-                    load_vec8<BF16>(x, (size_t)j * plane_i + n * P2i + (size_t)(ih + 1) * Wp + (iw + 1), v);
+                    load_vec8<BF16>(x, in_base + (size_t)((ih + 1) * Wp + (iw + 1)), v);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) m[e] = fmaxf(m[e], v[e]);
                 }
             }
         }
-        store_vec8<BF16>(y, i, m);
+        store_vec8<BF16>(y, out_base + qq, m);
     }
 }
 
@@ -260,15 +287,18 @@ void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_i
 }
 
 void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, cudaStream_t st) {
-    const size_t n = (size_t)N * (H / 2 + 2) * (W / 2 + 2) * 10;
-    input_to_stem_planar_kernel<<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W);
+    const size_t smem = (size_t)3 * C * (W + 6) * sizeof(float);      // <= 36 KB for the supported widths
+    input_to_stem_planar_kernel<<<N * (H / 2 + 2), 256, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W);
 }
 
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
                     int stride, int pad, cudaStream_t st) {
-    const size_t n = (size_t)N * (P + 2) * (Q + 2) * (C_pad / 8);
-    if (is_bf16) maxpool_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
-    else maxpool_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
+    // the chunk planes are contiguous over the batch: (chunk, image) pairs are numbered jn = chunk * N + image
+    const int tx = Q + 2 <= 32 ? 32 : Q + 2 <= 64 ? 64 : 128, ty = 256 / tx;
+    const int rows = (C_pad / 8) * N * (P + 2);
+    const dim3 block(tx, ty), grid((rows + ty - 1) / ty);
+    if (is_bf16) maxpool_kernel<true><<<grid, block, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
+    else maxpool_kernel<false><<<grid, block, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
 }
 
 void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
