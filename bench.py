@@ -208,11 +208,12 @@ def run_gpu(args):
     dev = torch.device("cuda", local)
     peaks, peak_kind = load_peaks()
 
-    w = wl.workload(args.config, prune=args.prune)
+    w = wl.workload(args.config, prune=args.prune, aggressive=args.aggressive)
     dw, dbn = torch.from_numpy(w.weights).to(dev), torch.from_numpy(w.bn).to(dev)
     h = B.fp_fuse(w.net, dw, dbn, w.batch, B.FP_COMPUTE_BF16_TC, B.FP_DTYPE_BF16 if w.in_bf16 else B.FP_DTYPE_F32,
                   1, 0)
-    B.fp_prune(h, w.ratios)
+    if not args.no_prune:
+        B.fp_prune(h, w.ratios)
     n_classes = B.fp_query_int(h, B.FP_Q_N_CLASSES)
     x_host = torch.from_numpy(w.x)
     if w.in_bf16:
@@ -312,7 +313,9 @@ def run_gpu(args):
             "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "net": w.net.name, "batch_per_gpu": w.batch, "prune": w.ratio_spec,
-                       "norm": "l1", "fusion": "bn folded, shortcut+relu in conv epilogue, stages of 3x3 layers as one kernel", "cuda_graph": True,
+                       "norm": "l1", "pruned": not args.no_prune,
+                       "fusion": ("bn folded, shortcut filters stacked into the convolutions (Sec. IV-B)" if args.aggressive
+                                  else "bn folded, shortcut+relu in conv epilogue") + ", stages of 3x3 layers as one kernel", "cuda_graph": True,
                        "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world}"},
             "e2e": {"value": tot_units / (tot_ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(x_pinned.numel() * x_pinned.element_size()),
@@ -357,6 +360,11 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--prune", type=float, default=None)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--aggressive", action="store_true",
+                    help="fuse every block the paper's way (Sec. IV-B: identity / shortcut filters stacked into the "
+                         "convolutions, no add) instead of adding the shortcut in the epilogue")
+    ap.add_argument("--no-prune", action="store_true", help="run the fused graph without fp_prune (with --aggressive: "
+                                                            "the fused, not yet pruned operators of Table VII)")
     ap.add_argument("--per-op", action="store_true", help="add per-operator-class times to the JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
