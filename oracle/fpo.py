@@ -682,6 +682,45 @@ def pruned_model(net, weights, bn, ratios, norm=NORM_L1, masks=None):
     return prune_remove(g64, masks), masks, ranks, scores
 
 
+# ------------------------------------------------------------------------------------
+# dynamic (soft) filter pruning: the per-epoch loop of Algorithm 1
+# ------------------------------------------------------------------------------------
+
+def soft_prune_epoch(g32, ratios, norm=NORM_L2, updates=None):
+    """One pass of Algorithm 1's loop body over a fused graph built with precision='f32', in place.
+
+    `updates`: dict conv -> array shaped like that convolution's fused bank, standing for "update the
+    parameters W by using data X" (there is no trainer here): W <- W + update, one fp32 addition per
+    weight.  Then, for every convolution, the filters are scored on the updated weights, the lowest
+    n - m (fused operator) or floor(p*n) filters are zeroized - weights only, they stay in the bank and
+    the next epoch's update can bring them back - and the mask is returned.
+    Returns (masks, ranks, scores), scores taken before zeroizing.
+    """
+    if updates is not None:
+        for ci, dw in updates.items():
+            op = g32.conv_op.get(ci)
+            if op is None or dw is None:
+                continue
+            assert dw.shape == op["W"].shape
+            op["W"] = (op["W"].astype(np.float32) + np.asarray(dw, np.float32)).astype(np.float32)
+    masks, ranks, scores = select_masks(g32, ratios, norm)
+    for ci, mask in masks.items():
+        if mask is not None:
+            g32.conv_op[ci]["W"][~np.asarray(mask).astype(bool)] = 0.0
+    return masks, ranks, scores
+
+
+def soft_prune_extract(g32, masks):
+    """The last step of Algorithm 1: the model is obtained from the updated weights according to the masks
+    of the last epoch - masked filters are removed.  Returns an fp64 graph for fused_forward."""
+    g = _copy_graph(g32)
+    for op in g.ops:
+        for key in ("W", "b", "Wfc", "bfc"):
+            if key in op and op[key] is not None:
+                op[key] = np.asarray(op[key], dtype=np.float64)
+    return prune_remove(g, masks)
+
+
 def flops_and_params(g, in_hw):
     """Multiply-accumulate count per image and parameter count of a fused graph (bookkeeping pin)."""
     shapes = {0: in_hw}

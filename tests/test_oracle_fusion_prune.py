@@ -292,3 +292,72 @@ def test_planted_mistakes_are_caught(fpo):
         if o["kind"] == "conv" and o["res"] is not None and o["res"]["mode"] == "A":
             o["res"]["pad_lo"] = 3
     assert rel(fpo.fused_forward(h, w2.x), ref) > 1e-3
+
+
+# ------------------------------------------------------------------------------------------
+# dynamic (soft) pruning: the loop of Algorithm 1
+# ------------------------------------------------------------------------------------------
+
+def _soft_setup(fpo, p=0.4, aggressive=False):
+    w = wl.tiny_cifar(widths=(6, 10, 14), in_hw=8, batch=2, n_per_stage=1, p=p, aggressive=aggressive)
+    g32 = fpo.fuse(w.net, w.weights, w.bn, "f32")
+    return w, g32
+
+
+def test_soft_epoch_without_update_is_static_selection_plus_zeroing(fpo):
+    """With no weight update one epoch selects exactly the masks of the static scheme, zeroizes those filters
+    and nothing else; a second epoch then finds the same filters again (their score is exactly 0)."""
+    w, g32 = _soft_setup(fpo)
+    ref_masks, _, _ = fpo.select_masks(fpo.fuse(w.net, w.weights, w.bn, "f32"), w.ratios, fpo.NORM_L2)
+    before = {ci: op["W"].copy() for ci, op in g32.conv_op.items()}
+    masks, _, scores = fpo.soft_prune_epoch(g32, w.ratios, fpo.NORM_L2)
+    for ci, m in masks.items():
+        np.testing.assert_array_equal(m, ref_masks[ci])
+        W = g32.conv_op[ci]["W"]
+        assert (W[m == 0] == 0).all()
+        np.testing.assert_array_equal(W[m == 1], before[ci][m == 1])
+    masks2, _, scores2 = fpo.soft_prune_epoch(g32, w.ratios, fpo.NORM_L2)
+    for ci in masks:
+        np.testing.assert_array_equal(masks2[ci], masks[ci])
+        assert (scores2[ci][masks[ci] == 0] == 0).all()
+
+
+def test_soft_pruned_filter_can_recover(fpo):
+    """The point of the dynamic scheme: a zeroized filter that receives a large update is kept in the next epoch,
+    and another one takes its place (the number of pruned filters is the same every epoch)."""
+    w, g32 = _soft_setup(fpo)
+    masks, _, _ = fpo.soft_prune_epoch(g32, w.ratios, fpo.NORM_L2)
+    ci = 1
+    victim = int(np.nonzero(masks[ci] == 0)[0][0])
+    upd = {c: np.zeros_like(op["W"]) for c, op in g32.conv_op.items()}
+    upd[ci][victim] = 10.0
+    masks2, _, _ = fpo.soft_prune_epoch(g32, w.ratios, fpo.NORM_L2, upd)
+    assert masks2[ci][victim] == 1
+    assert masks2[ci].sum() == masks[ci].sum()
+    assert (masks2[ci] != masks[ci]).sum() == 2
+
+
+def test_soft_extraction_equals_zeroed_model(fpo):
+    """Removing the masked filters of the last epoch gives the same outputs as running the unshrunk model with
+    those filters (and their folded shifts) zeroed."""
+    w, g32 = _soft_setup(fpo)
+    rng = np.random.default_rng(3)
+    for _ in range(3):
+        upd = {c: (0.05 * rng.standard_normal(op["W"].shape)).astype(np.float32) for c, op in g32.conv_op.items()}
+        masks, _, _ = fpo.soft_prune_epoch(g32, w.ratios, fpo.NORM_L2, upd)
+    removed = fpo.soft_prune_extract(g32, masks)
+    full = fpo.soft_prune_extract(g32, {ci: None for ci in masks})
+    zeroed = fpo.prune_zero(full, masks)
+    a, b = fpo.fused_forward(removed, w.x), fpo.fused_forward(zeroed, w.x)
+    assert np.abs(a - b).max() <= 1e-12 * max(np.abs(b).max(), 1.0)
+
+
+def test_soft_epoch_fused_operators_lose_n_minus_m(fpo):
+    w, g32 = _soft_setup(fpo, p=0.0, aggressive=True)
+    masks, _, _ = fpo.soft_prune_epoch(g32, w.ratios, fpo.NORM_L2)
+    for ci, m in masks.items():
+        if m is None:
+            continue
+        op = g32.conv_op[ci]
+        if op["role"] in ("aggr1", "aggr2"):
+            assert int(m.sum()) == op["n_orig"]
