@@ -341,6 +341,20 @@ def run_gpu(args):
                           "launches": g[0], "us_per_launch": round(g[1] / g[0], 2),
                           "GBps": round(g[2] / g[1] * 1e6 / 1e9, 1) if g[1] > 0 else None,
                           "TFLOPs": round(g[3] / g[1] * 1e6 / 1e12, 2) if g[1] > 0 else None} for k, g in groups.items()]
+    if rank == 0 and args.soft_epochs > 0:
+        # The loop body of Algorithm 1 on the device (not part of a forward step): update + score + select + zeroize
+        # over all fused fp32 banks.  Algorithmic bytes per weight: 12 (W += dW) + 4 (score) + at most 4 (zeroize).
+        n_w = sum(B.conv_bank_elems(h))
+        upd = torch.randn(n_w, device=dev) * 0.01
+        B.fp_soft_prune_epoch(h, w.ratios, upd)             # warm-up
+        torch.cuda.synchronize()
+        t = time.perf_counter()
+        for _ in range(args.soft_epochs):
+            B.fp_soft_prune_epoch(h, w.ratios, upd)
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t) / args.soft_epochs
+        out["soft_prune_epoch"] = {"ms": 1e3 * dt, "weights": n_w, "convolutions": len([e for e in B.conv_bank_elems(h) if e]),
+                                   "GBps": 16.0 * n_w / dt / 1e9, "timed": "host wall clock around the synchronous call"}
     B.fp_destroy(h)
     if rank == 0:
         if world == 1 and not args.no_cpu:
@@ -363,6 +377,8 @@ def main():
     ap.add_argument("--aggressive", action="store_true",
                     help="fuse every block the paper's way (Sec. IV-B: identity / shortcut filters stacked into the "
                          "convolutions, no add) instead of adding the shortcut in the epilogue")
+    ap.add_argument("--soft-epochs", type=int, default=0,
+                    help="after the benchmark, time this many passes of the dynamic pruning loop (fp_soft_prune_epoch)")
     ap.add_argument("--no-prune", action="store_true", help="run the fused graph without fp_prune (with --aggressive: "
                                                             "the fused, not yet pruned operators of Table VII)")
     ap.add_argument("--per-op", action="store_true", help="add per-operator-class times to the JSON line")

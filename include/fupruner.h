@@ -173,7 +173,8 @@ typedef enum {
                                 measured now as differences of the times of the forward's prefixes (launches 0..i
                                 minus launches 0..i-1), each prefix replayed as a CUDA graph `index` times (0 = 10)
                                 between two events; a layer inside a fused run reports 0 except the run's first;
-                                synchronises */
+                                synchronises */,
+    FP_Q_CONV_BANK_ELEMS = 15 /* int64: weights in the fused fp32 bank of conv `index` (K_fused*C_fused*R*S), 0 if absorbed */
 } fp_query_what;
 
 typedef struct {
@@ -194,6 +195,33 @@ typedef struct {
 } fp_op_info;
 
 fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_out, size_t bytes);
+
+/*
+ * fp_soft_prune_epoch - one pass of the loop body of Algorithm 1 (dynamic filter pruning, Sec. IV-C): the
+ * fused fp32 filter banks are updated, every convolution's filters are scored on the updated weights (Eq. 6
+ * or the l1 sum, same fixed summation order as fp_score), and the lowest n - m (fused operator) or
+ * floor(ratio * n + 1e-9) filters are ZEROIZED in place - weights only; they stay in the bank, and the next
+ * epoch's update can bring them back.  The masks of the epoch are kept (FP_Q_MASK / FP_Q_RANK); the graph
+ * that fp_forward runs is NOT changed until fp_soft_prune_finish.
+ *   d_updates   device fp32 or NULL.  Stands for "update the parameters W by using data X" (the library has no
+ *               trainer): the concatenation, over the convolutions of the description in order (convolutions
+ *               absorbed by aggressive fusion skipped), of one addend per weight of the fused bank,
+ *               K_fused x C_fused x R x S each (FP_Q_CONV_BANK_ELEMS gives the count); W <- W + update, one
+ *               fp32 addition per weight.
+ *   h_ratios    host, one double per convolution, or NULL (= all 0); ignored for fused operators.
+ * After the first epoch the banks no longer hold the original fused weights, so a later fp_prune scores the
+ * updated, partly zeroized weights.
+ * Errors: FP_ERR_ARG, FP_ERR_EMPTY_LAYER, FP_ERR_CUDA.  Synchronous.
+ */
+fp_status fp_soft_prune_epoch(fp_handle h, int32_t norm, const double* h_ratios, const float* d_updates);
+
+/*
+ * fp_soft_prune_finish - the last step of Algorithm 1: the pruned model is obtained from the updated weights
+ * according to the masks of the last epoch: masked filters (and the matching input channels of their
+ * consumers) are removed, filters repacked, activation memory and launch plans rebuilt, as fp_prune does.
+ * Errors: FP_ERR_ARG (no epoch has run), FP_ERR_EMPTY_LAYER, FP_ERR_NOMEM, FP_ERR_CUDA.  Synchronous.
+ */
+fp_status fp_soft_prune_finish(fp_handle h);
 
 /*
  * fp_rank_filters_static - score, rank and mask the filters of ONE filter bank without allocating.

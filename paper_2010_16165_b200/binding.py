@@ -22,10 +22,10 @@ FP_COMPUTE_BF16_TC, FP_COMPUTE_FP32, FP_COMPUTE_BF16_SIMT = 0, 1, 2
 FP_NORM_L1, FP_NORM_L2 = 0, 1
 (FP_Q_N_CONVS, FP_Q_CONV_K_FUSED, FP_Q_CONV_K_KEPT, FP_Q_CONV_C_KEPT, FP_Q_MASK, FP_Q_RANK, FP_Q_N_CLASSES,
  FP_Q_FLOPS, FP_Q_BYTES, FP_Q_N_OPS, FP_Q_OP_INFO, FP_Q_OP_OUTPUT, FP_Q_DEVICE_STATUS, FP_Q_N_LAUNCHES,
- FP_Q_OP_TIMES) = range(15)
+ FP_Q_OP_TIMES, FP_Q_CONV_BANK_ELEMS) = range(16)
 
 EXPORTS = ["fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_score", "fp_query", "fp_destroy",
-           "fp_last_error", "fp_rank_filters_static"]
+           "fp_last_error", "fp_rank_filters_static", "fp_soft_prune_epoch", "fp_soft_prune_finish"]
 FP_STATIC_RANK_MAX_FILTERS = 4096
 
 
@@ -76,6 +76,8 @@ def lib():
         L.fp_score.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
         L.fp_query.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t]
         L.fp_destroy.argtypes = [ctypes.c_void_p]
+        L.fp_soft_prune_epoch.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+        L.fp_soft_prune_finish.argtypes = [ctypes.c_void_p]
         L.fp_rank_filters_static.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
@@ -172,6 +174,28 @@ def fp_rank_filters_static(d_filters, K, per_filter, norm, q, d_rank, d_mask, st
     d_mask uint8[K] CUDA tensors provided by the caller.  Asynchronous on `stream`."""
     _check(lib().fp_rank_filters_static(d_filters.data_ptr(), K, per_filter, norm, q, d_rank.data_ptr(),
                                         d_mask.data_ptr(), stream.cuda_stream if stream is not None else None))
+
+
+def fp_soft_prune_epoch(h, ratios=None, d_updates=None, norm=FP_NORM_L2):
+    """One pass of Algorithm 1's loop body.  d_updates: CUDA float32 tensor (concatenated addends of all fused
+    banks, see conv_bank_elems) or None."""
+    r = np.ascontiguousarray(ratios, dtype=np.float64) if ratios is not None else None
+    _check(lib().fp_soft_prune_epoch(h, norm, r.ctypes.data if r is not None else None,
+                                     d_updates.data_ptr() if d_updates is not None else None))
+
+
+def fp_soft_prune_finish(h):
+    _check(lib().fp_soft_prune_finish(h))
+
+
+def conv_bank_elems(h):
+    """Weights in the fused fp32 bank of every convolution of the description (0 where absorbed)."""
+    out = []
+    for ci in range(fp_query_int(h, FP_Q_N_CONVS)):
+        v = ctypes.c_int64()
+        _check(lib().fp_query(h, FP_Q_CONV_BANK_ELEMS, ci, ctypes.byref(v), 8))
+        out.append(int(v.value))
+    return out
 
 
 def fp_destroy(h):

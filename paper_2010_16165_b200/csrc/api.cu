@@ -139,6 +139,11 @@ struct fp_handle_s {
     double* d_scores = nullptr; int32_t* d_rank = nullptr; uint8_t* d_mask = nullptr;
     std::map<GraphKey, cudaGraphExec_t> graphs;
     const void* last_input = nullptr; int last_batch = 0;
+    int soft_epochs = 0;                   // passes of fp_soft_prune_epoch since fp_fuse
+    // dynamic pruning over all banks at once: bank table, filter -> bank map, scores / ranks / masks of all filters
+    fp::SoftBank* d_soft_banks = nullptr; int32_t* d_soft_map = nullptr;
+    double* d_soft_scores = nullptr; int32_t* d_soft_rank = nullptr; uint8_t* d_soft_mask = nullptr;
+    int soft_total = 0;
     int stem_packed = 0;                   // network input stored in the packed form of a 7x7/2 first convolution
     int act_is_bf16() const { return compute != FP_COMPUTE_FP32; }
     size_t act_elem() const { return act_is_bf16() ? 2 : 4; }
@@ -938,6 +943,74 @@ extern "C" fp_status fp_prune(fp_handle h, int32_t norm, const double* h_ratios,
     return replan(h);
 }
 
+// One pass of Algorithm 1's loop body: update, score, select, zeroize in place.  The running graph is untouched.
+extern "C" fp_status fp_soft_prune_epoch(fp_handle h, int32_t norm, const double* h_ratios, const float* d_updates) {
+    if (!h) return fail(FP_ERR_ARG, "fp_soft_prune_epoch: NULL handle");
+    if (norm != FP_NORM_L1 && norm != FP_NORM_L2) return fail(FP_ERR_ARG, "fp_soft_prune_epoch: bad norm");
+    // validate everything before the banks are touched
+    std::vector<int> q(h->convs.size(), 0);
+    for (size_t i = 0; i < h->convs.size(); ++i) {
+        const FConv& f = h->convs[i];
+        if (f.role != 0) q[i] = f.K - f.n_orig;
+        else {
+            const double r = h_ratios ? h_ratios[f.conv_index] : 0.0;
+            if (!(r >= 0.0) || r > 1.0) return fail(FP_ERR_ARG, "fp_soft_prune_epoch: ratio of convolution %d outside [0,1]", f.conv_index);
+            q[i] = (int)std::floor(r * (double)f.K + 1e-9);
+        }
+        if (q[i] >= f.K) return fail(FP_ERR_EMPTY_LAYER, "fp_soft_prune_epoch: convolution %d would keep no filter", f.conv_index);
+    }
+    // bank table in description order (the order of the update array), filters numbered bank by bank
+    std::vector<fp::SoftBank> banks;
+    std::vector<int32_t> map;
+    std::vector<size_t> fused_of;
+    long long off = 0;
+    int k_off = 0, max_K = 1;
+    for (int ci = 0; ci < h->n_desc_convs; ++ci) {
+        if (h->conv_to_fused[ci] < 0) continue;
+        const size_t i = (size_t)h->conv_to_fused[ci];
+        const FConv& f = h->convs[i];
+        fp::SoftBank b;
+        b.w = f.d_w32; b.dw_off = off; b.K = f.K; b.per = f.C * f.R * f.S; b.q = q[i]; b.k_off = k_off;
+        for (int k = 0; k < f.K; ++k) map.push_back((int32_t)banks.size());
+        banks.push_back(b);
+        fused_of.push_back(i);
+        off += (long long)f.K * b.per;
+        k_off += f.K;
+        max_K = std::max(max_K, f.K);
+    }
+    if (!h->d_soft_banks) {
+        h->soft_total = k_off;
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_soft_banks, banks.size() * sizeof(fp::SoftBank)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_soft_map, map.size() * sizeof(int32_t)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_soft_scores, (size_t)k_off * sizeof(double)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_soft_rank, (size_t)k_off * sizeof(int32_t)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&h->d_soft_mask, (size_t)k_off));
+        CK(cudaMemcpy(h->d_soft_map, map.data(), map.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    }
+    CK(cudaMemcpy(h->d_soft_banks, banks.data(), banks.size() * sizeof(fp::SoftBank), cudaMemcpyHostToDevice));
+    fp::launch_soft_update_score(h->d_soft_banks, h->d_soft_map, k_off, d_updates, norm, h->d_soft_scores, 0);
+    fp::launch_soft_rank(h->d_soft_banks, (int)banks.size(), max_K, h->d_soft_scores, h->d_soft_rank, h->d_soft_mask, 0);
+    fp::launch_soft_zeroize(h->d_soft_banks, h->d_soft_map, k_off, h->d_soft_mask, 0);
+    CK(cudaGetLastError());
+    std::vector<int32_t> all_rank(k_off);
+    std::vector<uint8_t> all_mask(k_off);
+    CK(cudaMemcpy(all_rank.data(), h->d_soft_rank, (size_t)k_off * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(all_mask.data(), h->d_soft_mask, (size_t)k_off, cudaMemcpyDeviceToHost));
+    for (size_t bi = 0; bi < banks.size(); ++bi) {
+        FConv& f = h->convs[fused_of[bi]];
+        f.rank.assign(all_rank.begin() + banks[bi].k_off, all_rank.begin() + banks[bi].k_off + f.K);
+        f.mask.assign(all_mask.begin() + banks[bi].k_off, all_mask.begin() + banks[bi].k_off + f.K);
+    }
+    ++h->soft_epochs;
+    return FP_OK;
+}
+
+extern "C" fp_status fp_soft_prune_finish(fp_handle h) {
+    if (!h) return fail(FP_ERR_ARG, "fp_soft_prune_finish: NULL handle");
+    if (h->soft_epochs == 0) return fail(FP_ERR_ARG, "fp_soft_prune_finish: no fp_soft_prune_epoch has run");
+    return replan(h);
+}
+
 extern "C" fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch, float* d_logits, void* stream) {
     if (!h || !d_input || !d_logits) return fail(FP_ERR_ARG, "fp_forward: NULL argument");
     if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward: batch must be positive");
@@ -1056,6 +1129,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
         case FP_Q_CONV_K_FUSED: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K : 0; return FP_OK;
         case FP_Q_CONV_K_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->K_kept : 0; return FP_OK;
         case FP_Q_CONV_C_KEPT: TRY(need(4)); TRY(conv_of(&f)); *(int32_t*)h_out = f ? f->C_kept : 0; return FP_OK;
+        case FP_Q_CONV_BANK_ELEMS: TRY(need(8)); TRY(conv_of(&f)); *(int64_t*)h_out = f ? (int64_t)f->K * f->C * f->R * f->S : 0; return FP_OK;
         case FP_Q_MASK:
             TRY(conv_of(&f));
             if (!f) return fail(FP_ERR_ARG, "fp_query: convolution %d was absorbed by fusion", index);

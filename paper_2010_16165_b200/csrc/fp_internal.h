@@ -52,6 +52,24 @@ void launch_identity_filters(float* dst, int C_dst, int R, int S, int k0, int c0
 void launch_count_nonfinite(const float* p, size_t n, int* d_count, cudaStream_t st);
 void launch_score_filters(const float* w, int K, int per_filter, int norm, double* scores, cudaStream_t st);
 void launch_rank_mask(const double* scores, int K, int q, int32_t* rank, uint8_t* mask, cudaStream_t st);
+// Algorithm 1's loop body over ALL filter banks of a model in three launches.  One SoftBank per convolution;
+// filter_bank[g] names the bank of global filter g (filters of all banks numbered consecutively, bank by bank).
+struct SoftBank {
+    float* w;             // K x per fp32, updated and zeroized in place
+    long long dw_off;     // element offset of the bank's addends in the update array
+    int K, per, q;        // filters, weights per filter, filters to zeroize
+    int k_off;            // global number of the bank's first filter
+};
+// w += dw (one fp32 addition per weight; dw may be nullptr) and the filter scores of the updated weights, in the
+// fixed summation order of launch_score_filters
+void launch_soft_update_score(const SoftBank* banks, const int32_t* filter_bank, int total_filters, const float* dw,
+                              int norm, double* scores, cudaStream_t st);
+// per bank: rank by (score, index) ascending, mask the first q (one block per bank)
+void launch_soft_rank(const SoftBank* banks, int n_banks, int max_K, const double* scores, int32_t* rank, uint8_t* mask,
+                      cudaStream_t st);
+// masked filters become zero
+void launch_soft_zeroize(const SoftBank* banks, const int32_t* filter_bank, int total_filters, const uint8_t* mask,
+                         cudaStream_t st);
 // Convolution filters: packed[rs][cp/8][kr][cp%8] = w[row_src[kr]][chan_src[cp]][rs] (zero where an index is -1)
 void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
                         int C_pad, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st);

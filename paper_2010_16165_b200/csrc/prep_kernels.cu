@@ -92,6 +92,59 @@ __global__ void rank_mask_kernel(const double* __restrict__ scores, int K, int q
     }
 }
 
+// Algorithm 1's loop body over all banks.  One warp per filter: lane l updates and accumulates elements l, l+32, ...
+// in increasing order, then the 32 partial sums are combined pairwise at distances 16, 8, 4, 2, 1 - the order
+// that defines a score (see score_filters_kernel).
+__global__ void soft_update_score_kernel(const SoftBank* __restrict__ banks, const int32_t* __restrict__ filter_bank,
+                                         int total_filters, const float* __restrict__ dw, int norm,
+                                         double* __restrict__ scores) {
+    const int g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (g >= total_filters) return;
+    const SoftBank b = banks[filter_bank[g]];
+    const int k = g - b.k_off;
+    float* f = b.w + (size_t)k * b.per;
+    const float* d = dw ? dw + b.dw_off + (size_t)k * b.per : nullptr;
+    double s = 0.0;
+    for (int t = lane; t < b.per; t += 32) {
+        float v = f[t];
+        if (d) { v = __fadd_rn(v, d[t]); f[t] = v; }
+        const double x = (double)v;
+        s = __dadd_rn(s, norm ? __dmul_rn(x, x) : fabs(x));
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) s = __dadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
+    if (lane == 0) scores[g] = s;
+}
+
+__global__ void soft_rank_kernel(const SoftBank* __restrict__ banks, const double* __restrict__ scores,
+                                 int32_t* __restrict__ rank, uint8_t* __restrict__ mask) {
+    extern __shared__ double sh[];
+    const SoftBank b = banks[blockIdx.x];
+    for (int i = threadIdx.x; i < b.K; i += blockDim.x) sh[i] = scores[b.k_off + i];
+    __syncthreads();
+    for (int k = threadIdx.x; k < b.K; k += blockDim.x) {
+        const double sk = sh[k];
+        int before = 0;
+        for (int j = 0; j < b.K; ++j) {
+            const double sj = sh[j];
+            before += (sj < sk) || (sj == sk && j < k);
+        }
+        rank[b.k_off + k] = before;
+        mask[b.k_off + k] = before >= b.q ? 1 : 0;
+    }
+}
+
+__global__ void soft_zeroize_kernel(const SoftBank* __restrict__ banks, const int32_t* __restrict__ filter_bank,
+                                    int total_filters, const uint8_t* __restrict__ mask) {
+    const int g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (g >= total_filters || mask[g]) return;
+    const SoftBank b = banks[filter_bank[g]];
+    float* f = b.w + (size_t)(g - b.k_off) * b.per;
+    for (int t = lane; t < b.per; t += 32) f[t] = 0.0f;
+}
+
 // Filters of one convolution in the order the MMA wants them: tap-major, then chunks of 8 input
 // channels, then the filter, then the channel within the chunk.  For a fixed tap and chunk the
 // K_pad x 8 block is a stack of 16-byte rows - the canonical K-major operand layout without swizzle.
@@ -213,6 +266,23 @@ void launch_score_filters(const float* w, int K, int per_filter, int norm, doubl
 
 void launch_rank_mask(const double* scores, int K, int q, int32_t* rank, uint8_t* mask, cudaStream_t st) {
     rank_mask_kernel<<<1, 256, (size_t)K * sizeof(double), st>>>(scores, K, q, rank, mask);
+}
+
+void launch_soft_update_score(const SoftBank* banks, const int32_t* filter_bank, int total_filters, const float* dw,
+                              int norm, double* scores, cudaStream_t st) {
+    const int warps_per_block = 8;
+    soft_update_score_kernel<<<(total_filters + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+        banks, filter_bank, total_filters, dw, norm, scores);
+}
+void launch_soft_rank(const SoftBank* banks, int n_banks, int max_K, const double* scores, int32_t* rank, uint8_t* mask,
+                      cudaStream_t st) {
+    soft_rank_kernel<<<n_banks, 256, (size_t)max_K * sizeof(double), st>>>(banks, scores, rank, mask);
+}
+void launch_soft_zeroize(const SoftBank* banks, const int32_t* filter_bank, int total_filters, const uint8_t* mask,
+                         cudaStream_t st) {
+    const int warps_per_block = 8;
+    soft_zeroize_kernel<<<(total_filters + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+        banks, filter_bank, total_filters, mask);
 }
 
 void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
