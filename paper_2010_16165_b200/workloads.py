@@ -298,7 +298,8 @@ def inner_bottleneck_ratios(p):
 
 
 def workload(config, batch=None, prune=None, aggressive=False):
-    """The five benchmark-shaped workloads.  ``config`` in 1..5; batch/prune override the defaults."""
+    """The five benchmark-shaped workloads (``config`` 1..5) and the two other networks of the paper's Table II
+    (6: ResNet-32, 7: ResNet-34); batch/prune override the defaults."""
     seed = BASE_SEED + config
     if config == 1:
         net = resnet_cifar(3, aggressive=aggressive)
@@ -321,7 +322,15 @@ def workload(config, batch=None, prune=None, aggressive=False):
         p = 0.4 if prune is None else prune
         return Workload(f"resnet50_b{batch or 128}_inner{p}", net, batch or 128, seed, True,
                         inner_bottleneck_ratios(p), f"inner bottleneck {p}")
-    raise ValueError("config must be 1..5")
+    if config == 6:      # the paper's second CIFAR model (Table II), shaped like config 2
+        net = resnet_cifar(5, aggressive=aggressive)
+        p = 0.3 if prune is None else prune
+        return Workload(f"resnet32_b{batch or 256}_p{p}", net, batch or 256, seed, True, uniform_ratios(p), f"uniform {p}")
+    if config == 7:      # the paper's second ImageNet model (Table II), shaped like config 4
+        net = resnet_imagenet_basic((3, 4, 6, 3), aggressive=aggressive)
+        p = 0.3 if prune is None else prune
+        return Workload(f"resnet34_b{batch or 64}_p{p}", net, batch or 64, seed, True, uniform_ratios(p), f"uniform {p}")
+    raise ValueError("config must be 1..7")
 
 
 def tiny_cifar(n_per_stage=1, widths=(8, 16, 24), in_hw=8, batch=2, seed=7, aggressive=False, p=0.0,

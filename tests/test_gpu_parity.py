@@ -377,6 +377,12 @@ def test_config5_resnet50(B, fpo):
     _full_config(B, fpo, w1, 1, also_fp32=False)
 
 
+def test_paper_models_resnet32_and_resnet34(B, fpo):
+    """The two networks of the paper's Table II that the five workloads do not cover."""
+    _full_config(B, fpo, wl.workload(6), 6)
+    _full_config(B, fpo, wl.workload(7, batch=8), 1)
+
+
 def test_config1_aggressive_fused_unpruned_and_pruned(B, fpo):
     """The paper's own graph: dilated convolutions, no add; then pruned back by n-m filters."""
     w = wl.workload(1, aggressive=True)
