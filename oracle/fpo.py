@@ -393,6 +393,45 @@ def fuse(net, weights, bn, precision="f64"):
                 # ---- aggressive fusion of the block (Sec. IV-B) ---------------------------
                 f1 = producer[h_tid]
                 n2 = nodes[conv2_id]
+                fa = producer.get(f1["src"]) if f1["kind"] == "conv" else None
+                if (fa is not None and fa["kind"] == "conv" and fa["src"] == x_tid and n2["R"] == 1 and n2["S"] == 1):
+                    # ---- bottleneck block (not in the paper, which stops at basic blocks): the block input is
+                    #      carried through all three convolutions.  conv1'' = [W1 ; I] (1x1), conv2'' = diag(W2, I at
+                    #      the centre tap) so that the pass-through is subsampled with conv2's stride, conv3'' =
+                    #      [W3 | S] with S the identity or the projection's 1x1 filters; no add remains. ----
+                    fb = f1                                               # the 3x3 convolution
+                    if not (fa["relu"] and fb["relu"] and fa["res"] is None and fb["res"] is None
+                            and fa["W"].shape[2:] == (1, 1) and fa["stride"] == 1 and fa["pad"] == 0
+                            and fb["W"].shape[2:] == (3, 3) and fb["pad"] == 1
+                            and n2["stride"] == 1 and n2["pad"] == 0 and mode in ("id", "proj")):
+                        raise ValueError("aggressive fusion of a three-convolution block needs 1x1 - 3x3 - 1x1")
+                    xp = producer.get(x_tid)
+                    if xp is None or (xp["kind"] == "conv" and not xp["relu"]):
+                        raise ValueError("aggressive fusion needs a block input that is a ReLU output")
+                    Kw, C = fa["W"].shape[0], fa["W"].shape[1]
+                    K3 = W2.shape[0]
+                    fa["W"] = np.concatenate([fa["W"], _identity_filters(C, C, 1, 1, 0, dt)], axis=0)
+                    fa["b"] = np.concatenate([fa["b"], np.zeros(C, dtype=dt)])
+                    fa["role"], fa["K_full"] = "aggr1", Kw + C
+                    Wd = np.zeros((Kw + C, Kw + C, 3, 3), dtype=dt)
+                    Wd[:Kw, :Kw] = fb["W"]
+                    Wd[Kw:, Kw:] = _identity_filters(C, C, 3, 3, 0, dt)
+                    fb["W"] = Wd
+                    fb["b"] = np.concatenate([fb["b"], np.zeros(C, dtype=dt)])
+                    fb["role"], fb["K_full"] = "aggr1", Kw + C
+                    absorbed = ()
+                    if mode == "id":
+                        Sw, bsum = _identity_filters(K3, C, 1, 1, 0, dt), b2
+                    else:
+                        ps = sc["in0"]
+                        Ws, bs, _ = folded(ps)
+                        if nodes[ps]["stride"] != fb["stride"] or nodes[ps]["pad"] != 0 or Ws.shape[2:] != (1, 1):
+                            raise ValueError("projection shortcut must be 1x1 with the 3x3 convolution's stride")
+                        Sw, bsum, absorbed = Ws, (b2 + bs).astype(dt), (ps,)
+                    o = emit_conv(conv2_id, np.concatenate([W2, Sw], axis=1), bsum, h_tid, True, None, role="aggr2",
+                                  absorbed=absorbed)
+                    tensor_of[relu_id] = o["out"]
+                    continue
                 if not (f1["kind"] == "conv" and f1["src"] == x_tid and f1["relu"] and f1["res"] is None
                         and f1["W"].shape[2:] == (3, 3) and f1["pad"] == 1
                         and n2["R"] == 3 and n2["S"] == 3 and n2["stride"] == 1 and n2["pad"] == 1):

@@ -114,9 +114,9 @@ def _basic_block(net, x, C, K, stride, shortcut, block, aggressive, pad_lo=0):
     return net.relu(y, **kw)
 
 
-def _bottleneck(net, x, C, width, stride, project, block):
+def _bottleneck(net, x, C, width, stride, project, block, aggressive=0):
     """1x1-3x3(stride)-1x1 bottleneck, expansion 4; stride sits on the 3x3 conv."""
-    kw = dict(block=block)
+    kw = dict(block=block, aggressive=aggressive)
     K = 4 * width
     h = net.relu(net.bn(net.conv(x, width, C, 1, 1, 0, **kw), width, **kw), **kw)
     h = net.relu(net.bn(net.conv(h, width, width, 3, stride, 1, **kw), width, **kw), **kw)
@@ -178,7 +178,7 @@ def resnet_imagenet_basic(layers=(2, 2, 2, 2), widths=(64, 128, 256, 512), in_hw
 
 
 def resnet_imagenet_bottleneck(layers=(3, 4, 6, 3), widths=(64, 128, 256, 512), in_hw=224,
-                               n_classes=1000, name=None, stem_k=7, stem_width=64):
+                               n_classes=1000, name=None, stem_k=7, stem_width=64, aggressive=False):
     """ImageNet-shaped ResNet-50: bottleneck blocks, projection on the first block of every stage."""
     net = Net(3, in_hw, in_hw, name or f"resnet{3 * sum(layers) + 2}")
     x = net.relu(net.bn(net.conv(-1, stem_width, 3, stem_k, 2, stem_k // 2), stem_width))
@@ -188,7 +188,7 @@ def resnet_imagenet_bottleneck(layers=(3, 4, 6, 3), widths=(64, 128, 256, 512), 
     for si, wd in enumerate(widths):
         for bi in range(layers[si]):
             first = bi == 0
-            x = _bottleneck(net, x, C, wd, 2 if (first and si > 0) else 1, first, block)
+            x = _bottleneck(net, x, C, wd, 2 if (first and si > 0) else 1, first, block, _aggr(aggressive, block))
             C = 4 * wd
             block += 1
     x = net.gavgpool(x, C)
@@ -348,6 +348,7 @@ def tiny_imagenet_basic(layers=(1, 1, 1), widths=(8, 12, 20), in_hw=32, batch=2,
     return Workload("tiny_imagenet_basic", net, batch, seed, False, uniform_ratios(p), f"uniform {p}")
 
 
-def tiny_bottleneck(layers=(1, 2), widths=(4, 8), in_hw=32, batch=2, seed=13, p=0.0):
-    net = resnet_imagenet_bottleneck(layers, widths, in_hw, n_classes=6, name="tiny_bottleneck", stem_width=8)
+def tiny_bottleneck(layers=(1, 2), widths=(4, 8), in_hw=32, batch=2, seed=13, p=0.0, aggressive=False):
+    net = resnet_imagenet_bottleneck(layers, widths, in_hw, n_classes=6, name="tiny_bottleneck", stem_width=8,
+                                     aggressive=aggressive)
     return Workload("tiny_bottleneck", net, batch, seed, False, inner_bottleneck_ratios(p), f"inner {p}")

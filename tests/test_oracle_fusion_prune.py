@@ -361,3 +361,41 @@ def test_soft_epoch_fused_operators_lose_n_minus_m(fpo):
         op = g32.conv_op[ci]
         if op["role"] in ("aggr1", "aggr2"):
             assert int(m.sum()) == op["n_orig"]
+
+
+# ------------------------------------------------------------------------------------------
+# aggressive fusion of bottleneck blocks (the pass-through carried through three convolutions)
+# ------------------------------------------------------------------------------------------
+
+def test_aggressive_bottleneck_equals_unfused(fpo):
+    w = wl.tiny_bottleneck(aggressive=True)
+    g = fpo.fuse(w.net, w.weights, w.bn)
+    assert not any(op["kind"] == "conv" and op["res"] is not None for op in g.ops), "an add survived"
+    ref = fpo.unfused_forward(w.net, w.weights, w.bn, w.x)
+    got = fpo.fused_forward(g, w.x)
+    assert np.abs(got - ref).max() <= 1e-12 * np.abs(ref).max()
+    # and the same as the epilogue form of the same network
+    w0 = wl.tiny_bottleneck(aggressive=False)
+    np.testing.assert_array_equal(w0.weights, w.weights)
+    g0 = fpo.fuse(w0.net, w0.weights, w0.bn)
+    assert np.abs(fpo.fused_forward(g0, w.x) - got).max() <= 1e-12 * np.abs(ref).max()
+
+
+def test_aggressive_bottleneck_loses_n_minus_m(fpo):
+    w = wl.tiny_bottleneck(aggressive=True)
+    g32 = fpo.fuse(w.net, w.weights, w.bn, "f32")
+    masks, _, _ = fpo.select_masks(g32, np.zeros(w.net.n_convs()), fpo.NORM_L1)
+    n_fused = 0
+    for ci, m in masks.items():
+        if m is None:
+            continue
+        op = g32.conv_op[ci]
+        if op["role"] in ("aggr1", "aggr2"):
+            n_fused += 1
+            assert int(m.sum()) == op["n_orig"] and len(m) >= op["n_orig"]
+    assert n_fused == 9          # three blocks x three convolutions
+    # removal and zeroing of that selection agree
+    g = fpo.fuse(w.net, w.weights, w.bn)
+    a = fpo.fused_forward(fpo.prune_remove(g, masks), w.x)
+    b = fpo.fused_forward(fpo.prune_zero(g, masks), w.x)
+    assert np.abs(a - b).max() <= 1e-12 * max(np.abs(b).max(), 1.0)
