@@ -41,7 +41,8 @@ typedef enum {
     FP_ERR_NONFINITE = -4,    /* NaN/Inf in weights or BN statistics                            */
     FP_ERR_CUDA = -5,         /* a CUDA runtime/driver call failed (message has the CUDA error) */
     FP_ERR_NOMEM = -6,        /* device allocation failed                                       */
-    FP_ERR_UNSUPPORTED = -7,  /* valid request the library cannot run (e.g. aggressive bottleneck) */
+    FP_ERR_UNSUPPORTED = -7,  /* valid request the library cannot run (e.g. an aggressive block that is neither
+                                 3x3-3x3 nor 1x1-3x3-1x1, an image wider than 512 pixels)            */
     FP_ERR_TIMEOUT = -8,      /* a bounded device-side wait ran out; results are invalid        */
     FP_ERR_EMPTY_LAYER = -9,  /* a mask or ratio would remove every filter of a convolution     */
     FP_ERR_BOUNDS = -10       /* batch larger than max_batch, size beyond a stated maximum      */

@@ -253,6 +253,76 @@ struct Builder {
         return false;
     }
 
+    // Aggressive fusion of a three-convolution (bottleneck) block, which the paper does not describe (it stops at
+    // two-convolution blocks): the block input is carried through all three convolutions.  conv1'' = [W1' ; I]
+    // (1x1), conv2'' = diag(W2', I at the centre tap) - the pass-through is subsampled with conv2's stride -,
+    // conv3'' = [W3' | S] with S the identity or the projection's folded 1x1 filters; no add remains.
+    fp_status fuse_bottleneck(int id, int relu_id, int conv3_id, int fbi, int x_tid, int h_tid, int mode, int proj_id) {
+        const fp_node& c3 = h->nodes[conv3_id];
+        const FConv fb0 = h->convs[fbi];                                   // the 3x3 convolution
+        const int pa = h->tensors[fb0.src].producer;
+        if (pa < 0 || h->ops[pa].kind != 0)
+            return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion needs a 1x1 - 3x3 - 1x1 block", id);
+        const int fai = h->ops[pa].idx;
+        const FConv fa0 = h->convs[fai];                                   // the first 1x1 convolution
+        if (fa0.src != x_tid || !fa0.relu || !fb0.relu || fa0.res_mode || fb0.res_mode || fa0.role || fb0.role ||
+            fa0.R != 1 || fa0.S != 1 || fa0.stride != 1 || fa0.pad != 0 || fb0.R != 3 || fb0.S != 3 || fb0.pad != 1 ||
+            c3.stride != 1 || c3.pad != 0 || mode == 1)
+            return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion needs a 1x1 - 3x3 - 1x1 block with an identity or projection shortcut", id);
+        if (!is_relu_output(x_tid))
+            return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion needs a block input that is a ReLU output", id);
+        const int C = fa0.C, Kw = fa0.K;
+        if (fb0.K != Kw || fb0.C != Kw || c3.C != Kw) return fail(FP_ERR_SHAPE, "node %d: bottleneck widths differ", id);
+        {   // conv1'': C identity filters under the 1x1 convolution
+            float *nw, *nb;
+            TRY(dev_alloc(h->fixed_buffers, (void**)&nw, (size_t)(Kw + C) * C * sizeof(float)));
+            TRY(dev_alloc(h->fixed_buffers, (void**)&nb, (size_t)(Kw + C) * sizeof(float)));
+            CK(cudaMemsetAsync(nw, 0, (size_t)(Kw + C) * C * sizeof(float), st));
+            CK(cudaMemsetAsync(nb, 0, (size_t)(Kw + C) * sizeof(float), st));
+            CK(cudaMemcpyAsync(nw, fa0.d_w32, (size_t)Kw * C * sizeof(float), cudaMemcpyDeviceToDevice, st));
+            CK(cudaMemcpyAsync(nb, fa0.d_b32, (size_t)Kw * sizeof(float), cudaMemcpyDeviceToDevice, st));
+            fp::launch_identity_filters(nw, C, 1, 1, Kw, 0, C, C, 0, st);
+            FConv& fa = h->convs[fai];
+            fa.d_w32 = nw; fa.d_b32 = nb; fa.K = Kw + C; fa.role = 1;
+            h->tensors[fa.out].C_full = Kw + C;
+        }
+        {   // conv2'': block diagonal, the pass-through on the centre tap
+            const int n = Kw + C;
+            float *nw, *nb;
+            TRY(dev_alloc(h->fixed_buffers, (void**)&nw, (size_t)n * n * 9 * sizeof(float)));
+            TRY(dev_alloc(h->fixed_buffers, (void**)&nb, (size_t)n * sizeof(float)));
+            CK(cudaMemsetAsync(nw, 0, (size_t)n * n * 9 * sizeof(float), st));
+            CK(cudaMemsetAsync(nb, 0, (size_t)n * sizeof(float), st));
+            CK(cudaMemcpy2DAsync(nw, (size_t)n * 9 * sizeof(float), fb0.d_w32, (size_t)Kw * 9 * sizeof(float),
+                                 (size_t)Kw * 9 * sizeof(float), Kw, cudaMemcpyDeviceToDevice, st));
+            CK(cudaMemcpyAsync(nb, fb0.d_b32, (size_t)Kw * sizeof(float), cudaMemcpyDeviceToDevice, st));
+            fp::launch_identity_filters(nw, n, 3, 3, Kw, Kw, C, C, 0, st);
+            FConv& fb = h->convs[fbi];
+            fb.d_w32 = nw; fb.d_b32 = nb; fb.K = n; fb.C = n; fb.role = 1;
+            h->tensors[fb.out].C_full = n;
+        }
+        int ci;
+        TRY(emit_conv(conv3_id, h_tid, 1, C, &ci));            // K3 x (Kw + C), conv3 folded into columns [0,Kw)
+        FConv& f = h->convs[ci];
+        f.role = 2;
+        if (mode == 0) {
+            if (f.K != C) return fail(FP_ERR_SHAPE, "node %d: identity shortcut needs as many filters as block inputs", id);
+            fp::launch_identity_filters(f.d_w32, f.C, 1, 1, 0, Kw, f.K, C, 0, st);
+        } else {
+            TRY(check_conv_node(proj_id));
+            const fp_node& pr = h->nodes[proj_id];
+            if (pr.R != 1 || pr.S != 1 || pr.pad != 0 || pr.stride != fb0.stride || pr.C != C || pr.K != f.K)
+                return fail(FP_ERR_UNSUPPORTED, "node %d: projection shortcut must be 1x1 with the 3x3 convolution's stride", id);
+            const fp_node& pb = h->nodes[cons[proj_id][0]];
+            fp::launch_fold_weights(d_weights + pr.w_off, d_bn + pb.bn_off, pr.K, pr.C, 1, 1, h->eps, f.d_w32, f.C, 1, 1,
+                                    0, Kw, 0, 0, st);
+            fp::launch_fold_bias(d_bn + pb.bn_off, pr.K, h->eps, f.d_b32, 0, 1, st);
+            h->conv_to_fused[conv_number[proj_id]] = -1;
+        }
+        node_tensor[relu_id] = h->convs[ci].out;
+        return FP_OK;
+    }
+
     fp_status handle_add(int id) {
         const fp_node& n = h->nodes[id];
         if (cons[id].size() != 1 || h->nodes[cons[id][0]].op != FP_RELU)
@@ -303,6 +373,10 @@ struct Builder {
                 return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion needs a two-convolution block", id);
             const int f1i = h->ops[p1].idx;
             const FConv f1c = h->convs[f1i];
+            if (c2.R == 1 && c2.S == 1) {
+                TRY(fuse_bottleneck(id, relu_id, conv2_id, f1i, x_tid, h_tid, mode, proj_id));
+                return FP_OK;
+            }
             if (f1c.src != x_tid || !f1c.relu || f1c.res_mode != 0 || f1c.role != 0 || f1c.R != 3 || f1c.S != 3 ||
                 f1c.pad != 1 || c2.R != 3 || c2.S != 3 || c2.stride != 1 || c2.pad != 1)
                 return fail(FP_ERR_UNSUPPORTED, "node %d: aggressive fusion supports 3x3 two-convolution blocks only", id);

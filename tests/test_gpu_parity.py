@@ -205,6 +205,34 @@ def test_tiny_bottleneck(B, fpo, compute):
         g.close()
 
 
+@pytest.mark.parametrize("compute", ["fp32", "tc"])
+def test_tiny_bottleneck_aggressive(B, fpo, compute):
+    """Three-convolution blocks fused the paper's way: the pass-through rides through 1x1 - 3x3 - 1x1, no add."""
+    w = wl.tiny_bottleneck(aggressive=True)
+    mode = B.FP_COMPUTE_FP32 if compute == "fp32" else B.FP_COMPUTE_BF16_TC
+    tol = TOL_FP32 if compute == "fp32" else TOL_BF16
+    g = Gpu(B, w, mode, keep_outputs=1)
+    try:
+        assert all(o.res_mode == 0 for o in B.op_infos(g.h)), "an add survived"
+        assert err(g.forward(w.x), fpo.unfused_forward(w.net, w.weights, w.bn, w.x)) < tol
+        zeros = np.zeros(w.net.n_convs())
+        B.fp_prune(g.h, zeros)                       # fused operators go back to their original filter counts
+        gp, masks, ranks, _ = fpo.pruned_model(w.net, w.weights, w.bn, zeros)
+        for ci, (m, r) in B.masks_and_ranks(g.h).items():
+            if masks[ci] is None:
+                assert m is None
+            else:
+                np.testing.assert_array_equal(m, masks[ci])
+                np.testing.assert_array_equal(r, ranks[ci])
+        got = g.forward(w.x)
+        ref = fpo.fused_forward(gp, w.x)
+        if not err(got, ref) < tol:
+            _compare_ops(B, g, w, gp, fpo, tol)
+        assert err(got, ref) < tol
+    finally:
+        g.close()
+
+
 def test_per_operator_outputs_tc(B, fpo):
     """Every fused operator's activation, not only the logits (several tiles, ragged tails)."""
     w = wl.tiny_cifar(widths=(16, 32, 64), in_hw=20, batch=3, n_per_stage=2, p=0.3)
@@ -294,12 +322,10 @@ def test_error_codes(B):
         assert e.value.status == B.FP_ERR_ARG
     finally:
         B.fp_destroy(h)
-    # aggressive fusion of a bottleneck block is not supported
-    wb = wl.tiny_bottleneck()
+    # a valid description the kernels cannot run: images wider than 512 pixels
+    wb = wl.tiny_cifar()
     net = copy.deepcopy(wb.net)
-    for n in net.nodes:
-        if n["block_id"] >= 0:
-            n["aggressive"] = 1
+    net.in_W = 600
     with pytest.raises(B.FpError) as e:
         B.fp_fuse(net, to_dev(wb.weights), to_dev(wb.bn), 2, B.FP_COMPUTE_FP32)
     assert e.value.status == B.FP_ERR_UNSUPPORTED
