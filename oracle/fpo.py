@@ -39,7 +39,7 @@ import subprocess
 
 import numpy as np
 
-OP_CONV, OP_BN, OP_RELU, OP_ADD, OP_SHORTCUT_A, OP_MAXPOOL, OP_GAVGPOOL, OP_FC = range(8)
+OP_CONV, OP_BN, OP_RELU, OP_ADD, OP_SHORTCUT_A, OP_MAXPOOL, OP_GAVGPOOL, OP_FC, OP_CONCAT = range(9)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
@@ -204,6 +204,8 @@ def unfused_forward(net, weights, bn, x, return_all=False):
             v = relu(a)
         elif op == OP_ADD:
             v = add(a, vals[n["in1"]])
+        elif op == OP_CONCAT:
+            v = np.concatenate([a, vals[n["in1"]]], axis=1)
         elif op == OP_SHORTCUT_A:
             v = shortcut_a(a, n["K"], n["stride"], n["pad_lo"])
         elif op == OP_MAXPOOL:
@@ -279,7 +281,7 @@ def _consumer_map(net):
     cons = {i: [] for i in range(-1, len(net.nodes))}
     for i, n in enumerate(net.nodes):
         cons[n["in0"]].append(i)
-        if n["op"] == OP_ADD:
+        if n["op"] in (OP_ADD, OP_CONCAT):
             cons[n["in1"]].append(i)
     return cons
 
@@ -352,7 +354,24 @@ def fuse(net, weights, bn, precision="f64"):
         if op == OP_CONV:
             W, b, bn_id = folded(i)
             nxt = cons[bn_id]
-            if len(nxt) == 1 and nodes[nxt[0]]["op"] == OP_RELU:
+            # the concatenation structure (Sec. IV-B.1): y = concat(conv(x), x) becomes one convolution with the
+            # identity filters of xconv-C stacked under W: y = new_conv(x, [W ; I])
+            last = nxt[0] if (len(nxt) == 1 and nodes[nxt[0]]["op"] == OP_RELU) else bn_id
+            cc = cons[last]
+            if len(cc) == 1 and nodes[cc[0]]["op"] == OP_CONCAT and nodes[cc[0]]["in0"] == last \
+                    and nodes[cc[0]]["in1"] == n["in0"]:
+                K, C, R, S = W.shape
+                if n["stride"] != 1 or R != S or R % 2 == 0 or n["pad"] != R // 2:
+                    raise ValueError("the concatenation structure needs a stride-1 'same' convolution")
+                relu_flag = last != bn_id
+                xp = producer.get(tensor_of[n["in0"]])
+                if relu_flag and (xp is None or (xp["kind"] == "conv" and not xp["relu"])):
+                    raise ValueError("fusing concat(relu(conv(x)), x) needs x to be a ReLU output")
+                Wc = np.concatenate([W, _identity_filters(C, C, R, S, 0, dt)], axis=0)
+                bc = np.concatenate([b, np.zeros(C, dtype=dt)])
+                o = emit_conv(i, Wc, bc, tensor_of[n["in0"]], relu_flag, None, role="aggr1", n_orig=K)
+                tensor_of[cc[0]] = o["out"]
+            elif len(nxt) == 1 and nodes[nxt[0]]["op"] == OP_RELU:
                 o = emit_conv(i, W, b, tensor_of[n["in0"]], True, None)
                 tensor_of[nxt[0]] = o["out"]
             elif len(nxt) == 1 and nodes[nxt[0]]["op"] == OP_ADD:
@@ -480,7 +499,7 @@ def fuse(net, weights, bn, precision="f64"):
             o = dict(kind="head", src=tensor_of[n["in0"]], Wfc=Wfc, bfc=bfc, out=new_tid())
             g.ops.append(o)
             producer[o["out"]] = o
-        elif op in (OP_BN, OP_RELU, OP_SHORTCUT_A, OP_FC):
+        elif op in (OP_BN, OP_RELU, OP_SHORTCUT_A, OP_FC, OP_CONCAT):
             pass  # consumed by the patterns above
         else:
             raise ValueError(f"unknown op {op}")

@@ -26,8 +26,8 @@ from __future__ import annotations
 
 import numpy as np
 
-OP_CONV, OP_BN, OP_RELU, OP_ADD, OP_SHORTCUT_A, OP_MAXPOOL, OP_GAVGPOOL, OP_FC = range(8)
-OP_NAMES = ["conv", "bn", "relu", "add", "shortcut_a", "maxpool", "gavgpool", "fc"]
+OP_CONV, OP_BN, OP_RELU, OP_ADD, OP_SHORTCUT_A, OP_MAXPOOL, OP_GAVGPOOL, OP_FC, OP_CONCAT = range(9)
+OP_NAMES = ["conv", "bn", "relu", "add", "shortcut_a", "maxpool", "gavgpool", "fc", "concat"]
 
 BASE_SEED = 20201016
 
@@ -70,6 +70,11 @@ class Net:
     def shortcut_a(self, src, C, K, stride, pad_lo=0, block=-1, aggressive=0):
         return self._add(op=OP_SHORTCUT_A, in0=src, C=C, K=K, stride=stride, pad_lo=pad_lo,
                          block_id=block, aggressive=aggressive)
+
+    def concat(self, a, b, Ka, Cb):
+        """Channel concatenation [a ; b]: a = the (BN / ReLU of a) convolution's output with Ka channels, b = that
+        convolution's input with Cb channels (the concatenation structure of Sec. IV-B.1)."""
+        return self._add(op=OP_CONCAT, in0=a, in1=b, K=Ka + Cb, C=Cb)
 
     def maxpool(self, src, C, R=3, stride=2, pad=1):
         return self._add(op=OP_MAXPOOL, in0=src, K=C, C=C, R=R, S=R, stride=stride, pad=pad)
@@ -346,6 +351,25 @@ def tiny_imagenet_basic(layers=(1, 1, 1), widths=(8, 12, 20), in_hw=32, batch=2,
     net = resnet_imagenet_basic(layers, widths, in_hw, n_classes=7, aggressive=aggressive,
                                 name="tiny_imagenet_basic", stem_k=stem_k)
     return Workload("tiny_imagenet_basic", net, batch, seed, False, uniform_ratios(p), f"uniform {p}")
+
+
+def concat_net(growth=(6, 10, 5), stem=8, in_hw=12, n_classes=4, name="concat_net"):
+    """A small network of concatenation structures (DenseNet-like growth): x <- concat(relu(bn(conv3x3(x))), x)."""
+    net = Net(3, in_hw, in_hw, name)
+    x = net.relu(net.bn(net.conv(-1, stem, 3, 3, 1, 1), stem))
+    C = stem
+    for g in growth:
+        h = net.relu(net.bn(net.conv(x, g, C, 3, 1, 1), g))
+        x = net.concat(h, x, g, C)
+        C += g
+    x = net.gavgpool(x, C)
+    net.fc(x, n_classes, C)
+    net.n_blocks = 0
+    return net
+
+
+def tiny_concat(batch=3, seed=19, p=0.0, **kw):
+    return Workload("tiny_concat", concat_net(**kw), batch, seed, False, uniform_ratios(p), f"uniform {p}")
 
 
 def tiny_bottleneck(layers=(1, 2), widths=(4, 8), in_hw=32, batch=2, seed=13, p=0.0, aggressive=False):

@@ -399,3 +399,39 @@ def test_aggressive_bottleneck_loses_n_minus_m(fpo):
     a = fpo.fused_forward(fpo.prune_remove(g, masks), w.x)
     b = fpo.fused_forward(fpo.prune_zero(g, masks), w.x)
     assert np.abs(a - b).max() <= 1e-12 * max(np.abs(b).max(), 1.0)
+
+
+# ------------------------------------------------------------------------------------------
+# the concatenation structure (Sec. IV-B.1): y = concat(conv(x), x)  ->  new_conv(x, [W ; I])
+# ------------------------------------------------------------------------------------------
+
+def test_concat_structure_fused_equals_unfused(fpo):
+    w = wl.tiny_concat()
+    g = fpo.fuse(w.net, w.weights, w.bn)
+    convs = [op for op in g.ops if op["kind"] == "conv"]
+    assert [op["W"].shape[0] for op in convs] == [8, 6 + 8, 10 + 14, 5 + 24]       # filters: own + pass-through
+    assert len(g.ops) == 5                                                          # 4 convolutions + head: no concat left
+    ref = fpo.unfused_forward(w.net, w.weights, w.bn, w.x)
+    got = fpo.fused_forward(g, w.x)
+    assert np.abs(got - ref).max() <= 1e-12 * np.abs(ref).max()
+
+
+def test_concat_identity_filters_reproduce_the_input(fpo):
+    """x = xconv(x, W~): the stacked identity filters alone return the block input, channel for channel."""
+    rng = np.random.default_rng(2)
+    x = np.abs(rng.standard_normal((2, 5, 6, 7)))
+    Wt = fpo._identity_filters(5, 5, 3, 3)
+    np.testing.assert_array_equal(fpo.conv2d(x, Wt, 1, 1), x)
+
+
+def test_concat_structure_conservative_pruning(fpo):
+    """A fused concatenation operator has n = K + C filters and m = K originally: it loses n - m."""
+    w = wl.tiny_concat()
+    g32 = fpo.fuse(w.net, w.weights, w.bn, "f32")
+    masks, _, _ = fpo.select_masks(g32, np.zeros(w.net.n_convs()), fpo.NORM_L1)
+    kept = [int(masks[ci].sum()) for ci in sorted(masks)]
+    assert kept == [8, 6, 10, 5]
+    g = fpo.fuse(w.net, w.weights, w.bn)
+    a = fpo.fused_forward(fpo.prune_remove(g, masks), w.x)
+    b = fpo.fused_forward(fpo.prune_zero(g, masks), w.x)
+    assert np.abs(a - b).max() <= 1e-12 * max(np.abs(b).max(), 1.0)
