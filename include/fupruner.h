@@ -59,7 +59,11 @@ typedef enum {
                            with `pad_lo` zero channels before and K-C-pad_lo after the copy     */
     FP_MAXPOOL = 5,     /* R x R window, stride, pad; padded positions never win                */
     FP_GAVGPOOL = 6,    /* mean over all spatial positions                                      */
-    FP_FC = 7           /* K x C matrix + K bias                                                */
+    FP_FC = 7,          /* K x C matrix + K bias                                                */
+    FP_CONCAT = 8       /* channel concatenation [in0 ; in1] of the concatenation structure of Sec. IV-B.1:
+                           in0 = the BN (or ReLU) of a stride-1 "same" convolution with K - C filters, in1 =
+                           that convolution's input with C channels.  Always fused: the convolution gets C
+                           identity filters (the auxiliary convolution xconv-C) and no concatenation remains */
 } fp_op;
 
 typedef struct {

@@ -245,6 +245,26 @@ struct Builder {
         return FP_OK;
     }
 
+    // K_id identity filters (the auxiliary convolution xconv-C) under the filters of fused convolution `fi`:
+    // its output becomes [conv(x) ; x].  The operator is then a fused one: n = K + K_id filters, m = K originally.
+    fp_status stack_identity_filters(int fi, int K_id) {
+        const FConv f0 = h->convs[fi];
+        const int K1 = f0.K, C = f0.C, RS = f0.R * f0.S;
+        float *nw, *nb;
+        const size_t cnt = (size_t)(K1 + K_id) * C * RS;
+        TRY(dev_alloc(h->fixed_buffers, (void**)&nw, cnt * sizeof(float)));
+        TRY(dev_alloc(h->fixed_buffers, (void**)&nb, (size_t)(K1 + K_id) * sizeof(float)));
+        CK(cudaMemsetAsync(nw, 0, cnt * sizeof(float), st));
+        CK(cudaMemsetAsync(nb, 0, (size_t)(K1 + K_id) * sizeof(float), st));
+        CK(cudaMemcpyAsync(nw, f0.d_w32, (size_t)K1 * C * RS * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        CK(cudaMemcpyAsync(nb, f0.d_b32, (size_t)K1 * sizeof(float), cudaMemcpyDeviceToDevice, st));
+        fp::launch_identity_filters(nw, C, f0.R, f0.S, K1, 0, K_id, C, 0, st);
+        FConv& f = h->convs[fi];
+        f.d_w32 = nw; f.d_b32 = nb; f.K = K1 + K_id; f.role = 1;
+        h->tensors[f.out].C_full = K1 + K_id;
+        return FP_OK;
+    }
+
     bool is_relu_output(int tid) const {
         const int px = h->tensors[tid].producer;
         if (px < 0) return false;
@@ -443,11 +463,12 @@ struct Builder {
         int nc = 0;
         for (int i = 0; i < nn; ++i) {
             const fp_node& n = h->nodes[i];
-            if (n.op < FP_CONV || n.op > FP_FC) return fail(FP_ERR_DESC, "node %d: unknown op %d", i, n.op);
+            if (n.op < FP_CONV || n.op > FP_CONCAT) return fail(FP_ERR_DESC, "node %d: unknown op %d", i, n.op);
             if (n.in0 < -1 || n.in0 >= i) return fail(FP_ERR_DESC, "node %d: in0 must name an earlier node", i);
-            if (n.op == FP_ADD && (n.in1 < -1 || n.in1 >= i)) return fail(FP_ERR_DESC, "node %d: in1 must name an earlier node", i);
+            const bool two = n.op == FP_ADD || n.op == FP_CONCAT;
+            if (two && (n.in1 < -1 || n.in1 >= i)) return fail(FP_ERR_DESC, "node %d: in1 must name an earlier node", i);
             if (n.in0 >= 0) cons[n.in0].push_back(i);
-            if (n.op == FP_ADD && n.in1 >= 0) cons[n.in1].push_back(i);
+            if (two && n.in1 >= 0) cons[n.in1].push_back(i);
             if (n.op == FP_CONV) conv_number[i] = nc++;
         }
         h->n_desc_convs = nc;
@@ -467,7 +488,24 @@ struct Builder {
                     const int src = tensor_of(n.in0);
                     if (src < 0) return fail(FP_ERR_DESC, "node %d: input is not a materialised tensor", i);
                     int ci;
-                    if (nxt.size() == 1 && h->nodes[nxt[0]].op == FP_RELU) {
+                    // The concatenation structure (Sec. IV-B.1): y = concat(conv(x), x) becomes one convolution with
+                    // the identity filters of xconv-C stacked under its own: y = new_conv(x, [W' ; I]).
+                    const bool has_relu = nxt.size() == 1 && h->nodes[nxt[0]].op == FP_RELU;
+                    const int last = has_relu ? nxt[0] : bn_id;
+                    if (cons[last].size() == 1 && h->nodes[cons[last][0]].op == FP_CONCAT &&
+                        h->nodes[cons[last][0]].in0 == last && h->nodes[cons[last][0]].in1 == n.in0) {
+                        const int cat = cons[last][0];
+                        if (n.stride != 1 || n.R != n.S || n.R % 2 == 0 || n.pad != n.R / 2)
+                            return fail(FP_ERR_UNSUPPORTED, "node %d: the concatenation structure needs a stride-1 'same' convolution", i);
+                        if (has_relu && !is_relu_output(src))
+                            return fail(FP_ERR_UNSUPPORTED, "node %d: fusing concat(relu(conv(x)), x) needs x to be a ReLU output", i);
+                        if (h->nodes[cat].K != n.K + n.C) return fail(FP_ERR_SHAPE, "node %d: concatenation has %d channels, operands %d", cat, h->nodes[cat].K, n.K + n.C);
+                        TRY(emit_conv(i, src, has_relu ? 1 : 0, 0, &ci));
+                        TRY(stack_identity_filters(ci, n.C));
+                        node_tensor[cat] = h->convs[ci].out;
+                        break;
+                    }
+                    if (has_relu) {
                         TRY(emit_conv(i, src, 1, 0, &ci));
                         node_tensor[nxt[0]] = h->convs[ci].out;
                     } else {

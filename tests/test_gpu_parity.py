@@ -233,6 +233,32 @@ def test_tiny_bottleneck_aggressive(B, fpo, compute):
         g.close()
 
 
+@pytest.mark.parametrize("compute", ["fp32", "tc"])
+def test_concat_structures(B, fpo, compute):
+    """y = concat(conv(x), x) (Sec. IV-B.1) runs as one convolution with identity filters; pruned back by n - m."""
+    w = wl.tiny_concat()
+    mode = B.FP_COMPUTE_FP32 if compute == "fp32" else B.FP_COMPUTE_BF16_TC
+    tol = TOL_FP32 if compute == "fp32" else TOL_BF16
+    g = Gpu(B, w, mode, keep_outputs=1)
+    try:
+        infos = [o for o in B.op_infos(g.h) if o.kind == 0]
+        assert [o.K for o in infos] == [8, 14, 24, 29]
+        assert err(g.forward(w.x), fpo.unfused_forward(w.net, w.weights, w.bn, w.x)) < tol
+        zeros = np.zeros(w.net.n_convs())
+        B.fp_prune(g.h, zeros)
+        gp, masks, ranks, _ = fpo.pruned_model(w.net, w.weights, w.bn, zeros)
+        for ci, (m, r) in B.masks_and_ranks(g.h).items():
+            np.testing.assert_array_equal(m, masks[ci])
+            np.testing.assert_array_equal(r, ranks[ci])
+        got = g.forward(w.x)
+        ref = fpo.fused_forward(gp, w.x)
+        if not err(got, ref) < tol:
+            _compare_ops(B, g, w, gp, fpo, tol)
+        assert err(got, ref) < tol
+    finally:
+        g.close()
+
+
 def test_per_operator_outputs_tc(B, fpo):
     """Every fused operator's activation, not only the logits (several tiles, ragged tails)."""
     w = wl.tiny_cifar(widths=(16, 32, 64), in_hw=20, batch=3, n_per_stage=2, p=0.3)
