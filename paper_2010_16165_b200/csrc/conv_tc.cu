@@ -59,6 +59,7 @@ struct TcParams {
     int tpk, kblocks;                   // gather: taps per K block, K blocks per tile
     int tps;                            // streamed filters: 128-position tiles per pipeline step (share each filter block)
     int a_stage_bytes, b_stage_bytes, b_bank_bytes;
+    int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
     int* status;
 };
 
@@ -235,7 +236,8 @@ conv_tc_kernel(const TcParams p) {
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
     const uint32_t ctrl_addr = smem_u32(smem_raw);
     float* bias_s = reinterpret_cast<float*>(smem_raw + sizeof(Ctrl));            // K_pad floats
-    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + (uint32_t)p.a.K_pad * 4u + 1023u) & ~1023u;
+    int2* lut = reinterpret_cast<int2*>(smem_raw + sizeof(Ctrl) + (size_t)p.a.K_pad * 4u);   // gather mode only
+    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + (uint32_t)p.a.K_pad * 4u + (uint32_t)p.lut_bytes + 1023u) & ~1023u;
     const uint32_t b_region = MODE == MODE_FLAT_RESIDENT ? (uint32_t)p.b_bank_bytes
                               : MODE == MODE_FLAT_STREAM ? (uint32_t)(p.b_stages * p.b_stage_bytes) : 0u;
     const uint32_t a_base = b_base + ((b_region + 127u) & ~127u);
@@ -265,6 +267,21 @@ conv_tc_kernel(const TcParams p) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     for (int i = threadIdx.x; i < p.a.K_pad; i += blockDim.x) bias_s[i] = p.a.bias[i];   // filters' data: safe before the dependency wait
+    if (MODE == MODE_GATHER) {
+        // Plane i of K block kb holds channel chunk c of tap (r, s): its offset from the tile's first tap, in
+        // 16-byte vectors, and r, s, "in use" and the block's plane count, are the same for every tile.
+        for (int e = threadIdx.x; e < p.kblocks * 8; e += blockDim.x) {
+            const int kb = e >> 3, i = e & 7;
+            int tap0, g, ntap, cgg;
+            if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
+            else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
+            const int planes = ntap * cgg;
+            const int tt = i / cgg, c = i - tt * cgg;
+            const int tap = tap0 + tt, r = tap / p.a.S, sx = tap - r * p.a.S;
+            lut[e] = i < planes ? make_int2((g * p.cg + c) * (int)p.plane_in + r * p.Wp_in + sx, r | (sx << 8) | (1 << 16) | (planes << 24))
+                                : make_int2(0, planes << 24);
+        }
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_base)), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -636,28 +653,26 @@ conv_tc_kernel(const TcParams p) {
             const int hp = (int)fdiv((uint32_t)rem, p.div_qp), wq = rem - hp * p.Qp;
             const bool interior = f < p.m_total && hp >= 1 && hp <= p.a.P && wq >= 1 && wq <= p.a.Q;
             const int ih0 = (hp - 1) * p.a.stride - p.a.pad, iw0 = (wq - 1) * p.a.stride - p.a.pad;
+            const long long base = (long long)n * p.P2_in + (long long)(ih0 + 1) * p.Wp_in + (iw0 + 1);
+            uint32_t rmask = 0, smask = 0;       // filter rows / columns that fall inside the image
+            if (interior) {
+                for (int r = 0; r < p.a.R; ++r) rmask |= (uint32_t)(ih0 + r >= 0 && ih0 + r < p.a.H) << r;
+                for (int sx = 0; sx < p.a.S; ++sx) smask |= (uint32_t)(iw0 + sx >= 0 && iw0 + sx < p.a.W) << sx;
+            }
             for (int kb = 0; kb < p.kblocks && ok; ++kb) {
-                int tap0, g, ntap, cgg;
-                if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
-                else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
+                // the eight loads have separate destinations, so all of them are in flight together
                 uint4 v[8];
+                const int2* L = lut + kb * 8;
+                const int planes = L[0].y >> 24;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = make_uint4(0, 0, 0, 0);
-                int r = tap0 / p.a.S, s = tap0 - r * p.a.S;
-                for (int tt = 0; tt < ntap; ++tt) {
-                    const int ih = ih0 + r, iw = iw0 + s;
-                    const bool valid = interior && ih >= 0 && ih < p.a.H && iw >= 0 && iw < p.a.W;
-                    const long long src = (long long)n * p.P2_in + (long long)(ih + 1) * p.Wp_in + (iw + 1);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int c = i - tt * cgg;          // plane i holds chunk c of tap tap0+tt
-                        if (valid && c >= 0 && c < cgg) v[i] = __ldg(xv + (long long)(g * p.cg + c) * p.plane_in + src);
-                    }
-                    if (++s == p.a.S) { s = 0; ++r; }
+                for (int i = 0; i < 8; ++i) {
+                    const int2 e = L[i];
+                    const bool valid = ((e.y >> 16) & (rmask >> (e.y & 0xff)) & (smask >> ((e.y >> 8) & 0xff)) & 1) != 0;
+                    v[i] = make_uint4(0, 0, 0, 0);
+                    if (valid) v[i] = __ldg(xv + base + e.x);
                 }
                 if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
                 uint8_t* dst = smem_raw + (a_base - ctrl_addr) + stage * stage_bytes + m * 16;
-                const int planes = ntap * cgg;
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (i < planes) *reinterpret_cast<uint4*>(dst + i * 128 * 16) = v[i];
@@ -775,11 +790,21 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         if (plan->tpk < 1) plan->tpk = 1;
         const int planes = plan->groups > 1 ? plan->cg : plan->tpk * cchunks;
         const unsigned stage = (unsigned)(planes * 128 * 16 + planes * n_tile * 16);
-        plan->a_stages = 6;
-        while (plan->a_stages > 2 && smem + plan->a_stages * stage > 120 * 1024) --plan->a_stages;
+        if ((long long)a.N * (a.H + 2) * (a.W + 2) * cchunks >= (1ll << 31)) { snprintf(err, err_len, "input of more than 2^31 vectors"); return 1; }
+        const int kblocks = plan->groups > 1 ? taps * plan->groups : (taps + plan->tpk - 1) / plan->tpk;
+        smem += (unsigned)kblocks * 64u;                 // the plane-offset table
+        // The loader threads wait out one load latency per K block, so co-resident CTAs are what hides it:
+        // four CTAs with two or three stages each where they fit, else two CTAs with up to six stages.
+        plan->a_stages = 3;
+        want_ctas = 4;
+        while (plan->a_stages > 2 && smem + plan->a_stages * stage > 56 * 1024) --plan->a_stages;
+        if (smem + plan->a_stages * stage > 56 * 1024) {
+            plan->a_stages = 6;
+            want_ctas = 2;
+            while (plan->a_stages > 2 && smem + plan->a_stages * stage > 120 * 1024) --plan->a_stages;
+        }
         plan->b_stages = plan->a_stages;
         smem += plan->a_stages * stage;
-        want_ctas = 2;
     }
     if (plan->tps < 1) plan->tps = 1;
     plan->tmem_cols = pow2_at_least(2 * plan->tps * n_tile < 32 ? 32 : 2 * plan->tps * n_tile);
@@ -843,6 +868,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.tpk = plan.tpk > 0 ? plan.tpk : 1;
     p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
     p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
+    p.lut_bytes = plan.flat ? 0 : p.kblocks * 64;
     p.status = d_status;
     p.div_ntiles = make_fastdiv((uint32_t)plan.n_tiles);
     p.div_p2out = make_fastdiv((uint32_t)p.P2_out);
