@@ -794,7 +794,8 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         const int kblocks = plan->groups > 1 ? taps * plan->groups : (taps + plan->tpk - 1) / plan->tpk;
         smem += (unsigned)kblocks * 64u;                 // the plane-offset table
         // The loader threads wait out one load latency per K block, so co-resident CTAs are what hides it:
-        // four CTAs with two or three stages each where they fit, else two CTAs with up to six stages.
+        // small stages leave shared memory for up to four CTAs with two or three stages each (the register
+        // count below decides how many really fit), large ones get two CTAs with up to six stages.
         plan->a_stages = 3;
         want_ctas = 4;
         while (plan->a_stages > 2 && smem + plan->a_stages * stage > 56 * 1024) --plan->a_stages;
