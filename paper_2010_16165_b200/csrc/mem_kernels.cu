@@ -176,6 +176,71 @@ __global__ void maxpool_kernel(const void* __restrict__ x, void* __restrict__ y,
     }
 }
 
+// 3x3 / stride-2 / pad-1 max pooling of bf16 activations, the ImageNet stem's pooling.  The generic kernel above
+// issues nine 16-byte loads per output whose addresses are 32 bytes apart between neighbouring threads (eight
+// cache lines per warp-wide load), and the L1 pipeline, not DRAM, bounds it.  Here a warp that owns 32 neighbouring
+// outputs reads the 64 input columns under them with two fully coalesced loads per input row (lane l holds
+// columns 2*q0 + l and 2*q0 + 32 + l; lane 0 also fetches column 2*q0 - 1), takes the maximum down the three rows
+// first, then across each window of three columns with warp shuffles.  The maximum of bf16 values is one of them,
+// so packed bf16 compares give the same result as fp32 ones.  Same block shape as the generic kernel.
+__device__ __forceinline__ Vec8h vmax(const Vec8h& a, const Vec8h& b) {
+    Vec8h r;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r.v[i] = __hmax2(a.v[i], b.v[i]);
+    return r;
+}
+__device__ __forceinline__ Vec8h vshfl(const Vec8h& a, int src_lane) {
+    Vec8h r;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t w = __shfl_sync(0xffffffffu, *reinterpret_cast<const uint32_t*>(&a.v[i]), src_lane);
+        r.v[i] = *reinterpret_cast<const __nv_bfloat162*>(&w);
+    }
+    return r;
+}
+__global__ void maxpool3s2_bf16_kernel(const Vec8h* __restrict__ x, Vec8h* __restrict__ y, int N, int H, int W, int chunks,
+                                       int P, int Q) {
+    const int Wp = W + 2, P2i = (H + 2) * Wp, Qp = Q + 2, P2o = (P + 2) * Qp;
+    const int rows_per_image = P + 2;
+    const int row = blockIdx.x * blockDim.y + threadIdx.y;
+    if (row >= chunks * N * rows_per_image) return;                           // the same for a whole warp
+    const int jn = row / rows_per_image, pp = row - jn * rows_per_image;     // jn = chunk * N + image
+    const int p = pp - 1;
+    const size_t in_base = (size_t)jn * P2i, out_base = (size_t)jn * P2o + (size_t)pp * Qp;
+    const int lane = threadIdx.x & 31;
+    Vec8h ninf, zero;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { ninf.v[i] = __floats2bfloat162_rn(-INFINITY, -INFINITY); zero.v[i] = __floats2bfloat162_rn(0.0f, 0.0f); }
+    for (int qq0 = threadIdx.x - lane; qq0 < Qp; qq0 += blockDim.x) {         // warp-uniform: all 32 lanes take part
+        const int qq = qq0 + lane, q = qq - 1;
+        if (p < 0 || p >= P) {                                                // border row: zeros
+            if (qq < Qp) y[out_base + qq] = zero;
+            continue;
+        }
+        const int c0 = 2 * (qq0 - 1);                  // input column under the warp's first output
+        const int ca = c0 + lane, cb = c0 + 32 + lane, ce = c0 - 1;
+        Vec8h A = ninf, B = ninf, E = ninf;
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const int ih = 2 * p - 1 + r;
+            if (ih < 0 || ih >= H) continue;
+            const Vec8h* src = x + in_base + (size_t)(ih + 1) * Wp + 1;
+            if (ca >= 0 && ca < W) A = vmax(A, src[ca]);
+            if (cb >= 0 && cb < W) B = vmax(B, src[cb]);
+            if (lane == 0 && ce >= 0 && ce < W) E = vmax(E, src[ce]);
+        }
+        // windows centred on the even lanes: W_A[l] = max(A[l-1], A[l], A[l+1]) with A[-1] = E; W_B alike with B[-1] = A[31]
+        Vec8h upA = vshfl(A, (lane + 31) & 31), dnA = vshfl(A, (lane + 1) & 31);
+        Vec8h upB = vshfl(B, (lane + 31) & 31), dnB = vshfl(B, (lane + 1) & 31);
+        const Vec8h a31 = upA;                          // on lane 0 the rotation delivered A[31]
+        if (lane == 0) { upA = E; upB = a31; }
+        const Vec8h WA = vmax(vmax(upA, A), dnA), WB = vmax(vmax(upB, B), dnB);
+        // output j of the warp sits over columns 2j-1 .. 2j+1: window 2j of A (j < 16) or 2j-32 of B
+        const Vec8h fa = vshfl(WA, (2 * lane) & 31), fb = vshfl(WB, (2 * lane) & 31);
+        if (qq < Qp) y[out_base + qq] = (q >= 0 && q < Q) ? (lane < 16 ? fa : fb) : zero;
+    }
+}
+
 // Head, step 1: spatial sum per channel in fp32.  One warp per (image, chunk of 8 channels): lanes
 // stride over the interior positions with 16-byte loads, shuffle-reduce, and write 8 sums.
 template <bool BF16>
@@ -297,7 +362,9 @@ void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, in
     const int tx = Q + 2 <= 32 ? 32 : Q + 2 <= 64 ? 64 : 128, ty = 256 / tx;
     const int rows = (C_pad / 8) * N * (P + 2);
     const dim3 block(tx, ty), grid((rows + ty - 1) / ty);
-    if (is_bf16) maxpool_kernel<true><<<grid, block, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
+    if (is_bf16 && R == 3 && stride == 2 && pad == 1)
+        maxpool3s2_bf16_kernel<<<grid, block, 0, st>>>((const Vec8h*)x, (Vec8h*)y, N, H, W, C_pad / 8, P, Q);
+    else if (is_bf16) maxpool_kernel<true><<<grid, block, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
     else maxpool_kernel<false><<<grid, block, 0, st>>>(x, y, N, H, W, C_pad / 8, P, Q, R, stride, pad);
 }
 
