@@ -138,6 +138,66 @@ __global__ void input_to_stem_planar_kernel(const void* __restrict__ in, int in_
     }
 }
 
+// The same packing for exactly three input channels (RGB): with C fixed, tap s and channel c of packed channel j
+// are compile-time constants, so a vector is eight shared-memory loads at immediate offsets (no table, no
+// divisions), and the rows are staged row by row.  One thread per output column.
+__global__ void input_to_stem_planar_rgb_kernel(const void* __restrict__ in, int in_is_bf16, __nv_bfloat16* __restrict__ out,
+                                                int N, int H, int W) {
+    constexpr int C = 3;
+    extern __shared__ float rows[];                  // [3 rows: 2p-1, 2p, 2p+1][C][W + 6], zero where outside the image
+    const int P = H / 2, Q = W / 2, Qp = Q + 2, P2 = (P + 2) * Qp;
+    const int n = blockIdx.x / (P + 2), pp = blockIdx.x - n * (P + 2);
+    const int p = pp - 1;
+    const size_t plane = (size_t)N * P2;
+    Vec8h* outv = reinterpret_cast<Vec8h*>(out) + (size_t)n * P2 + (size_t)pp * Qp;
+    Vec8h zero;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) zero.v[e] = __floats2bfloat162_rn(0.0f, 0.0f);
+    if (p < 0 || p >= P) {                           // border row: zeros in every chunk
+        for (int j8 = 0; j8 < 10; ++j8)
+            for (int qq = threadIdx.x; qq < Qp; qq += blockDim.x) outv[(size_t)j8 * plane + qq] = zero;
+        return;
+    }
+    const int Ws = W + 6;
+    for (int rc = 0; rc < 3 * C; ++rc) {
+        const int r = rc / C, c = rc - r * C;
+        const int ih = 2 * p - 1 + r;
+        const bool row_in = ih >= 0 && ih < H;
+        const size_t src = (((size_t)n * C + c) * H + (row_in ? ih : 0)) * W;
+        for (int col = threadIdx.x; col < Ws; col += blockDim.x) {
+            const int iw = col - 3;
+            float v = 0.0f;
+            if (row_in && iw >= 0 && iw < W)
+                v = in_is_bf16 ? __bfloat162float(((const __nv_bfloat16*)in)[src + iw]) : ((const float*)in)[src + iw];
+            rows[rc * Ws + col] = v;
+        }
+    }
+    __syncthreads();
+    for (int qq = threadIdx.x; qq < Qp; qq += blockDim.x) {
+        const int q = qq - 1;
+        const bool inside = q >= 0 && q < Q;
+#pragma unroll
+        for (int group = 0; group < 3; ++group) {    // 0 = E (row 2p), 1 = O' (row 2p-1), 2 = O (row 2p+1)
+            const int r = group == 0 ? 1 : group == 1 ? 0 : 2;
+            const float* base = rows + r * C * Ws + (inside ? 2 * q : 0);    // input column 2q + s - 3 sits at 2q + s
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int j = k * 8 + e, sx = j / C, c = j - sx * C;     // constants after unrolling
+                    v[e] = (sx < 7 && inside) ? base[c * Ws + sx] : 0.0f;
+                }
+                Vec8h o;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o.v[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                outv[(size_t)(group * 3 + k) * plane + qq] = o;
+            }
+        }
+        outv[(size_t)9 * plane + qq] = zero;
+    }
+}
+
 // Max pooling; padded positions never win.  Output border positions are written as zeros.
 // blockIdx.x = (chunk, image, output row incl. borders), threads run along the row: no divisions per element,
 // 32-bit arithmetic, and a warp reads runs of neighbouring vectors.
@@ -353,7 +413,8 @@ void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_i
 
 void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, cudaStream_t st) {
     const size_t smem = (size_t)3 * C * (W + 6) * sizeof(float);      // <= 36 KB for the supported widths
-    input_to_stem_planar_kernel<<<N * (H / 2 + 2), 256, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W);
+    if (C == 3) input_to_stem_planar_rgb_kernel<<<N * (H / 2 + 2), 128, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, H, W);
+    else input_to_stem_planar_kernel<<<N * (H / 2 + 2), 256, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W);
 }
 
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
