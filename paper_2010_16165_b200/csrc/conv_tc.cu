@@ -743,7 +743,10 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     const long long bank = (long long)taps * a.C_pad * a.K_pad * 2;
     bool bank_fits = plan->flat && bank <= 100 * 1024;
     if (!bank_fits) {
-        while (m_tiles * n_tiles < 148 && n_tile > 64) {      // few position tiles: split the filters to fill the SMs
+        // Few position tiles: split the filters over more CTAs, but only while that doubles the SMs in use.  An MMA
+        // costs about the same for 64 filters as for 128, so a split that merely puts two half-width CTAs on an SM
+        // doubles the work (measured, ResNet-18 batch 64: 512->359 filters at 7x7, 72 us split in six, 39 us in three).
+        while (m_tiles * n_tiles * 2 <= 148 && n_tile > 64) {
             n_tiles *= 2;
             n_tile = round_up_i((a.K_pad + n_tiles - 1) / n_tiles, 16);
         }
@@ -762,11 +765,14 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         // (measured on the ResNet-18 stem at batch 64: 89 us resident, 61 us streamed).
         const bool wide_halo = 2 * plan->halo > 128;
         if (!bank_fits || wide_halo) {
-            // several 128-position tiles per step share every streamed filter block (less filter traffic)
+            // Several 128-position tiles per step share every streamed filter block.  Layers with few positions
+            // and many filters re-stream the bank once per position tile and are bound by L2 bandwidth, so
+            // sharing pays even when it leaves only half of the SMs with a CTA (measured, same network: 368->512
+            // filters at 7x7, 55 us with 164 single-tile CTAs, 32 us with 84 two-tile CTAs).
             for (int tps = 4; tps > 1; tps >>= 1) {
                 const unsigned a_try = (unsigned)(plan->cg * round_up_i(tps * 128 + 2 * plan->halo, 8) * 16);
                 if (2 * tps * n_tile <= 512 && tps * 128 + plan->halo + 8 <= kGuardVectors &&
-                    ((m_tiles + tps - 1) / tps) * n_tiles >= 148 &&
+                    ((m_tiles + tps - 1) / tps) * n_tiles >= 74 &&
                     smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * a_try <= kSmemMax) { plan->tps = tps; break; }
             }
         }
