@@ -832,7 +832,10 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (ctas > tmem_ctas) ctas = tmem_ctas;
     if (ctas > want_ctas) ctas = want_ctas;
     if (ctas < 1) ctas = 1;
-    const int epi = n_tile >= 64 ? 8 : 4;
+    // Wide filter tiles get eight epilogue warps, except in gather mode when there are more tiles than SMs: the
+    // eight-warp form needs too many registers for a second CTA on the SM, and a second CTA is what hides the
+    // loaders' latency there (measured on ResNet-50, batch 128: every strided layer about 30 % faster with four).
+    const int epi = (n_tile >= 64 && (plan->flat || m_tiles * n_tiles <= 148)) ? 8 : 4;
     plan->epi_warps = epi;
     const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
     const void* fn = kernel_for(mode, epi);
