@@ -334,41 +334,61 @@ __global__ void pool_sum_kernel(const void* __restrict__ x, int N, int H, int W,
 }
 
 // Head, step 2: logits[n][k] = sum_c sums[n][c] * Wfc[k][c] + b[k]; the 1/(H*W) of the average is
-// already folded into Wfc.  A block handles 4 images x 32 classes: the channel sums of its images sit
-// in shared memory and every FC row it reads serves all four images.
-constexpr int kFcImages = 4, kFcClasses = 32;
+// already folded into Wfc.  A block handles IMG images x 32 classes, the channels in slabs of 512: the slab of
+// channel sums of its images sits in shared memory and every FC row it reads serves all of them (16 images per
+// block instead of 4 was measured and is slower at batch 64-256: fewer blocks, and L2 is not the bound).
+// A warp owns the classes k0 + warp + 8*t and walks their FC rows together: four independent row loads per
+// step.  Each (image, class) sum has a fixed order: lanes stride over the channels, then a butterfly over the lanes.
+constexpr int kFcClasses = 32, kFcSlab = 512;
+template <int IMG>
 __global__ void fc_kernel(const float* __restrict__ sums, int N, int C_pad, const float* __restrict__ fcw,
                           const float* __restrict__ fcb, int n_classes, float* __restrict__ logits) {
-    extern __shared__ float sh[];          // kFcImages * C_pad
-    const int n0 = blockIdx.x * kFcImages, k0 = blockIdx.y * kFcClasses;
-    for (int i = threadIdx.x; i < kFcImages * C_pad; i += blockDim.x) {
-        const int img = i / C_pad;
-        sh[i] = (n0 + img < N) ? sums[(size_t)(n0 + img) * C_pad + (i - img * C_pad)] : 0.0f;
+    extern __shared__ float sh[];          // IMG * kFcSlab
+    const int n0 = blockIdx.x * IMG, k0 = blockIdx.y * kFcClasses;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kWarps = 8, kPerWarp = kFcClasses / kWarps;       // launched with 256 threads
+    const float* wr[kPerWarp];
+    float acc[kPerWarp][IMG];
+#pragma unroll
+    for (int t = 0; t < kPerWarp; ++t) {
+        const int k = k0 + warp + kWarps * t;
+        wr[t] = fcw + (size_t)(k < n_classes ? k : 0) * C_pad;
+#pragma unroll
+        for (int i = 0; i < IMG; ++i) acc[t][i] = 0.0f;
     }
-    __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (int kk = warp; kk < kFcClasses; kk += nwarps) {
-        const int k = k0 + kk;
-        if (k >= n_classes) break;
-        const float* wr = fcw + (size_t)k * C_pad;
-        float acc[kFcImages];
+    for (int c0 = 0; c0 < C_pad; c0 += kFcSlab) {
+        const int cw = C_pad - c0 < kFcSlab ? C_pad - c0 : kFcSlab;
+        __syncthreads();                   // the previous slab has been consumed
+        for (int img = warp; img < IMG; img += kWarps)
+            for (int cc = lane; cc < cw; cc += 32)
+                sh[img * kFcSlab + cc] = (n0 + img < N) ? sums[(size_t)(n0 + img) * C_pad + c0 + cc] : 0.0f;
+        __syncthreads();
+#pragma unroll 4
+        for (int c = lane; c < cw; c += 32) {      // unrolled: 16 row loads in flight per lane
+            float wv[kPerWarp];
 #pragma unroll
-        for (int i = 0; i < kFcImages; ++i) acc[i] = 0.0f;
-        for (int c = lane; c < C_pad; c += 32) {
-            const float wv = wr[c];
+            for (int t = 0; t < kPerWarp; ++t) wv[t] = wr[t][c0 + c];
 #pragma unroll
-            for (int i = 0; i < kFcImages; ++i) acc[i] = fmaf(sh[i * C_pad + c], wv, acc[i]);
+            for (int i = 0; i < IMG; ++i) {
+                const float sv = sh[i * kFcSlab + c];
+#pragma unroll
+                for (int t = 0; t < kPerWarp; ++t) acc[t][i] = fmaf(sv, wv[t], acc[t][i]);
+            }
         }
+    }
 #pragma unroll
-        for (int i = 0; i < kFcImages; ++i) {
+    for (int t = 0; t < kPerWarp; ++t) {
+        const int k = k0 + warp + kWarps * t;
 #pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) acc[i] += __shfl_xor_sync(0xffffffffu, acc[i], d);
+        for (int i = 0; i < IMG; ++i) {
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) acc[t][i] += __shfl_xor_sync(0xffffffffu, acc[t][i], d);
         }
-        if (lane == 0) {
+        if (lane == 0 && k < n_classes) {
             const float b = fcb ? fcb[k] : 0.0f;
 #pragma unroll
-            for (int i = 0; i < kFcImages; ++i)
-                if (n0 + i < N) logits[(size_t)(n0 + i) * n_classes + k] = acc[i] + b;
+            for (int i = 0; i < IMG; ++i)
+                if (n0 + i < N) logits[(size_t)(n0 + i) * n_classes + k] = acc[t][i] + b;
         }
     }
 }
@@ -435,8 +455,8 @@ void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, con
     const int blocks = (int)((warps * 32 + 255) / 256);
     if (is_bf16) pool_sum_kernel<true><<<blocks, 256, 0, st>>>(x, N, H, W, C_pad / 8, pool_scratch);
     else pool_sum_kernel<false><<<blocks, 256, 0, st>>>(x, N, H, W, C_pad / 8, pool_scratch);
-    dim3 grid((N + kFcImages - 1) / kFcImages, (n_classes + kFcClasses - 1) / kFcClasses);
-    fc_kernel<<<grid, 256, (size_t)kFcImages * C_pad * sizeof(float), st>>>(pool_scratch, N, C_pad, fcw, fcb, n_classes, logits);
+    const int classes = (n_classes + kFcClasses - 1) / kFcClasses;
+    fc_kernel<4><<<dim3((N + 3) / 4, classes), 256, 4 * kFcSlab * sizeof(float), st>>>(pool_scratch, N, C_pad, fcw, fcb, n_classes, logits);
 }
 
 void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
