@@ -783,10 +783,28 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         if (bank_fits) {
             plan->b_resident = 1;
             plan->b_stages = 1;
-            plan->a_stages = 4;
-            unsigned fixed = smem + (unsigned)round_up_i((int)bank, 128);
-            while (plan->a_stages > 2 && fixed + plan->a_stages * a_stage > 110 * 1024) --plan->a_stages;
-            smem = fixed + plan->a_stages * a_stage;
+            const unsigned fixed = smem + (unsigned)round_up_i((int)bank, 128);
+            auto fit = [&](int cg, int* stages) {
+                const unsigned st = (unsigned)(cg * plan->rows_a * 16);
+                *stages = 4;
+                while (*stages > 2 && fixed + *stages * st > 110 * 1024) --*stages;
+                return fixed + *stages * st;
+            };
+            unsigned total = fit(plan->cg, &plan->a_stages);
+            // One thread issues a CTA's MMAs, about 100 cycles apiece, and that bounds a layer of few filters; a
+            // second CTA on the SM doubles the rate.  Where only the activation stages keep a second CTA out,
+            // they are halved to four channel chunks (measured, 64 -> 48 filters at 56x56, batch 64: 27 -> 20 us).
+            if (plan->cg == 8 && total + 1024u > kSmemPerSm / 2) {
+                int st4;
+                const unsigned t4 = fit(4, &st4);
+                if (t4 + 1024u <= kSmemPerSm / 2) {
+                    plan->cg = 4;
+                    plan->groups = (cchunks + 3) / 4;
+                    plan->a_stages = st4;
+                    total = t4;
+                }
+            }
+            smem = total;
         } else {
             plan->b_resident = 0;
             plan->b_stages = 8;      // filter blocks are small next to the copy latency: keep many in flight
