@@ -833,7 +833,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         if (smem + plan->a_stages * stage > 56 * 1024) {
             plan->a_stages = 6;
             want_ctas = 2;
-            while (plan->a_stages > 2 && smem + plan->a_stages * stage > 120 * 1024) --plan->a_stages;
+            while (plan->a_stages > 2 && smem + plan->a_stages * stage > kSmemPerSm / 2 - 1024u) --plan->a_stages;   // two CTAs must fit
         }
         plan->b_stages = plan->a_stages;
         smem += plan->a_stages * stage;
