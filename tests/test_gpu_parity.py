@@ -450,3 +450,29 @@ def test_config1_aggressive_fused_unpruned_and_pruned(B, fpo):
             np.testing.assert_array_equal(m[0], masks[ci])
     finally:
         g.close()
+
+
+def test_maxpool_windows_of_negative_values(B, fpo):
+    """Max pooling right after a batch norm without ReLU, every other channel shifted far below zero, so a padded
+    position that took part in a window as 0 (instead of being ignored) would win it.  Odd height, a width that
+    leaves the second warp of a row partly empty; compared operator by operator."""
+    net = wl.Net(3, 37, 70, "pool_negative")
+    x = net.bn(net.conv(-1, 16, 3, 3, 1, 1), 16)
+    x = net.maxpool(x, 16)
+    x = net.gavgpool(x, 16)
+    net.fc(x, 5, 16)
+    net.n_blocks = 0
+    w = wl.Workload("pool_negative", net, 2, 23, True, wl.uniform_ratios(0.0), "none")
+    node = [n for n in net.nodes if n["op"] == wl.OP_BN][0]
+    w.bn[node["bn_off"] + 16:node["bn_off"] + 32:2] = -3.0        # beta of every other channel: all-negative windows
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, keep_outputs=1)
+    try:
+        got = g.forward(w.x)
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        ref_all = fpo.fused_forward(gp, w.x, return_all=True)
+        pooled = [ref_all[op["out"]] for op in gp.ops][1]
+        assert (pooled < 0).mean() > 0.05, "the case must contain windows whose maximum is negative"
+        _compare_ops(B, g, w, gp, fpo, TOL_BF16)
+        assert err(got, fpo.fused_forward(gp, w.x)) < TOL_BF16
+    finally:
+        g.close()
