@@ -99,6 +99,12 @@ typedef struct {
     int32_t use_graph;                  /* 1: fp_forward replays a captured CUDA graph          */
     int32_t keep_outputs;               /* 1: every operator keeps its own output buffer (needed for
                                            FP_Q_OP_OUTPUT on any operator; default 0 reuses memory) */
+    int32_t scatter;                    /* pruned convolutions that write a residual stream (their output is a shortcut
+                                           operand, so the tensor keeps its full width): 0 = compute only the kept
+                                           filters and scatter them into the full-width tensor where that pays (wide
+                                           layers with a long reduction), zero filter rows elsewhere; 1 = scatter
+                                           wherever it saves accumulator columns; -1 = always zero rows.  The
+                                           result is the same in every case (Algorithm 1's removal of masked filters) */
 } fp_model_desc;
 
 /*
@@ -130,6 +136,10 @@ fp_status fp_fuse(const fp_model_desc* desc, const float* d_weights, size_t n_we
  *               bytes (1 keep / 0 prune) for that convolution; or NULL.
  * Always starts from the unpruned fused weights, so ratios of 0 restore the unpruned model.
  * Errors: FP_ERR_ARG, FP_ERR_EMPTY_LAYER, FP_ERR_NOMEM, FP_ERR_CUDA.  Synchronous.
+ * Arguments are checked, and every mask selected, before anything is changed: FP_ERR_ARG and
+ * FP_ERR_EMPTY_LAYER leave the previous graph running.  A failure while the new graph is being built
+ * (FP_ERR_NOMEM, FP_ERR_CUDA) leaves the handle without a graph: fp_forward then returns FP_ERR_ARG
+ * until a later fp_prune succeeds.
  */
 fp_status fp_prune(fp_handle h, int32_t norm, const double* h_ratios, const uint8_t* const* h_masks);
 
@@ -171,7 +181,11 @@ typedef enum {
     FP_Q_N_OPS = 9,          /* int32: fused operators in execution order                         */
     FP_Q_OP_INFO = 10,       /* fp_op_info of fused operator `index`                              */
     FP_Q_OP_OUTPUT = 11,     /* float[batch*C*H*W] NCHW, logical channels: output of fused operator
-                                `index` from the last fp_forward (debug; synchronises the device)  */
+                                `index` for the input of the last fp_forward (debug; synchronises the device).
+                                Without keep_outputs the launches up to that operator are run again first (the
+                                last input must still be alive), and a layer inside a fused run, whose output
+                                never reaches memory, is refused with FP_ERR_UNSUPPORTED - the run's last
+                                layer can be read */
     FP_Q_DEVICE_STATUS = 12, /* int32: 0, or FP_ERR_TIMEOUT if a bounded device wait ran out       */
     FP_Q_N_LAUNCHES = 13,    /* int32: kernels one fp_forward launches                             */
     FP_Q_OP_TIMES = 14       /* float[N_OPS]: milliseconds per fused operator of a forward of the last batch size,

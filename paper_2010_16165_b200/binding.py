@@ -40,7 +40,7 @@ class fp_model_desc(ctypes.Structure):
     _fields_ = [("n_nodes", ctypes.c_int32), ("nodes", ctypes.POINTER(fp_node)),
                 ("in_C", ctypes.c_int32), ("in_H", ctypes.c_int32), ("in_W", ctypes.c_int32),
                 ("in_dtype", ctypes.c_int32), ("compute", ctypes.c_int32), ("bn_eps", ctypes.c_float),
-                ("use_graph", ctypes.c_int32), ("keep_outputs", ctypes.c_int32)]
+                ("use_graph", ctypes.c_int32), ("keep_outputs", ctypes.c_int32), ("scatter", ctypes.c_int32)]
 
 
 class fp_op_info(ctypes.Structure):
@@ -99,11 +99,11 @@ def make_nodes(node_dicts):
 
 
 def fp_fuse(net, d_weights, d_bn, max_batch, compute=FP_COMPUTE_BF16_TC, in_dtype=FP_DTYPE_F32, use_graph=0,
-            keep_outputs=0):
+            keep_outputs=0, scatter=0):
     """net: workloads.Net; d_weights/d_bn: CUDA float32 torch tensors.  Returns an opaque handle."""
     nodes = make_nodes(net.nodes)
     desc = fp_model_desc(len(net.nodes), nodes, net.in_C, net.in_H, net.in_W, in_dtype, compute,
-                         float(net.bn_eps), use_graph, keep_outputs)
+                         float(net.bn_eps), use_graph, keep_outputs, scatter)
     h = ctypes.c_void_p()
     _check(lib().fp_fuse(ctypes.byref(desc), d_weights.data_ptr(), d_weights.numel(), d_bn.data_ptr(),
                          d_bn.numel(), max_batch, ctypes.byref(h)))

@@ -75,6 +75,10 @@ struct FConv {
     std::vector<int32_t> rank;
     // derived by replan()
     int compact = 0;           // 1: pruned filters are physically removed from the output tensor
+    int scatter = 0;           // 1: only kept filters are computed, scattered into a full-width output (residual stream)
+    int n_tile_forced = 0;     // scatter: filters per CTA tile the packed bank was laid out for
+    int32_t* d_out_map = nullptr;   // scatter: output channel -> packed filter row (-1 = no filter kept)
+    int32_t* d_chunk0 = nullptr;    // scatter: first output chunk of every filter tile, and the end
     int K_kept = 0, K_rows = 0, K_pad = 0, C_kept = 0, C_pad = 0;
     void* d_wp = nullptr;      // packed filters in the compute type, K_pad x R x S x C_pad
     float* d_bp = nullptr;
@@ -145,6 +149,8 @@ struct fp_handle_s {
     double* d_soft_scores = nullptr; int32_t* d_soft_rank = nullptr; uint8_t* d_soft_mask = nullptr;
     int soft_total = 0;
     int stem_packed = 0;                   // network input stored in the packed form of a 7x7/2 first convolution
+    int scatter_policy = 0;                // fp_model_desc::scatter
+    int planned = 0;                       // 1: buffers, packed banks and launch plans match the masks (set by replan)
     int act_is_bf16() const { return compute != FP_COMPUTE_FP32; }
     size_t act_elem() const { return act_is_bf16() ? 2 : 4; }
     size_t in_elem() const { return in_dtype == FP_DTYPE_BF16 ? 2 : 4; }
@@ -605,7 +611,7 @@ fp_status upload_i32(fp_handle h, const std::vector<int32_t>& v, int32_t** out) 
 }
 
 bool chain_candidate(fp_handle h, const FConv& f) {
-    if (h->compute != FP_COMPUTE_BF16_TC || h->keep_outputs) return false;
+    if (h->compute != FP_COMPUTE_BF16_TC || h->keep_outputs || f.scatter) return false;
     if (f.R != 3 || f.S != 3 || f.stride != 1 || f.pad != 1) return false;
     if (h->stem_packed && f.src == 0) return false;
     const Tensor& s = h->tensors[f.src];
@@ -699,7 +705,22 @@ fp_status find_chains(fp_handle h, const std::vector<std::vector<Use>>& uses) {
     return FP_OK;
 }
 
+// Geometry of the launch of fused convolution f (no pointers, no channel counts of the output).
+void conv_geometry(fp_handle h, const FConv& f, fp::ConvArgs* a) {
+    const Tensor& src = h->tensors[f.src];
+    const Tensor& out = h->tensors[f.out];
+    a->N = h->max_batch; a->H = src.H; a->W = src.W; a->C_pad = src.C_pad; a->P = out.H; a->Q = out.W;
+    a->R = f.R; a->S = f.S; a->stride = f.stride; a->pad = f.pad; a->relu = f.relu;
+    if (h->stem_packed && f.src == 0) {      // 3x1 stride-1 convolution over the packed input, at the output resolution
+        a->H = out.H; a->W = out.W; a->C_pad = 80; a->R = 3; a->S = 1; a->stride = 1; a->pad = 1;
+    }
+}
+
+// Rebuilds everything that depends on the masks.  The old buffers are released first, so while this runs - and
+// after it failed half-way (out of memory, a layer left without filters) - the handle has no plan: `planned` stays
+// 0 and every call that would launch kernels refuses until a later fp_prune succeeds.
 fp_status replan(fp_handle h) {
+    h->planned = 0;
     drop_graphs(h);
     CK(cudaDeviceSynchronize());
     free_list(h->act_buffers);
@@ -733,20 +754,84 @@ fp_status replan(fp_handle h) {
             f.K_kept = (int)kept.size();
             f.compact = (f.res_mode == 0 && compactable(h, uses, f.out)) ? 1 : 0;
             f.C_kept = src.C; f.C_pad = src.C_pad;
-            std::vector<int32_t> row_src, chan_src(f.C_pad, -1);
-            if (f.compact) {
-                f.K_rows = f.K_kept;
-                out.keep = kept;
-                for (int k : kept) row_src.push_back(k);
-            } else {
-                f.K_rows = f.K;
-                out.keep.resize(f.K);
-                for (int k = 0; k < f.K; ++k) { out.keep[k] = k; row_src.push_back(f.mask[k] ? k : -1); }
+            // A convolution that writes a residual stream (its output is added to, or read as, a shortcut) cannot drop
+            // output channels: other layers write them too.  On the tensor-core path it still computes only its kept
+            // filters and scatters them into the full-width tensor in the epilogue; layers that can join a fused run of
+            // layers, and the validation paths, keep pruned filters as zero rows instead.
+            f.scatter = 0; f.n_tile_forced = 0; f.d_out_map = nullptr; f.d_chunk0 = nullptr;
+            if (!f.compact && h->compute == FP_COMPUTE_BF16_TC && round_up(f.K_kept, 16) < round_up(f.K, 16)) {
+                const bool runs_fused = !h->keep_outputs && f.R == 3 && f.S == 3 && f.stride == 1 && f.pad == 1 &&
+                                        !(h->stem_packed && f.src == 0) &&
+                                        fp::chain_layer_supported(src.H, src.W, round_up(f.K, 16), src.C_pad);
+                // It has to pay: an MMA over n filters costs the tensor pipe about max(n/2, 32 + n/4) cycles (the second
+                // term is the operand fetch), so 64 -> 48 or 128 -> 96 columns save a tenth while the scattering epilogue
+                // costs more than that on layers with a short reduction; it is used where the tensor-pipe cost of the
+                // kept filters is at most 0.8 of the full width's and the reduction is at least 1024 long.
+                fp::ConvArgs ga;
+                memset(&ga, 0, sizeof(ga));
+                conv_geometry(h, f, &ga);
+                auto pipe_cost = [&](int K_pad) {
+                    int nt = 0, nts = 0;
+                    fp::conv_tc_filter_tile(ga, K_pad, &nt, &nts);
+                    return nts * std::max(nt / 2, 32 + nt / 4);
+                };
+                const bool pays = 5 * pipe_cost(round_up(f.K_kept, 16)) <= 4 * pipe_cost(round_up(f.K, 16)) &&
+                                  ga.R * ga.S * ga.C_pad >= 1024;
+                if (!runs_fused && h->scatter_policy >= 0 && (pays || h->scatter_policy > 0)) f.scatter = 1;
             }
-            f.K_pad = round_up(f.K_rows, 16);
-            row_src.resize(f.K_pad, -1);
+            std::vector<int32_t> row_src, chan_src(f.C_pad, -1);
+            if (f.scatter) {
+                // Filter tiles must own whole output chunks (8 channels = one 16-byte vector per position): fill each tile
+                // with consecutive chunks while their kept filters fit, and pad its rows with zero filters.
+                fp::ConvArgs ga;
+                memset(&ga, 0, sizeof(ga));
+                conv_geometry(h, f, &ga);
+                const int out_C_pad = round_up(f.K, 16), n_chunks = out_C_pad / 8;
+                int n_tile = 0, n_tiles = 0;
+                fp::conv_tc_filter_tile(ga, round_up(f.K_kept, 16), &n_tile, &n_tiles);
+                std::vector<int> cnt(n_chunks, 0);
+                for (int k : kept) ++cnt[k / 8];
+                std::vector<int32_t> chunk0;
+                for (;;) {
+                    chunk0.assign(1, 0);
+                    int cur = 0;
+                    for (int q = 0; q < n_chunks; ++q) {
+                        if (cur + cnt[q] > n_tile) { chunk0.push_back(q); cur = 0; }
+                        cur += cnt[q];
+                    }
+                    chunk0.push_back(n_chunks);
+                    if ((int)chunk0.size() - 1 <= n_tiles || n_tile >= 128) break;
+                    n_tile += 16;            // chunk-aligned tiles wasted too many rows: widen the tile and try again
+                }
+                n_tiles = (int)chunk0.size() - 1;
+                std::vector<int32_t> out_map(out_C_pad, -1);
+                row_src.assign((size_t)n_tiles * n_tile, -1);
+                for (int t = 0; t < n_tiles; ++t) {
+                    int r = t * n_tile;
+                    for (int c = chunk0[t] * 8; c < chunk0[t + 1] * 8 && c < f.K; ++c)
+                        if (f.mask[c]) { row_src[r] = c; out_map[c] = r; ++r; }
+                }
+                f.K_rows = f.K; f.K_pad = n_tiles * n_tile; f.n_tile_forced = n_tile;
+                out.keep.resize(f.K);
+                for (int k = 0; k < f.K; ++k) out.keep[k] = k;
+                TRY(upload_i32(h, out_map, &f.d_out_map));
+                TRY(upload_i32(h, chunk0, &f.d_chunk0));
+                out.C = f.K; out.C_pad = out_C_pad;
+            } else {
+                if (f.compact) {
+                    f.K_rows = f.K_kept;
+                    out.keep = kept;
+                    for (int k : kept) row_src.push_back(k);
+                } else {
+                    f.K_rows = f.K;
+                    out.keep.resize(f.K);
+                    for (int k = 0; k < f.K; ++k) { out.keep[k] = k; row_src.push_back(f.mask[k] ? k : -1); }
+                }
+                f.K_pad = round_up(f.K_rows, 16);
+                row_src.resize(f.K_pad, -1);
+                out.C = f.K_rows; out.C_pad = f.K_pad;
+            }
             for (int c = 0; c < src.C; ++c) chan_src[c] = src.keep[c];
-            out.C = f.K_rows; out.C_pad = f.K_pad;
             // pack filters and bias
             int32_t *d_row, *d_chan;
             TRY(upload_i32(h, row_src, &d_row));
@@ -833,11 +918,11 @@ fp_status replan(fp_handle h) {
         fp::ConvArgs& a = f.args;
         memset(&a, 0, sizeof(a));
         a.x = src.d; a.y = out.d; a.w = f.d_wp; a.bias = f.d_bp;
-        a.N = h->max_batch; a.H = src.H; a.W = src.W; a.C_pad = f.C_pad; a.P = out.H; a.Q = out.W;
-        a.K_pad = f.K_pad; a.R = f.R; a.S = f.S; a.stride = f.stride; a.pad = f.pad; a.relu = f.relu;
-        if (h->stem_packed && f.src == 0) {      // 3x1 stride-1 convolution over the packed input, at the output resolution
-            a.H = out.H; a.W = out.W; a.C_pad = 80; a.R = 3; a.S = 1; a.stride = 1; a.pad = 1;
-        }
+        conv_geometry(h, f, &a);
+        a.C_pad = (h->stem_packed && f.src == 0) ? 80 : f.C_pad;
+        a.K_pad = f.K_pad;
+        a.scatter = f.scatter; a.out_C_pad = out.C_pad; a.out_map = f.d_out_map; a.tile_chunk0 = f.d_chunk0;
+        a.n_tile_forced = f.n_tile_forced;
         a.res_mode = f.res_mode;
         if (f.res_mode) {
             const Tensor& r = h->tensors[f.res_tid];
@@ -857,7 +942,14 @@ fp_status replan(fp_handle h) {
         ch.args.x = f0.args.x; ch.args.res = f0.args.res; ch.args.y = fl.args.y; ch.args.w = ch.d_blob;
     }
     CK(cudaDeviceSynchronize());
+    h->planned = 1;
     return FP_OK;
+}
+
+fp_status need_plan(fp_handle h, const char* who) {
+    if (h->planned) return FP_OK;
+    return fail(FP_ERR_ARG, "%s: the last fp_prune / fp_soft_prune_finish failed and left the handle without a plan; "
+                            "call fp_prune again", who);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -942,6 +1034,7 @@ extern "C" fp_status fp_fuse(const fp_model_desc* desc, const float* d_weights, 
     if (desc->in_C <= 0 || desc->in_H <= 0 || desc->in_W <= 0) return fail(FP_ERR_ARG, "fp_fuse: bad input shape");
     if (desc->in_dtype != FP_DTYPE_F32 && desc->in_dtype != FP_DTYPE_BF16) return fail(FP_ERR_ARG, "fp_fuse: bad in_dtype");
     if (desc->compute < 0 || desc->compute > 2) return fail(FP_ERR_ARG, "fp_fuse: bad compute mode");
+    if (desc->scatter < -1 || desc->scatter > 1) return fail(FP_ERR_ARG, "fp_fuse: bad scatter policy");
     if (!(desc->bn_eps > 0.0f) || !std::isfinite(desc->bn_eps)) return fail(FP_ERR_ARG, "fp_fuse: bn_eps must be positive");
     int dev = 0;
     cudaDeviceProp prop;
@@ -954,6 +1047,7 @@ extern "C" fp_status fp_fuse(const fp_model_desc* desc, const float* d_weights, 
     h->in_C = desc->in_C; h->in_H = desc->in_H; h->in_W = desc->in_W;
     h->in_dtype = desc->in_dtype; h->compute = desc->compute; h->use_graph = desc->use_graph;
     h->keep_outputs = desc->keep_outputs;
+    h->scatter_policy = desc->scatter;
     h->eps = desc->bn_eps; h->max_batch = max_batch;
     fp_status s = FP_OK;
     auto body = [&]() -> fp_status {
@@ -1127,6 +1221,7 @@ extern "C" fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch,
     if (!h || !d_input || !d_logits) return fail(FP_ERR_ARG, "fp_forward: NULL argument");
     if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward: batch must be positive");
     if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward: batch %d exceeds max_batch %d", batch, h->max_batch);
+    TRY(need_plan(h, "fp_forward"));
     cudaStream_t st = (cudaStream_t)stream;
     h->last_input = d_input; h->last_batch = batch;
     const bool graphable = h->use_graph && st != 0 && st != cudaStreamLegacy && st != cudaStreamPerThread;
@@ -1165,6 +1260,7 @@ extern "C" fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t b
     if (!h || !h_input || !h_logits) return fail(FP_ERR_ARG, "fp_forward_host: NULL argument");
     if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward_host: batch must be positive");
     if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward_host: batch %d exceeds max_batch %d", batch, h->max_batch);
+    TRY(need_plan(h, "fp_forward_host"));
     cudaStream_t st = (cudaStream_t)stream;
     const size_t in_bytes = (size_t)batch * h->in_C * h->in_H * h->in_W * h->in_elem();
     CK(cudaMemcpyAsync(h->d_in_stage, h_input, in_bytes, cudaMemcpyHostToDevice, st));
@@ -1271,6 +1367,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             if (index < 0 || index >= (int)h->ops.size() || h->ops[index].kind == 2)
                 return fail(FP_ERR_ARG, "fp_query: operator %d has no activation output", index);
             if (h->last_batch <= 0) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
+            TRY(need_plan(h, "fp_query"));
             if (h->ops[index].kind == 3 && h->stem_packed) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is stored in packed form");
             if (h->ops[index].kind == 3 && h->input_fused) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is converted inside the first fused run "
                                                                         "and never stored (set keep_outputs to run every layer on its own)");
@@ -1283,6 +1380,13 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             TRY(need(cnt * sizeof(float)));
             float* d_tmp;
             CK(cudaDeviceSynchronize());
+            if (!h->keep_outputs) {
+                // Buffers are reused once their last reader has run, so the tensor may have been overwritten since:
+                // run the forward's launches up to this operator again (same input, same kernels) and stop there.
+                if (!h->last_input) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
+                for (int j = 0; j <= index; ++j) launch_op(h, j, h->last_input, h->last_batch, h->d_logits_stage, 0);
+                CK(cudaDeviceSynchronize());
+            }
             CK(cudaMalloc(&d_tmp, cnt * sizeof(float)));
             fp::launch_planar_to_nchw_f32(t.d, h->act_is_bf16(), d_tmp, h->last_batch, t.H, t.W, t.C_pad, t.C, 0);
             cudaError_t e = cudaMemcpy(h_out, d_tmp, cnt * sizeof(float), cudaMemcpyDeviceToHost);
@@ -1301,6 +1405,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             const int n = (int)h->ops.size();
             TRY(need((size_t)n * sizeof(float)));
             if (h->last_batch <= 0 || !h->last_input) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
+            TRY(need_plan(h, "fp_query"));
             // Operator i's time = (time of the launches 0..i) - (time of the launches 0..i-1), each prefix of the forward
             // captured as a CUDA graph - the way fp_forward runs them, programmatic dependent launch included - and
             // replayed `reps` times back to back between two events.  An event between two kernels would cost more

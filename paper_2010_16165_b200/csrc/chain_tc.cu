@@ -558,7 +558,8 @@ int plan_chain_tc(const ChainArgs& a, ChainPlan* plan, char* err, size_t err_len
         const unsigned smem = (unsigned)sizeof(ChainCtrl) + 128u + 2u * wbuf + 2u * (unsigned)max_chunks * rows * 16u;
         if (smem > kSmemMax) break;
         const int groups = (a.N + G - 1) / G;
-        const int rounds = (groups + 147) / 148;
+        const int sms = sm_count();
+        const int rounds = (groups + sms - 1) / sms;
         const double cost = rounds * (tiles + 1.5);
         if (best_G == 0 || cost <= best_cost) { best_G = G; best_cost = cost; }
     }
@@ -579,14 +580,11 @@ int plan_chain_tc(const ChainArgs& a, ChainPlan* plan, char* err, size_t err_len
     unsigned smem = (unsigned)sizeof(ChainCtrl) + 128u + 2u * wbuf + 2u * (unsigned)plan->buf_bytes;
     if (smem < kSmemMin) smem = kSmemMin;
     plan->smem_bytes = smem;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
-            snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
-            cudaGetLastError();
-            return 1;
-        }
-        attr_set = true;
+    // a per-device attribute: set it for the device this plan is made on (cheap, so not cached)
+    if (cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
+        snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
+        cudaGetLastError();
+        return 1;
     }
     plan->valid = 1;
     return 0;
@@ -611,7 +609,8 @@ void launch_chain_tc(const ChainPlan& plan, const ChainArgs& a, int* d_status, c
     p.rWp = a.res_W + 2; p.rP2 = (a.res_H + 2) * (a.res_W + 2);
     p.plane_res = (long long)a.N * p.rP2;
     p.status = d_status;
-    int grid = p.n_groups < 148 ? p.n_groups : 148;
+    const int sms = sm_count();
+    int grid = p.n_groups < sms ? p.n_groups : sms;
     if (grid < 1) grid = 1;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));

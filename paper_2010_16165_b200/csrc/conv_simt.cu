@@ -85,7 +85,8 @@ __global__ void conv_simt_kernel(ConvArgs a) {
 void launch_conv_simt(const ConvArgs& a, int is_bf16, cudaStream_t st) {
     const size_t total = (size_t)a.N * (a.P + 2) * (a.Q + 2) * (a.K_pad / 8);
     size_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    const size_t cap = (size_t)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     if (is_bf16) conv_simt_kernel<__nv_bfloat16><<<(int)blocks, 256, 0, st>>>(a);
     else conv_simt_kernel<float><<<(int)blocks, 256, 0, st>>>(a);

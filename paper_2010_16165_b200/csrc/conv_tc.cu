@@ -30,6 +30,7 @@
 //                 global memory, all roles leave their loops, tensor memory is released and the
 //                 kernel returns (results are then invalid and the host reports FP_ERR_TIMEOUT).
 #include "fp_internal.h"
+#include "tc_common.cuh"
 
 #include <cstdio>
 #include <cstring>
@@ -38,15 +39,11 @@ namespace fp {
 
 namespace {
 
+using namespace tc;
+
 constexpr int kMaxStages = 8;
-constexpr uint32_t kWaitLimit = 1u << 24;          // polls per wait, and
-constexpr long long kWaitCycles = 2000000000LL;    // SM clock cycles per wait (about a second)
 
 enum { MODE_FLAT_RESIDENT = 0, MODE_FLAT_STREAM = 1, MODE_GATHER = 2 };
-
-// Division by a run-time constant as multiply-high + shift (n < 2^31, d >= 1).
-struct FastDiv { uint32_t mul, shift, d; };
-__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f) { return (__umulhi(n, f.mul) + n) >> f.shift; }
 
 struct TcParams {
     ConvArgs a;
@@ -60,98 +57,9 @@ struct TcParams {
     int tps;                            // streamed filters: 128-position tiles per pipeline step (share each filter block)
     int a_stage_bytes, b_stage_bytes, b_bank_bytes;
     int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
+    int scatter_bytes;                  // scattered output: channel -> accumulator column map and the tiles' chunk ranges
     int* status;
 };
-
-// ---- PTX wrappers -------------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the time limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 32) __nanosleep(32);
-        if ((i & 127) == 127) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) return false;
-        }
-    }
-    return false;
-}
-
-// Contiguous global -> shared copy by the bulk-copy engine; completion is counted in bytes on `bar`.
-__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Same, with both descriptors given by their low words; the high word (stride offset 128 B,
-// descriptor version 1, no swizzle) is the same constant for every operand block of this kernel.
-__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %5};\n\t"
-        "mov.b64 db, {%2, %5};\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0x4008u) : "memory");
-}
-// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, K-major, no swizzle: rows of 16 bytes, 8 rows contiguous
-// (one 128-byte core matrix), `sbo` = 128 bytes between 8-row groups, `lbo` bytes between the two
-// 8-channel halves of a K=16 step.  Descriptor version 1 (bit 46).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)(128 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    return d;
-}
 
 // Issues the MMAs of one K block of a FLAT-mode tile: R*R filter taps x KSTEPS K=16 steps, fully
 // unrolled so that the single issuing thread spends a handful of instructions per MMA.  Operand
@@ -241,7 +149,11 @@ conv_tc_kernel(const TcParams p) {
     const uint32_t ctrl_addr = smem_u32(smem_raw);
     float* bias_s = reinterpret_cast<float*>(smem_raw + sizeof(Ctrl));            // K_pad floats
     int2* lut = reinterpret_cast<int2*>(smem_raw + sizeof(Ctrl) + (size_t)p.a.K_pad * 4u);   // gather mode only
-    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + (uint32_t)p.a.K_pad * 4u + (uint32_t)p.lut_bytes + 1023u) & ~1023u;
+    int* smap = reinterpret_cast<int*>(smem_raw + sizeof(Ctrl) + (size_t)p.a.K_pad * 4u + (size_t)p.lut_bytes);   // scattered output only
+    int* schunk0 = smap + p.a.out_C_pad;
+    float* sstrip = reinterpret_cast<float*>(schunk0 + ((p.n_tiles + 1 + 3) & ~3));          // EPI warps x 32 rows x 33 words
+    const uint32_t b_base = (ctrl_addr + (uint32_t)sizeof(Ctrl) + (uint32_t)p.a.K_pad * 4u + (uint32_t)p.lut_bytes +
+                             (uint32_t)p.scatter_bytes + 1023u) & ~1023u;
     const uint32_t b_region = MODE == MODE_FLAT_RESIDENT ? (uint32_t)p.b_bank_bytes
                               : MODE == MODE_FLAT_STREAM ? (uint32_t)(p.b_stages * p.b_stage_bytes) : 0u;
     const uint32_t a_base = b_base + ((b_region + 127u) & ~127u);
@@ -271,6 +183,10 @@ conv_tc_kernel(const TcParams p) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     for (int i = threadIdx.x; i < p.a.K_pad; i += blockDim.x) bias_s[i] = p.a.bias[i];   // filters' data: safe before the dependency wait
+    if (p.a.scatter) {
+        for (int i = threadIdx.x; i < p.a.out_C_pad; i += blockDim.x) smap[i] = p.a.out_map[i];
+        for (int i = threadIdx.x; i <= p.n_tiles; i += blockDim.x) schunk0[i] = p.a.tile_chunk0[i];
+    }
     if (MODE == MODE_GATHER) {
         // Plane i of K block kb holds channel chunk c of tap (r, s): its offset from the tile's first tap, in
         // 16-byte vectors, and r, s, "in use" and the block's plane count, are the same for every tile.
@@ -507,7 +423,7 @@ conv_tc_kernel(const TcParams p) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) rq[i] = make_uint4(0, 0, 0, 0);
             const bool res1 = interior && p.a.res_mode == 1;
-            if (res1) {
+            if (res1 && !p.a.scatter) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (c_begin + i * 8 < c_end) rq[i] = __ldg(res + vec0 + (long long)((c_begin >> 3) + i) * p.plane_out);
@@ -525,6 +441,87 @@ conv_tc_kernel(const TcParams p) {
                 res_vec = (long long)n * rP2 + (long long)((hp - 1) * p.a.res_stride + 1) * rWp + ((wq - 1) * p.a.res_stride + 1);
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((acc * p.tps + t) * p.n_tile);
+            if (p.a.scatter) {
+                // Scattered output: this filter tile owns the output chunks [q_begin, q_end) of the full-width tensor, and its
+                // accumulator columns are the kept filters of those chunks in channel order.  Columns are read 16 at a
+                // time and parked in a per-warp strip of shared memory (a ring of 32 columns per row, row pitch 33 words:
+                // conflict-free); a chunk of 8 output channels then picks its kept channels' columns from there by index -
+                // the same index in every lane - and takes the shortcut alone for the others.
+                int q_begin = schunk0[nt], q_end = schunk0[nt + 1];
+                if (EPI == 8) {
+                    const int mid = q_begin + (q_end - q_begin + 1) / 2;
+                    if (half) q_begin = mid; else q_end = mid;
+                }
+                float* strip = sstrip + ((warp - 2) * 32 + lane) * 33;
+                const long long rplane = (long long)p.a.N * (p.a.res_H + 2) * (p.a.res_W + 2);
+                uint4 rnext = make_uint4(0, 0, 0, 0);
+                if (res1 && q_begin < q_end) rnext = __ldg(res + (long long)q_begin * p.plane_out + f);
+                int loaded = -1;                 // accumulator columns [.., loaded) of this tile are in the strip
+                for (int q = q_begin; q < q_end; ++q) {
+                    const uint4 rcur = rnext;
+                    if (res1 && q + 1 < q_end) rnext = __ldg(res + (long long)(q + 1) * p.plane_out + f);
+                    const int4 m0 = *reinterpret_cast<const int4*>(smap + 8 * q);
+                    const int4 m1 = *reinterpret_cast<const int4*>(smap + 8 * q + 4);
+                    const int col[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                    int first = -1, last = -1;   // accumulator columns (within the tile) this chunk needs: consecutive ones
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (col[e] >= 0) { last = col[e] - k_base; if (first < 0) first = last; }
+                    if (loaded < 0 && first >= 0) loaded = first & ~15;                            // first group this warp needs
+                    while (last >= loaded && loaded >= 0) {
+                        uint32_t v[16];
+                        __syncwarp();
+                        tmem_ld16(taddr + (uint32_t)loaded, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) strip[(loaded & 16) + i] = __uint_as_float(v[i]);
+                        loaded += 16;
+                    }
+                    if (!exists) continue;
+                    uint4 o = make_uint4(0, 0, 0, 0);
+                    if (interior) {
+                        float fv[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) fv[e] = col[e] >= 0 ? strip[(col[e] - k_base) & 31] + bias_s[col[e]] : 0.0f;
+                        if (p.a.res_mode == 1) {
+                            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&rcur);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 g = __bfloat1622float2(h2[i]);
+                                fv[2 * i] += g.x;
+                                fv[2 * i + 1] += g.y;
+                            }
+                        } else if (p.a.res_mode == 2) {
+                            const int cs = 8 * q - p.a.res_pad_lo;
+                            if (cs >= 0 && cs + 8 <= p.a.res_C_pad && (cs & 7) == 0) {
+                                const uint4 raw = __ldg(res + (long long)(cs >> 3) * rplane + res_vec);
+                                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const float2 g = __bfloat1622float2(h2[i]);
+                                    fv[2 * i] += g.x;
+                                    fv[2 * i + 1] += g.y;
+                                }
+                            } else if (cs + 8 > 0 && cs < p.a.res_C) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const int c = cs + i;
+                                    if (c >= 0 && c < p.a.res_C)
+                                        fv[i] += __bfloat162float(res_s[((long long)(c >> 3) * rplane + res_vec) * 8 + (c & 7)]);
+                                }
+                            }
+                        }
+                        if (p.a.relu) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) fv[i] = fmaxf(fv[i], 0.0f);
+                        }
+                        __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) o2[i] = __floats2bfloat162_rn(fv[2 * i], fv[2 * i + 1]);
+                    }
+                    y[(long long)q * p.plane_out + f] = o;
+                }
+            } else
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 uint32_t v[16];
                 __syncwarp();
@@ -596,7 +593,7 @@ conv_tc_kernel(const TcParams p) {
                 // rotate the residual queue and refill its tail
 #pragma unroll
                 for (int i = 0; i < 6; ++i) rq[i] = rq[i + 2];
-                if (res1 && c0 + 64 < c_end) {
+                if (res1 && c0 + 64 < c_end) {   // (dense output only: this loop is not entered when the output is scattered)
                     const long long vn = vec0 + (long long)((c0 + 64) >> 3) * p.plane_out;
                     rq[6] = __ldg(res + vn);
                     rq[7] = __ldg(res + vn + p.plane_out);
@@ -703,15 +700,6 @@ conv_tc_kernel(const TcParams p) {
 }
 
 int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
-FastDiv make_fastdiv(uint32_t d) {
-    FastDiv f;
-    uint32_t shift = 0;
-    while ((1ull << shift) < d) ++shift;
-    f.shift = shift;
-    f.mul = (uint32_t)((((1ull << 32) * ((1ull << shift) - d)) / d) + 1);
-    f.d = d;
-    return f;
-}
 int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
 const void* kernel_for(int mode, int epi) {
@@ -723,10 +711,38 @@ const void* kernel_for(int mode, int epi) {
 constexpr unsigned kSmemMax = 232448u - 1024u;     // opt-in dynamic shared memory per CTA
 constexpr unsigned kSmemPerSm = 233472u;           // 228 KB per SM
 
+// Filters per CTA tile.  At most 128: two CTAs then share an SM's 512 tensor-memory columns, which doubles the
+// epilogue warps and the loads in flight; a 128-wide MMA already runs at the full tensor rate.
+void choose_filter_tile(const ConvArgs& a, int K_pad, int* n_tile_out, int* n_tiles_out) {
+    const int sms = sm_count();
+    const int taps = a.R * a.S;
+    const bool flat = a.stride == 1 && a.P == a.H && a.Q == a.W &&
+                      ((a.R == 1 && a.S == 1 && a.pad == 0) || (a.R == 3 && (a.S == 3 || a.S == 1) && a.pad == 1));
+    const long long m_total = (long long)a.N * (a.P + 2) * (a.Q + 2);
+    const long long m_tiles = (m_total + 127) / 128;
+    int n_tiles = (K_pad + 127) / 128;
+    int n_tile = round_up_i((K_pad + n_tiles - 1) / n_tiles, 16);
+    const long long bank = (long long)taps * a.C_pad * K_pad * 2;
+    if (!(flat && bank <= 100 * 1024)) {
+        // Few position tiles: split the filters over more CTAs, but only while that doubles the SMs in use.  An MMA
+        // costs about the same for 64 filters as for 128, so a split that merely puts two half-width CTAs on an SM
+        // doubles the work (measured, ResNet-18 batch 64: 512->359 filters at 7x7, 72 us split in six, 39 us in three).
+        while (m_tiles * n_tiles * 2 <= sms && n_tile > 64) {
+            n_tiles *= 2;
+            n_tile = round_up_i((K_pad + n_tiles - 1) / n_tiles, 16);
+        }
+    }
+    *n_tile_out = n_tile;
+    *n_tiles_out = (K_pad + n_tile - 1) / n_tile;
+}
+
 }  // namespace
+
+void conv_tc_filter_tile(const ConvArgs& a, int K_pad, int* n_tile, int* n_tiles) { choose_filter_tile(a, K_pad, n_tile, n_tiles); }
 
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len) {
     memset(plan, 0, sizeof(*plan));
+    const int sms = sm_count();
     if (a.C_pad % 16 || a.K_pad % 16) { snprintf(err, err_len, "channel counts must be padded to 16"); return 1; }
     if (a.W > kMaxWidth || a.Q > kMaxWidth) { snprintf(err, err_len, "images wider than %d are not supported", kMaxWidth); return 1; }
     const int cchunks = a.C_pad / 8;
@@ -744,25 +760,17 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (m_total + 128 >= (1ll << 31)) { snprintf(err, err_len, "more than 2^31 output positions"); return 1; }
 
     // --- filter tile ---
-    // at most 128 filters per tile: two CTAs then share an SM's 512 tensor-memory columns, which doubles the
-    // epilogue warps and the loads in flight; a 128-wide MMA already runs at the full tensor rate
-    int n_tiles = (a.K_pad + 127) / 128;
-    int n_tile = round_up_i((a.K_pad + n_tiles - 1) / n_tiles, 16);
+    int n_tile, n_tiles;
+    if (a.n_tile_forced > 0) { n_tile = a.n_tile_forced; n_tiles = (a.K_pad + n_tile - 1) / n_tile; }
+    else choose_filter_tile(a, a.K_pad, &n_tile, &n_tiles);
     const long long bank = (long long)taps * a.C_pad * a.K_pad * 2;
     bool bank_fits = plan->flat && bank <= 100 * 1024;
-    if (!bank_fits) {
-        // Few position tiles: split the filters over more CTAs, but only while that doubles the SMs in use.  An MMA
-        // costs about the same for 64 filters as for 128, so a split that merely puts two half-width CTAs on an SM
-        // doubles the work (measured, ResNet-18 batch 64: 512->359 filters at 7x7, 72 us split in six, 39 us in three).
-        while (m_tiles * n_tiles * 2 <= 148 && n_tile > 64) {
-            n_tiles *= 2;
-            n_tile = round_up_i((a.K_pad + n_tiles - 1) / n_tiles, 16);
-        }
-    }
-    n_tiles = (a.K_pad + n_tile - 1) / n_tile;
     plan->n_tile = n_tile; plan->n_tiles = n_tiles;
 
     unsigned smem = (unsigned)sizeof(Ctrl) + (unsigned)a.K_pad * 4u + 1024u;
+    unsigned scatter_smem = 0;
+    if (a.scatter) scatter_smem = (unsigned)round_up_i((a.out_C_pad + n_tiles + 1) * 4, 16) + 8u * 32u * 33u * 4u;
+    smem += scatter_smem;
     int want_ctas = 1;
     if (plan->flat) {
         plan->halo = ((a.R - 1) / 2) * (a.W + 2) + (a.S - 1) / 2;      // rows above + columns to the left
@@ -780,7 +788,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             for (int tps = 4; tps > 1; tps >>= 1) {
                 const unsigned a_try = (unsigned)(plan->cg * round_up_i(tps * 128 + 2 * plan->halo, 8) * 16);
                 if (2 * tps * n_tile <= 512 && tps * 128 + plan->halo + 8 <= kGuardVectors &&
-                    ((m_tiles + tps - 1) / tps) * n_tiles >= 74 &&
+                    ((m_tiles + tps - 1) / tps) * n_tiles >= sms / 2 &&
                     smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * a_try <= kSmemMax) { plan->tps = tps; break; }
             }
         }
@@ -861,20 +869,15 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     // Wide filter tiles get eight epilogue warps, except in gather mode when there are more tiles than SMs: the
     // eight-warp form needs too many registers for a second CTA on the SM, and a second CTA is what hides the
     // loaders' latency there (measured on ResNet-50, batch 128: every strided layer about 30 % faster with four).
-    const int epi = (n_tile >= 64 && (plan->flat || m_tiles * n_tiles <= 148)) ? 8 : 4;
+    const int epi = (n_tile >= 64 && (plan->flat || m_tiles * n_tiles <= sms)) ? 8 : 4;
     plan->epi_warps = epi;
     const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
     const void* fn = kernel_for(mode, epi);
-    static bool attr_set = false;
-    if (!attr_set) {
-        for (int m = 0; m < 3; ++m)
-            for (int e = 4; e <= 8; e += 4)
-                if (cudaFuncSetAttribute(kernel_for(m, e), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
-                    snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
-                    cudaGetLastError();
-                    return 1;
-                }
-        attr_set = true;
+    // a per-device attribute: set it for the device this plan is made on (cheap, so not cached)
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
+        snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
+        cudaGetLastError();
+        return 1;
     }
     cudaFuncAttributes fa;
     cudaError_t oe = cudaFuncGetAttributes(&fa, fn);
@@ -912,11 +915,12 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
     p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
     p.lut_bytes = plan.flat ? 0 : p.kblocks * 64;
+    p.scatter_bytes = a.scatter ? round_up_i((a.out_C_pad + plan.n_tiles + 1) * 4, 16) + 8 * 32 * 33 * 4 : 0;
     p.status = d_status;
     p.div_ntiles = make_fastdiv((uint32_t)plan.n_tiles);
     p.div_p2out = make_fastdiv((uint32_t)p.P2_out);
     p.div_qp = make_fastdiv((uint32_t)p.Qp);
-    int grid = 148 * plan.ctas_per_sm;
+    int grid = sm_count() * plan.ctas_per_sm;
     if (grid > p.total_tiles) grid = p.total_tiles;
     if (grid < 1) grid = 1;
     cudaLaunchConfig_t cfg;

@@ -21,6 +21,19 @@
 
 namespace fp {
 
+// Streaming multiprocessors of the current device (asked once per device; 148 on a B200).  Grids are sized from it.
+inline int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { cudaGetLastError(); n = 148; }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 constexpr int kGuardVectors = 1024;   // >= 128 + (W + 3) + 8 for every supported width (W <= 512)
 constexpr int kMaxWidth = 512;
 
@@ -37,6 +50,14 @@ struct ConvArgs {
     int relu;
     int res_mode;         // 0 none, 1 same shape as y, 2 subsample + zero-channel pad
     int res_H, res_W, res_C_pad, res_C, res_pad_lo, res_stride;
+    // Scattered output (tensor-core path): the K_pad packed filter rows hold only the kept filters of a convolution
+    // whose output tensor keeps its full width out_C_pad (a residual stream that other layers write too); output
+    // channel c takes accumulator column out_map[c], or only the shortcut when out_map[c] < 0.  Filter tile t
+    // (rows t*n_tile ..) owns the output chunks tile_chunk0[t] .. tile_chunk0[t+1]-1 and holds exactly their filters.
+    int scatter, out_C_pad;
+    const int32_t* out_map;        // [out_C_pad], device
+    const int32_t* tile_chunk0;    // [n_tiles + 1], device
+    int n_tile_forced;             // > 0: filters per CTA tile fixed by the caller (scatter), else chosen by the plan
 };
 
 // Filter preparation --------------------------------------------------------------------
@@ -119,6 +140,8 @@ struct ConvPlanTC {
     unsigned smem_bytes;
     int ctas_per_sm;
 };
+// Filters per CTA tile the plan would choose for K_pad filter rows of this geometry (used to lay out scattered banks).
+void conv_tc_filter_tile(const ConvArgs& a, int K_pad, int* n_tile, int* n_tiles);
 // Returns 0 on success, otherwise writes a message.
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len);
 void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st);

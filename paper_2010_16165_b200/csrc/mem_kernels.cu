@@ -417,7 +417,7 @@ __global__ void planar_to_nchw_f32_kernel(const void* __restrict__ x, float* __r
 
 inline int grid_for(size_t n, int threads) {
     size_t b = (n + threads - 1) / threads;
-    const size_t cap = 148 * 16;
+    const size_t cap = (size_t)sm_count() * 16;
     if (b < 1) b = 1;
     return (int)(b > cap ? cap : b);
 }

@@ -188,8 +188,10 @@ __global__ void repack_chain_kernel(const float* __restrict__ w, int C, const in
 
 // Filters of a 7x7 first convolution in the order the packed network input wants them (see
 // input_to_stem_planar_kernel): a 3x1 convolution over 80 packed channels.  Tap dr (0..2 = offsets
-// -1,0,+1), chunk 0-2 (group E) take filter row r = 2*dr + 1, chunks 3-5 (O') take r = 2*dr, chunks
-// 6-8 (O) take r = 6 at dr = 2 only; packed channel j = s*C + c within a group; everything else zero.
+// -1,0,+1), chunk 0-2 (group E) take filter row r = 2*dr + 1, chunks 3-5 (O') take r = 2*dr at dr = 0, 1,
+// chunks 6-8 (O) take r = 2*dr + 2 at dr = 1, 2; packed channel j = s*C + c within a group; everything else
+// zero.  (Input row 2p+1 is held twice, as O of packed row p and as O' of row p+1; it is taken from row p,
+// because below the last image row there is only the zero border.)
 __global__ void repack_stem_kernel(const float* __restrict__ w, int C, const int32_t* __restrict__ row_src, int K_pad,
                                    __nv_bfloat16* __restrict__ out) {
     const size_t total = (size_t)3 * 10 * K_pad * 8;
@@ -207,8 +209,8 @@ __global__ void repack_stem_kernel(const float* __restrict__ w, int C, const int
             const int sx = j / C, c = j - sx * C;
             int r = -1;
             if (group == 0) r = 2 * dr + 1;
-            else if (group == 1) r = 2 * dr;
-            else if (dr == 2) r = 6;
+            else if (group == 1) { if (dr < 2) r = 2 * dr; }
+            else if (dr >= 1) r = 2 * dr + 2;
             if (r >= 0 && sx < 7) v = w[(((size_t)ks * C + c) * 7 + r) * 7 + sx];
         }
         out[i] = __float2bfloat16_rn(v);
@@ -233,7 +235,8 @@ __global__ void pack_bias_kernel(const float* __restrict__ b, const int32_t* __r
     out[k] = row_src[k] >= 0 ? b[row_src[k]] : 0.0f;
 }
 
-static inline int blocks_for(size_t n, int threads, int cap = 148 * 8) {
+static inline int blocks_for(size_t n, int threads) {
+    const int cap = fp::sm_count() * 8;
     size_t b = (n + threads - 1) / threads;
     if (b < 1) b = 1;
     return (int)(b > (size_t)cap ? cap : b);
