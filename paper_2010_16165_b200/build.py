@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfupruner.so")
-SOURCES = ["api.cu", "prep_kernels.cu", "mem_kernels.cu", "conv_simt.cu", "conv_tc.cu", "chain_tc.cu", "static_rank.cu"]
+SOURCES = ["api.cu", "prep_kernels.cu", "mem_kernels.cu", "conv_simt.cu", "conv_tc.cu", "chain_tc.cu", "stem_pool.cu", "static_rank.cu"]
 
 
 def lib_path():

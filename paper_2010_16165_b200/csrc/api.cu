@@ -99,12 +99,14 @@ struct Chain {
     uint8_t* d_blob = nullptr;
 };
 
-struct Op { int kind; int idx; };   // kind: 0 conv, 1 pool, 2 head, 3 input conversion
+struct Op { int kind; int idx; };
+constexpr int kHostPieces = 8;     // fp_forward_host copies the input in up to this many pieces   // kind: 0 conv, 1 pool, 2 head, 3 input conversion
 
 struct GraphKey {
-    int batch; const void* in; const void* out; cudaStream_t st;
+    int batch; int first; const void* in; const void* out; cudaStream_t st;      // first: first operator of the captured range
     bool operator<(const GraphKey& o) const {
         if (batch != o.batch) return batch < o.batch;
+        if (first != o.first) return first < o.first;
         if (in != o.in) return in < o.in;
         if (out != o.out) return out < o.out;
         return st < o.st;
@@ -140,6 +142,8 @@ struct fp_handle_s {
     void* d_in_stage = nullptr;            // device staging for fp_forward_host
     float* d_logits_stage = nullptr;
     int* d_status = nullptr;
+    cudaStream_t copy_stream = nullptr;    // fp_forward_host: input pieces are copied here while earlier pieces are converted
+    cudaEvent_t copy_events[kHostPieces + 1] = {};
     double* d_scores = nullptr; int32_t* d_rank = nullptr; uint8_t* d_mask = nullptr;
     std::map<GraphKey, cudaGraphExec_t> graphs;
     const void* last_input = nullptr; int last_batch = 0;
@@ -149,6 +153,9 @@ struct fp_handle_s {
     double* d_soft_scores = nullptr; int32_t* d_soft_rank = nullptr; uint8_t* d_soft_mask = nullptr;
     int soft_total = 0;
     int stem_packed = 0;                   // network input stored in the packed form of a 7x7/2 first convolution
+    int stem_fused = 0;                    // operators 0-2 (input conversion, 7x7/2 convolution, 3x3/2 max pooling) run as one kernel
+    fp::StemPoolArgs stem_args;
+    fp::StemPoolPlan stem_plan;
     int scatter_policy = 0;                // fp_model_desc::scatter
     int planned = 0;                       // 1: buffers, packed banks and launch plans match the masks (set by replan)
     int act_is_bf16() const { return compute != FP_COMPUTE_FP32; }
@@ -613,7 +620,7 @@ fp_status upload_i32(fp_handle h, const std::vector<int32_t>& v, int32_t** out) 
 bool chain_candidate(fp_handle h, const FConv& f) {
     if (h->compute != FP_COMPUTE_BF16_TC || h->keep_outputs || f.scatter) return false;
     if (f.R != 3 || f.S != 3 || f.stride != 1 || f.pad != 1) return false;
-    if (h->stem_packed && f.src == 0) return false;
+    if ((h->stem_packed || h->stem_fused) && f.src == 0) return false;
     const Tensor& s = h->tensors[f.src];
     return fp::chain_layer_supported(s.H, s.W, f.K_pad, f.C_pad);
 }
@@ -743,6 +750,17 @@ fp_status replan(fp_handle h) {
         if (f.src == 0 && h->compute == FP_COMPUTE_BF16_TC && uses[0].size() == 1 && f.R == 7 && f.S == 7 &&
             f.stride == 2 && f.pad == 3 && f.C <= 3 && h->in_H % 2 == 0 && h->in_W % 2 == 0)
             h->stem_packed = 1;
+    // ... and, where a 3x3 / stride-2 max pooling is the only reader of that convolution and the input is bf16, input
+    // conversion, convolution and pooling run as one kernel (decided below, once the filter count is known).
+    h->stem_fused = 0;
+    bool stem_candidate = false;
+    if (h->stem_packed && !h->keep_outputs && h->in_dtype == FP_DTYPE_BF16 && h->ops.size() >= 3 && h->ops[1].kind == 0 &&
+        h->ops[2].kind == 1) {
+        const FConv& f = h->convs[h->ops[1].idx];
+        const Pool& pl = h->pools[h->ops[2].idx];
+        stem_candidate = f.src == 0 && f.relu && f.res_mode == 0 && pl.src == f.out && uses[f.out].size() == 1 &&
+                         pl.R == 3 && pl.stride == 2 && pl.pad == 1 && h->in_H % 4 == 0 && h->in_W % 8 == 0;
+    }
     for (const Op& op : h->ops) {
         if (op.kind == 0) {
             FConv& f = h->convs[op.idx];
@@ -775,8 +793,14 @@ fp_status replan(fp_handle h) {
                     fp::conv_tc_filter_tile(ga, K_pad, &nt, &nts);
                     return nts * std::max(nt / 2, 32 + nt / 4);
                 };
+                // And the layer has to fill the GPU more than twice over: with fewer tiles than that, fewer columns only
+                // mean fewer busy SMs, not a shorter kernel (measured, ResNet-18 at batch 64, 512 -> 359 filters at 7x7:
+                // 41 position tiles; 28 us with zero rows on 84 CTAs, 41 us scattered on 63).
+                int nt_s = 0, nts_s = 0;
+                fp::conv_tc_filter_tile(ga, round_up(f.K_kept, 16), &nt_s, &nts_s);
+                const long long m_tiles = ((long long)ga.N * (ga.P + 2) * (ga.Q + 2) + 127) / 128;
                 const bool pays = 5 * pipe_cost(round_up(f.K_kept, 16)) <= 4 * pipe_cost(round_up(f.K, 16)) &&
-                                  ga.R * ga.S * ga.C_pad >= 1024;
+                                  ga.R * ga.S * ga.C_pad >= 1024 && m_tiles * nts_s >= 2 * fp::sm_count();
                 if (!runs_fused && h->scatter_policy >= 0 && (pays || h->scatter_policy > 0)) f.scatter = 1;
             }
             std::vector<int32_t> row_src, chan_src(f.C_pad, -1);
@@ -832,6 +856,32 @@ fp_status replan(fp_handle h) {
                 out.C = f.K_rows; out.C_pad = f.K_pad;
             }
             for (int c = 0; c < src.C; ++c) chan_src[c] = src.keep[c];
+            if (f.src == 0 && stem_candidate && !f.scatter && fp::stem_pool_supported(f.C, h->in_H, h->in_W, f.K_pad)) {
+                h->stem_fused = 1;
+                h->stem_packed = 0;
+                int32_t* d_row;
+                TRY(upload_i32(h, row_src, &d_row));
+                f.d_row = d_row; f.d_chan = nullptr;
+                TRY(dev_alloc(h->pack_buffers, &f.d_wp, (size_t)160 * f.K_pad * 2));
+                TRY(dev_alloc(h->pack_buffers, (void**)&f.d_bp, (size_t)f.K_pad * sizeof(float)));
+                fp::launch_repack_stem_direct(f.d_w32, f.C, d_row, f.K_pad, (__nv_bfloat16*)f.d_wp, st);
+                fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);
+                f.tc.valid = 0;
+                continue;
+            }
+            // launch plan of the tensor-core kernel (geometry only; the pointers follow once memory is planned)
+            f.tc.valid = 0;
+            if (h->compute == FP_COMPUTE_BF16_TC) {
+                fp::ConvArgs ga;
+                memset(&ga, 0, sizeof(ga));
+                conv_geometry(h, f, &ga);
+                ga.C_pad = (h->stem_packed && f.src == 0) ? 80 : f.C_pad;
+                ga.K_pad = f.K_pad;
+                ga.scatter = f.scatter; ga.out_C_pad = out.C_pad; ga.n_tile_forced = f.n_tile_forced;
+                char msg[256];
+                if (fp::plan_conv_tc(ga, &f.tc, msg, sizeof(msg)) != 0)
+                    return fail(FP_ERR_UNSUPPORTED, "convolution %d: %s", f.conv_index, msg);
+            }
             // pack filters and bias
             int32_t *d_row, *d_chan;
             TRY(upload_i32(h, row_src, &d_row));
@@ -845,6 +895,15 @@ fp_status replan(fp_handle h) {
             else fp::launch_repack_conv(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad,
                                    bf16 ? (__nv_bfloat16*)f.d_wp : nullptr, bf16 ? nullptr : (float*)f.d_wp, st);
             fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);
+            if (f.tc.valid && f.tc.blocked_bank) {
+                // the streamed form of the kernel reads its bank block by block: one copy per pipeline stage
+                const int taps = packed_stem ? 3 : f.R * f.S, cchunks = (packed_stem ? 80 : f.C_pad) / 8;
+                void* blocked;
+                TRY(dev_alloc(h->pack_buffers, &blocked, (size_t)f.tc.n_tiles * taps * cchunks * f.tc.n_tile * 16));
+                fp::launch_reblock_bank((const __nv_bfloat16*)f.d_wp, taps, cchunks, f.K_pad, f.tc.n_tile, f.tc.n_tiles, f.tc.cg,
+                                        (__nv_bfloat16*)blocked, st);
+                f.d_wp = blocked;
+            }
         } else if (op.kind == 1) {
             const Pool& p = h->pools[op.idx];
             const Tensor& src = h->tensors[p.src];
@@ -888,6 +947,10 @@ fp_status replan(fp_handle h) {
             else if (op.kind == 0) tid = h->convs[op.idx].out;
             else if (op.kind == 1) tid = h->pools[op.idx].out;
             else if (op.kind == 3) tid = 0;
+            if (h->stem_fused && (i == 0 || i == 1)) {          // neither the converted input nor the first convolution's output exists
+                h->tensors[tid].d = nullptr;
+                continue;
+            }
             if (tid < 0) continue;
             Tensor& t = h->tensors[tid];
             // planar-8 with border, plus guard vectors before and after (halo reads of the first/last tiles)
@@ -929,17 +992,20 @@ fp_status replan(fp_handle h) {
             a.res = r.d; a.res_H = r.H; a.res_W = r.W; a.res_C_pad = r.C_pad; a.res_C = r.C;
             a.res_pad_lo = f.res_pad_lo; a.res_stride = f.res_stride;
         }
-        f.tc.valid = 0;
-        if (h->compute == FP_COMPUTE_BF16_TC) {
-            char msg[256];
-            if (fp::plan_conv_tc(a, &f.tc, msg, sizeof(msg)) != 0)
-                return fail(FP_ERR_UNSUPPORTED, "convolution %d: %s", f.conv_index, msg);
-        }
     }
     for (Chain& ch : h->chains) {
         const FConv& f0 = h->convs[ch.convs.front()];
         const FConv& fl = h->convs[ch.convs.back()];
         ch.args.x = f0.args.x; ch.args.res = f0.args.res; ch.args.y = fl.args.y; ch.args.w = ch.d_blob;
+    }
+    if (h->stem_fused) {
+        const FConv& f = h->convs[h->ops[1].idx];
+        fp::StemPoolArgs& a = h->stem_args;
+        memset(&a, 0, sizeof(a));
+        a.y = h->tensors[h->pools[h->ops[2].idx].out].d; a.w = f.d_wp; a.bias = f.d_bp;
+        a.N = h->max_batch; a.C = f.C; a.H = h->in_H; a.W = h->in_W; a.K_pad = f.K_pad; a.n0 = 0; a.n_count = h->max_batch;
+        char msg[256];
+        if (fp::plan_stem_pool(a, &h->stem_plan, msg, sizeof(msg)) != 0) return fail(FP_ERR_UNSUPPORTED, "%s", msg);
     }
     CK(cudaDeviceSynchronize());
     h->planned = 1;
@@ -956,10 +1022,20 @@ fp_status need_plan(fp_handle h, const char* who) {
 // execution
 // ---------------------------------------------------------------------------------------
 
-void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
+// n0, n_count: the images an input conversion handles (the other operators always run the whole batch)
+void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float* d_logits, cudaStream_t st, int n0 = 0,
+               int n_count = -1) {
+    if (n_count < 0) n_count = batch;
     const Op& op = h->ops[op_index];
     const int bf16 = h->act_is_bf16();
-    if (op.kind == 3 && h->input_fused) return;        // the first fused run reads the network input itself
+    if (op.kind == 3 && (h->input_fused || h->stem_fused)) return;        // the first kernel reads the network input itself
+    if (h->stem_fused && op_index == 2) return;         // pooled inside the first convolution's kernel
+    if (h->stem_fused && op_index == 1) {
+        fp::StemPoolArgs a = h->stem_args;
+        a.x = d_input; a.N = batch; a.n0 = n0; a.n_count = n_count;
+        fp::launch_stem_pool(h->stem_plan, a, h->d_status, st);
+        return;
+    }
     if (op.kind == 0 && h->op_chain[op_index] >= 0) {
         const Chain& ch = h->chains[h->op_chain[op_index]];
         if (op_index != ch.first_op) return;       // the run's first operator launches all of it
@@ -971,8 +1047,8 @@ void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float*
     }
     if (op.kind == 3) {
         const Tensor& t = h->tensors[0];
-        if (h->stem_packed) fp::launch_input_to_stem_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, batch, t.C, t.H, t.W, st);
-        else fp::launch_input_to_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, st);
+        if (h->stem_packed) fp::launch_input_to_stem_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, batch, t.C, t.H, t.W, n0, n_count, st);
+        else fp::launch_input_to_planar(d_input, h->in_dtype == FP_DTYPE_BF16, t.d, bf16, batch, t.C, t.H, t.W, t.C_pad, n0, n_count, st);
     } else if (op.kind == 0) {
         FConv& f = h->convs[op.idx];
         fp::ConvArgs a = f.args;
@@ -990,8 +1066,8 @@ void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float*
     }
 }
 
-void launch_all(fp_handle h, const void* d_input, int batch, float* d_logits, cudaStream_t st) {
-    for (int i = 0; i < (int)h->ops.size(); ++i) launch_op(h, i, d_input, batch, d_logits, st);
+void launch_all(fp_handle h, const void* d_input, int batch, float* d_logits, cudaStream_t st, int first = 0) {
+    for (int i = first; i < (int)h->ops.size(); ++i) launch_op(h, i, d_input, batch, d_logits, st);
 }
 
 fp_status all_ones_masks(fp_handle h) {
@@ -1019,6 +1095,10 @@ extern "C" fp_status fp_destroy(fp_handle h) {
     if (!h) return FP_OK;
     cudaDeviceSynchronize();
     drop_graphs(h);
+    if (h->copy_stream) {
+        cudaStreamDestroy(h->copy_stream);
+        for (cudaEvent_t e : h->copy_events) if (e) cudaEventDestroy(e);
+    }
     free_list(h->act_buffers);
     free_list(h->pack_buffers);
     free_list(h->fixed_buffers);
@@ -1217,32 +1297,27 @@ extern "C" fp_status fp_soft_prune_finish(fp_handle h) {
     return replan(h);
 }
 
-extern "C" fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch, float* d_logits, void* stream) {
-    if (!h || !d_input || !d_logits) return fail(FP_ERR_ARG, "fp_forward: NULL argument");
-    if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward: batch must be positive");
-    if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward: batch %d exceeds max_batch %d", batch, h->max_batch);
-    TRY(need_plan(h, "fp_forward"));
-    cudaStream_t st = (cudaStream_t)stream;
-    h->last_input = d_input; h->last_batch = batch;
+// Operators first .. last of the forward on `st`, as a replayed CUDA graph where the handle asks for one.
+static fp_status forward_from(fp_handle h, const void* d_input, int32_t batch, float* d_logits, cudaStream_t st, int first) {
     const bool graphable = h->use_graph && st != 0 && st != cudaStreamLegacy && st != cudaStreamPerThread;
     if (!graphable) {
-        launch_all(h, d_input, batch, d_logits, st);
+        launch_all(h, d_input, batch, d_logits, st, first);
         CK(cudaGetLastError());
         return FP_OK;
     }
-    GraphKey key{batch, d_input, d_logits, st};
+    GraphKey key{batch, first, d_input, d_logits, st};
     auto it = h->graphs.find(key);
     if (it == h->graphs.end()) {
         cudaStreamCaptureStatus cs;
         CK(cudaStreamIsCapturing(st, &cs));
         if (cs != cudaStreamCaptureStatusNone) {   // already inside someone else's capture: just record the launches
-            launch_all(h, d_input, batch, d_logits, st);
+            launch_all(h, d_input, batch, d_logits, st, first);
             CK(cudaGetLastError());
             return FP_OK;
         }
         cudaGraph_t g;
         CK(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-        launch_all(h, d_input, batch, d_logits, st);
+        launch_all(h, d_input, batch, d_logits, st, first);
         cudaError_t e = cudaStreamEndCapture(st, &g);
         if (e != cudaSuccess) return fail(FP_ERR_CUDA, "graph capture failed: %s", cudaGetErrorString(e));
         cudaGraphExec_t ge;
@@ -1256,15 +1331,51 @@ extern "C" fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch,
     return FP_OK;
 }
 
+extern "C" fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch, float* d_logits, void* stream) {
+    if (!h || !d_input || !d_logits) return fail(FP_ERR_ARG, "fp_forward: NULL argument");
+    if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward: batch must be positive");
+    if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward: batch %d exceeds max_batch %d", batch, h->max_batch);
+    TRY(need_plan(h, "fp_forward"));
+    h->last_input = d_input; h->last_batch = batch;
+    return forward_from(h, d_input, batch, d_logits, (cudaStream_t)stream, 0);
+}
+
 extern "C" fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t batch, float* h_logits, void* stream) {
     if (!h || !h_input || !h_logits) return fail(FP_ERR_ARG, "fp_forward_host: NULL argument");
     if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward_host: batch must be positive");
     if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward_host: batch %d exceeds max_batch %d", batch, h->max_batch);
     TRY(need_plan(h, "fp_forward_host"));
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t in_bytes = (size_t)batch * h->in_C * h->in_H * h->in_W * h->in_elem();
-    CK(cudaMemcpyAsync(h->d_in_stage, h_input, in_bytes, cudaMemcpyHostToDevice, st));
-    TRY(fp_forward(h, h->d_in_stage, batch, h->d_logits_stage, stream));
+    const size_t image_bytes = (size_t)h->in_C * h->in_H * h->in_W * h->in_elem();
+    h->last_input = h->d_in_stage; h->last_batch = batch;
+    // Where the forward starts with a layout conversion of its own, the input crosses the bus in pieces on a second
+    // stream and every piece is converted as soon as it has arrived, so only the last piece's copy is exposed; the
+    // rest of the network then runs once on the whole batch.  (Where the first fused run of layers reads the network
+    // input itself, the input is small: one copy, then the forward.)
+    const int pieces = (h->ops[0].kind == 3 && !h->input_fused && batch >= 2) ? std::min(kHostPieces, batch) : 1;
+    const int piece_op = h->stem_fused ? 1 : 0, tail_op = h->stem_fused ? 3 : 1;     // the kernel that takes the input in; what follows it
+    if (pieces > 1) {
+        if (!h->copy_stream) {
+            CK(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+            for (int i = 0; i <= kHostPieces; ++i) CK(cudaEventCreateWithFlags(&h->copy_events[i], cudaEventDisableTiming));
+        }
+        // the copies must not overtake work already queued on `st` that still reads the staging buffer
+        CK(cudaEventRecord(h->copy_events[kHostPieces], st));
+        CK(cudaStreamWaitEvent(h->copy_stream, h->copy_events[kHostPieces], 0));
+        for (int c = 0; c < pieces; ++c) {
+            const int n0 = (int)((long long)batch * c / pieces), n1 = (int)((long long)batch * (c + 1) / pieces);
+            CK(cudaMemcpyAsync((uint8_t*)h->d_in_stage + (size_t)n0 * image_bytes, (const uint8_t*)h_input + (size_t)n0 * image_bytes,
+                               (size_t)(n1 - n0) * image_bytes, cudaMemcpyHostToDevice, h->copy_stream));
+            CK(cudaEventRecord(h->copy_events[c], h->copy_stream));
+            CK(cudaStreamWaitEvent(st, h->copy_events[c], 0));
+            launch_op(h, piece_op, h->d_in_stage, batch, h->d_logits_stage, st, n0, n1 - n0);
+        }
+        CK(cudaGetLastError());
+        TRY(forward_from(h, h->d_in_stage, batch, h->d_logits_stage, st, tail_op));
+    } else {
+        CK(cudaMemcpyAsync(h->d_in_stage, h_input, (size_t)batch * image_bytes, cudaMemcpyHostToDevice, st));
+        TRY(forward_from(h, h->d_in_stage, batch, h->d_logits_stage, st, 0));
+    }
     CK(cudaMemcpyAsync(h_logits, h->d_logits_stage, (size_t)batch * h->n_classes * sizeof(float), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     return FP_OK;
@@ -1331,6 +1442,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             int n = (int)h->ops.size() + 1;                                  // the head is two kernels
             for (const Chain& ch : h->chains) n -= (int)ch.convs.size() - 1; // a fused run is one
             n -= h->input_fused;
+            n -= 2 * h->stem_fused;                                          // conversion, convolution and pooling are one
             *(int32_t*)h_out = n;
             return FP_OK;
         }
@@ -1369,7 +1481,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             if (h->last_batch <= 0) return fail(FP_ERR_ARG, "fp_query: no forward has run yet");
             TRY(need_plan(h, "fp_query"));
             if (h->ops[index].kind == 3 && h->stem_packed) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is stored in packed form");
-            if (h->ops[index].kind == 3 && h->input_fused) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is converted inside the first fused run "
+            if (h->ops[index].kind == 3 && (h->input_fused || h->stem_fused)) return fail(FP_ERR_UNSUPPORTED, "fp_query: the network input is converted inside the first fused run "
                                                                         "and never stored (set keep_outputs to run every layer on its own)");
             const Op& op = h->ops[index];
             const int tid = op.kind == 0 ? h->convs[op.idx].out : op.kind == 1 ? h->pools[op.idx].out : 0;
@@ -1423,7 +1535,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
                 // first run) adds nothing to the prefix
                 const Op& op = h->ops[i];
                 const bool silent = (op.kind == 0 && h->op_chain[i] >= 0 && h->chains[h->op_chain[i]].first_op != i) ||
-                                    (op.kind == 3 && h->input_fused);
+                                    (op.kind == 3 && (h->input_fused || h->stem_fused)) || (h->stem_fused && i == 2);
                 if (silent) { prefix[i] = i ? prefix[i - 1] : 0.f; continue; }
                 cudaGraph_t g = nullptr;
                 cudaGraphExec_t ge = nullptr;

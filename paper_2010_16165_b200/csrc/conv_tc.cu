@@ -43,7 +43,9 @@ using namespace tc;
 
 constexpr int kMaxStages = 8;
 
-enum { MODE_FLAT_RESIDENT = 0, MODE_FLAT_STREAM = 1, MODE_GATHER = 2 };
+// FLAT_STREAM: activations per K group and filters per (K group, tap) in two rings (convolutions with several taps);
+// FLAT_UNIFIED: one ring whose stages hold a K group's activations and filters together (1x1 convolutions).
+enum { MODE_FLAT_RESIDENT = 0, MODE_FLAT_STREAM = 1, MODE_GATHER = 2, MODE_FLAT_UNIFIED = 3 };
 
 struct TcParams {
     ConvArgs a;
@@ -55,7 +57,9 @@ struct TcParams {
     int n_tile, n_tiles, tmem_cols, total_tiles;
     int tpk, kblocks;                   // gather: taps per K block, K blocks per tile
     int tps;                            // streamed filters: 128-position tiles per pipeline step (share each filter block)
+    int n_producers;                    // streamed filters: producer warps in use (divides a_stages)
     int a_stage_bytes, b_stage_bytes, b_bank_bytes;
+    long long bank_tile_bytes;          // streamed filters: bytes of one filter tile's part of the bank (all taps, all chunks)
     int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
     int scatter_bytes;                  // scattered output: channel -> accumulator column map and the tiles' chunk ranges
     int* status;
@@ -137,12 +141,20 @@ __device__ __forceinline__ void raise(Ctrl* ctrl, int* status, int code) {
 }
 
 // Threads: warp 0 producer, warp 1 MMA, EPI epilogue warps (4, or 8 for wide filter tiles: two warps per
-// TMEM lane quarter, each taking half of the columns), then either 4 loader warps (GATHER) or 1 filter-producer
-// warp and 3 more MMA warps (FLAT_STREAM).  A single thread cannot issue MMAs as fast as the tensor pipe
+// TMEM lane quarter, each taking half of the columns), then either 4 loader warps (GATHER) or 4 filter-producer
+// warps and 3 more MMA warps (FLAT_STREAM).  One thread gets through a (wait, expect, copy) round of the bulk-copy
+// engine in about 500 cycles whatever the copy's size (measured: 4 KB to 32 KB copies all take 530 cycles per round
+// per thread, and the rate scales with the number of threads up to about 100 B/cycle per SM), so the filter blocks
+// of a streamed bank, 12-18 KB each, are issued round-robin by four warps.  A single thread cannot issue MMAs as fast as the tensor pipe
 // retires them (measured: 75-110 cycles per issued MMA against 56-64 of execution at N = 96-128), so in
 // FLAT_STREAM, where one CTA owns the SM, each 128-position tile of a step has an issuing warp of its own.
+constexpr int kProducers = 4;          // unified stages: warp 0 and three more warps issue the stages' copies in turn
+__host__ __device__ constexpr int extra_threads(int mode) {
+    return mode == MODE_FLAT_RESIDENT ? 0 : mode == MODE_FLAT_UNIFIED ? 32 * ((kProducers - 1) + 3) : 128;
+}
+
 template <int MODE, int EPI>
-__global__ void __launch_bounds__(64 + 32 * EPI + (MODE == MODE_FLAT_RESIDENT ? 0 : 128))
+__global__ void __launch_bounds__(64 + 32 * EPI + extra_threads(MODE))
 conv_tc_kernel(const TcParams p) {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
@@ -168,8 +180,12 @@ conv_tc_kernel(const TcParams p) {
     const uint32_t tempty0 = ctrl_addr + (uint32_t)offsetof(Ctrl, tmem_empty);
 
     // MMA-issuing warps: warp 1, plus (streamed filters) the last three warps, one per tile of a step
-    const uint32_t n_issuers = MODE == MODE_FLAT_STREAM ? (uint32_t)p.tps : 1u;
-    const int issuer = warp == 1 ? 0 : (MODE == MODE_FLAT_STREAM && warp >= 3 + EPI) ? warp - (2 + EPI) : -1;
+    const uint32_t n_issuers = (MODE == MODE_FLAT_STREAM || MODE == MODE_FLAT_UNIFIED) ? (uint32_t)p.tps : 1u;
+    const int issuer = warp == 1 ? 0
+                       : (MODE == MODE_FLAT_STREAM && warp >= 3 + EPI) ? warp - (2 + EPI)
+                       : (MODE == MODE_FLAT_UNIFIED && warp >= 1 + EPI + kProducers) ? warp - (EPI + kProducers) : -1;
+    // unified stages: producer warps (warp 0, then the first kProducers - 1 of the extra warps)
+    const int prod = MODE != MODE_FLAT_UNIFIED ? -1 : warp == 0 ? 0 : (warp >= 2 + EPI && warp < 1 + EPI + kProducers) ? warp - (1 + EPI) : -1;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(a_full0 + 8 * s, MODE == MODE_GATHER ? 129 : 1);   // gather: 128 loaders + the filter producer
@@ -229,7 +245,53 @@ conv_tc_kernel(const TcParams p) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    if (warp == 0) {
+    if (MODE == MODE_FLAT_UNIFIED && prod >= 0) {
+        // ------------------------------ producers, unified stages ------------------------------
+        // One stage per (step of tps position tiles, K group): the group's activation rows for all tiles of the step
+        // (one copy per channel chunk) and the group's filters for all taps (one copy: the bank is stored block by
+        // block in this order).  The stages are issued in turn by n_producers warps; that number divides the number of
+        // stages, so a stage is always refilled by the same warp: a warp that ran ahead onto a stage another warp still
+        // has to fill could not tell "two phases behind" from "ready" by the barrier's parity.
+        bool ok = true;
+        uint32_t stage = 0, phase = 0;
+        int turn = 0;
+        const uint32_t stage_bytes = (uint32_t)(p.a_stage_bytes + p.b_stage_bytes);
+        for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+            const int mt = (int)fdiv((uint32_t)tile, p.div_ntiles);
+            const int nt = tile - mt * p.n_tiles;
+            const long long f0 = (long long)mt * p.tps * 128;
+            for (int g = 0; g < p.groups; ++g) {
+                if (turn == prod) {
+                    bool w = true;
+                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w) { ok = false; break; }
+                    int cgg = p.cchunks - g * p.cg;
+                    if (cgg > p.cg) cgg = p.cg;
+                    const uint32_t fb = a_full0 + 8 * stage;
+                    const uint32_t dst = a_base + stage * stage_bytes;
+                    const uint32_t b_bytes = (uint32_t)(p.taps * cgg * p.n_tile * 16);
+                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16) + b_bytes);
+                    __syncwarp();
+                    if (lane < cgg)
+                        bulk_copy(dst + lane * p.rows_a * 16, xv + (long long)(g * p.cg + lane) * p.plane_in + f0 - p.halo,
+                                  (uint32_t)(p.rows_a * 16), fb);
+                    else if (lane >= 16) {
+                        // the group's filter block is one contiguous run of the bank: pieces of 16 KB, one per lane
+                        const uint32_t off = (uint32_t)(lane - 16) * 16384u;
+                        if (off < b_bytes)
+                            bulk_copy(dst + (uint32_t)p.a_stage_bytes + off,
+                                      reinterpret_cast<const uint8_t*>(p.a.w) + (long long)nt * p.bank_tile_bytes +
+                                          (long long)p.taps * (g * p.cg) * p.n_tile * 16 + off,
+                                      b_bytes - off < 16384u ? b_bytes - off : 16384u, fb);
+                    }
+                }
+                if (++turn == p.n_producers) turn = 0;
+                if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
+            }
+        }
+        if (!ok && lane == 0) raise(ctrl, p.status, 1);
+    } else if (warp == 0) {
         // ------------------------------ bulk-copy producer ------------------------------
         if (MODE != MODE_GATHER) {
             // One lane per channel chunk issues that chunk's copy, so the copies of a K block are issued
@@ -307,7 +369,33 @@ conv_tc_kernel(const TcParams p) {
                 const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.tps * p.n_tile);
                 uint32_t accumulate = 0;
-                if (MODE != MODE_GATHER) {
+                if (MODE == MODE_FLAT_UNIFIED) {
+                    // one wait and one commit per stage; each tile of the step has its own issuing warp and accumulator
+                    const uint32_t stage_bytes = (uint32_t)(p.a_stage_bytes + p.b_stage_bytes);
+                    const uint32_t a_ks = 2u * (uint32_t)p.rows_a, b_ks = 2u * (uint32_t)p.n_tile;
+                    const uint32_t d_acc = d_tmem + (uint32_t)(issuer * p.n_tile);
+                    for (int g = 0; g < p.groups && ok; ++g) {
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        int cgg = p.cchunks - g * p.cg;
+                        if (cgg > p.cg) cgg = p.cg;
+                        const int ksteps = cgg >> 1;
+                        const uint32_t sa = a_base + a_stage * stage_bytes;
+                        uint32_t a_row = ((sa >> 4) + (uint32_t)(issuer * 128)) | ((uint32_t)p.rows_a << 16);
+                        uint32_t b_lo = ((sa + (uint32_t)p.a_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
+                        const uint32_t b_tap = (uint32_t)(cgg * p.n_tile);
+                        for (int r = 0; r < p.a.R; ++r) {
+                            for (int sx = 0; sx < p.a.S; ++sx) {
+                                issue_ksteps(ksteps, d_acc, a_row + (uint32_t)sx, b_lo, a_ks, b_ks, idesc, accumulate);
+                                accumulate = 1;
+                                b_lo += b_tap;
+                            }
+                            a_row += (uint32_t)p.Wp_in;
+                        }
+                        umma_commit(a_empty0 + 8 * a_stage);     // releases the stage once these MMAs have read it
+                        if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
+                    }
+                } else if (MODE != MODE_GATHER) {
                     // Descriptors differ only in their 16-byte start-address field, so the inner loops
                     // just add row counts to the low word (rows are 16 bytes: one row = one address unit).
                     for (int g = 0; g < p.groups && ok; ++g) {
@@ -334,24 +422,16 @@ conv_tc_kernel(const TcParams p) {
                         } else
                         for (int r = 0; r < p.a.R && ok; ++r) {
                             for (int sx = 0; sx < p.a.S; ++sx) {
-                                uint32_t a_lo = a_row + (uint32_t)sx;
-                                uint32_t b_lo = b_tap;
-                                if (MODE == MODE_FLAT_STREAM) {
-                                    if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag)) { ok = false; break; }
-                                    tc_fence_after();
-                                    b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
-                                }
-                                // every 128-position tile of the step uses this filter block: its own accumulator
-                                // and issuing warp, its activation rows 128 further on
-                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_lo + (uint32_t)(issuer * 128), b_lo,
+                                // streamed filters: one block per (K group, tap).  Every 128-position tile of the step
+                                // uses it: its own accumulator and issuing warp, its activation rows 128 further on
+                                if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag)) { ok = false; break; }
+                                tc_fence_after();
+                                const uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
+                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_row + (uint32_t)sx + (uint32_t)(issuer * 128), b_lo,
                                              a_ks, b_ks, idesc, accumulate);
                                 accumulate = 1;
-                                if (MODE == MODE_FLAT_STREAM) {
-                                    umma_commit(b_empty0 + 8 * b_stage);
-                                    if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
-                                } else {
-                                    b_tap += b_tap_step;
-                                }
+                                umma_commit(b_empty0 + 8 * b_stage);
+                                if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
                             }
                             a_row += (uint32_t)p.Wp_in;
                         }
@@ -705,6 +785,7 @@ int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 const void* kernel_for(int mode, int epi) {
     if (mode == MODE_FLAT_RESIDENT) return epi == 8 ? (const void*)conv_tc_kernel<MODE_FLAT_RESIDENT, 8> : (const void*)conv_tc_kernel<MODE_FLAT_RESIDENT, 4>;
     if (mode == MODE_FLAT_STREAM) return epi == 8 ? (const void*)conv_tc_kernel<MODE_FLAT_STREAM, 8> : (const void*)conv_tc_kernel<MODE_FLAT_STREAM, 4>;
+    if (mode == MODE_FLAT_UNIFIED) return epi == 8 ? (const void*)conv_tc_kernel<MODE_FLAT_UNIFIED, 8> : (const void*)conv_tc_kernel<MODE_FLAT_UNIFIED, 4>;
     return epi == 8 ? (const void*)conv_tc_kernel<MODE_GATHER, 8> : (const void*)conv_tc_kernel<MODE_GATHER, 4>;
 }
 
@@ -750,10 +831,6 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     plan->flat = (a.stride == 1 && a.P == a.H && a.Q == a.W &&
                   ((a.R == 1 && a.S == 1 && a.pad == 0) || (a.R == 3 && (a.S == 3 || a.S == 1) && a.pad == 1))) ? 1 : 0;
     plan->cg = cchunks < 8 ? cchunks : 8;
-    // Streamed filters: every filter block costs the issuing thread a barrier test, a fence and a commit on top
-    // of its MMAs, so blocks of 12 chunks (six MMAs) instead of 8 (measured on ResNet-18, batch 64: the streamed
-    // layers 8-15 % faster; 16 chunks need so much shared memory that multi-tile steps no longer fit).
-    if (plan->flat && (long long)taps * a.C_pad * a.K_pad * 2 > 100 * 1024) plan->cg = cchunks < 12 ? cchunks : 12;
     plan->groups = (cchunks + plan->cg - 1) / plan->cg;
     const long long m_total = (long long)a.N * (a.P + 2) * (a.Q + 2);
     const long long m_tiles = (m_total + 127) / 128;
@@ -780,7 +857,49 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         // streamed form, whose steps of several tiles share one halo, even though its filters would fit
         // (measured on the ResNet-18 stem at batch 64: 89 us resident, 61 us streamed).
         const bool wide_halo = 2 * plan->halo > 128;
-        if (!bank_fits || wide_halo) {
+        bool stream = !bank_fits || wide_halo;
+        const bool unified = stream && taps == 1;
+        if (unified) {
+            // 1x1 convolutions with a streamed bank.  A stage holds one K group of channel chunks: its activation
+            // rows for the `tps` position tiles of a step and its filters - one wait and one commit per stage for the
+            // issuing threads, one expected-bytes arrival for the producer.  The K group is the largest that still
+            // leaves three stages (two in flight while one is read: at 60-100 B/cycle and a latency of one or two
+            // thousand cycles about 100 KB have to be in flight), since every stage costs its producer and the
+            // issuing threads a fixed 300-500 cycles.  (Measured on ResNet-50, batch 128: the 1024 -> 154 layers
+            // 30.9 -> 23.3 us, 512 -> 154 54 -> 40 us.  With several taps a stage would have to hold all taps' filters,
+            // which leaves room for two or three K-chunk pairs only: such layers were up to 1.7x slower this way and
+            // keep the two-ring form below.)
+            const unsigned avail = kSmemMax - smem;
+            int best_tps = 0, best_cg = 0, best_stages = 0;
+            for (int tps = 4; tps >= 1 && !best_tps; tps >>= 1) {
+                if (2 * tps * n_tile > 512 || tps * 128 + plan->halo + 8 > kGuardVectors) continue;
+                if (tps > 1 && ((m_tiles + tps - 1) / tps) * n_tiles < sms / 2) continue;
+                const int rows = round_up_i(tps * 128 + 2 * plan->halo, 8);
+                for (int cg = (cchunks < 16 ? cchunks : 16) & ~1; cg >= 2; cg -= 2) {
+                    const unsigned st = (unsigned)(cg * rows * 16 + taps * cg * n_tile * 16);
+                    int stages = (int)(avail / st);
+                    if (stages > kMaxStages) stages = kMaxStages;
+                    if (stages == 7) stages = 6;          // the producer warps (2, 3 or 4 of them) must divide the stages
+                    if (stages == 5) stages = 4;
+                    const int groups = (cchunks + cg - 1) / cg;
+                    if (stages >= (groups >= 3 ? 3 : 2)) { best_tps = tps; best_cg = cg; best_stages = stages; break; }
+                }
+            }
+            if (!best_tps) { snprintf(err, err_len, "tile does not fit shared memory"); return 1; }
+            plan->tps = best_tps; plan->cg = best_cg; plan->a_stages = best_stages;
+            plan->groups = (cchunks + best_cg - 1) / best_cg;
+            plan->rows_a = round_up_i(plan->tps * 128 + 2 * plan->halo, 8);
+            plan->b_resident = 0;
+            plan->b_stages = 0;
+            plan->blocked_bank = 1;
+            bank_fits = false;
+            smem += (unsigned)plan->a_stages * (unsigned)(plan->cg * plan->rows_a * 16 + taps * plan->cg * n_tile * 16);
+        } else {
+        if (stream) {
+            // Streamed filters: every filter block costs the issuing thread a barrier test, a fence and a commit on top
+            // of its MMAs, so blocks of 12 chunks (six MMAs) instead of 8 (measured on ResNet-18, batch 64: the streamed
+            // layers 8-15 % faster; 16 chunks need so much shared memory that multi-tile steps no longer fit).
+            if (!bank_fits) { plan->cg = cchunks < 12 ? cchunks : 12; plan->groups = (cchunks + plan->cg - 1) / plan->cg; }
             // Several 128-position tiles per step share every streamed filter block.  Layers with few positions
             // and many filters re-stream the bank once per position tile and are bound by L2 bandwidth, so
             // sharing pays even when it leaves only half of the SMs with a CTA (measured, same network: 368->512
@@ -788,7 +907,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             for (int tps = 4; tps > 1; tps >>= 1) {
                 const unsigned a_try = (unsigned)(plan->cg * round_up_i(tps * 128 + 2 * plan->halo, 8) * 16);
                 if (2 * tps * n_tile <= 512 && tps * 128 + plan->halo + 8 <= kGuardVectors &&
-                    ((m_tiles + tps - 1) / tps) * n_tiles >= sms / 2 &&
+                    ((m_tiles + tps - 1) / tps) * n_tiles >= sms * 2 / 5 &&
                     smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * a_try <= kSmemMax) { plan->tps = tps; break; }
             }
         }
@@ -829,6 +948,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             while (plan->a_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->a_stages;
             while (plan->b_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->b_stages;
             smem += (unsigned)round_up_i((int)(plan->b_stages * b_stage), 128) + plan->a_stages * a_stage;
+        }
         }
         want_ctas = 4;
     } else {
@@ -871,7 +991,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     // loaders' latency there (measured on ResNet-50, batch 128: every strided layer about 30 % faster with four).
     const int epi = (n_tile >= 64 && (plan->flat || m_tiles * n_tiles <= sms)) ? 8 : 4;
     plan->epi_warps = epi;
-    const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
+    const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : plan->blocked_bank ? MODE_FLAT_UNIFIED : MODE_FLAT_STREAM;
     const void* fn = kernel_for(mode, epi);
     // a per-device attribute: set it for the device this plan is made on (cheap, so not cached)
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
@@ -882,7 +1002,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     cudaFuncAttributes fa;
     cudaError_t oe = cudaFuncGetAttributes(&fa, fn);
     if (oe != cudaSuccess) { snprintf(err, err_len, "cudaFuncGetAttributes: %s", cudaGetErrorString(oe)); cudaGetLastError(); return 1; }
-    const int threads = 64 + 32 * epi + (mode == MODE_FLAT_RESIDENT ? 0 : 128);
+    const int threads = 64 + 32 * epi + extra_threads(mode);
     const int regs_per_warp = round_up_i(fa.numRegs * 32, 256);
     int occ = 65536 / (regs_per_warp * (threads / 32));
     if (occ > 2048 / threads) occ = 2048 / threads;
@@ -907,10 +1027,12 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.n_tile = plan.n_tile; p.n_tiles = plan.n_tiles; p.tmem_cols = plan.tmem_cols;
     const long long m_tiles = (p.m_total + 127) / 128;
     p.tps = plan.tps > 0 ? plan.tps : 1;
+    p.n_producers = plan.a_stages % 4 == 0 ? 4 : plan.a_stages % 3 == 0 ? 3 : plan.a_stages % 2 == 0 ? 2 : 1;
     p.total_tiles = (int)(((m_tiles + p.tps - 1) / p.tps) * plan.n_tiles);
     const int gplanes = plan.groups > 1 ? plan.cg : plan.tpk * p.cchunks;      // gather: planes per stage
     p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : gplanes * 128 * 16;
-    p.b_stage_bytes = plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
+    p.b_stage_bytes = plan.blocked_bank ? p.taps * plan.cg * plan.n_tile * 16 : plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
+    p.bank_tile_bytes = (long long)p.taps * p.cchunks * plan.n_tile * 16;
     p.tpk = plan.tpk > 0 ? plan.tpk : 1;
     p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
     p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
@@ -926,8 +1048,8 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
-    const int mode = !plan.flat ? MODE_GATHER : plan.b_resident ? MODE_FLAT_RESIDENT : MODE_FLAT_STREAM;
-    cfg.blockDim = dim3((unsigned)(64 + 32 * plan.epi_warps + (mode == MODE_FLAT_RESIDENT ? 0 : 128)));
+    const int mode = !plan.flat ? MODE_GATHER : plan.b_resident ? MODE_FLAT_RESIDENT : plan.blocked_bank ? MODE_FLAT_UNIFIED : MODE_FLAT_STREAM;
+    cfg.blockDim = dim3((unsigned)(64 + 32 * plan.epi_warps + extra_threads(mode)));
     cfg.dynamicSmemBytes = plan.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -94,6 +94,11 @@ void launch_soft_zeroize(const SoftBank* banks, const int32_t* filter_bank, int 
 // Convolution filters: packed[rs][cp/8][kr][cp%8] = w[row_src[kr]][chan_src[cp]][rs] (zero where an index is -1)
 void launch_repack_conv(const float* w, int C, int RS, const int32_t* row_src, int K_pad, const int32_t* chan_src,
                         int C_pad, __nv_bfloat16* out_bf16, float* out_f32, cudaStream_t st);
+// Streamed filter bank: from packed[rs][cp/8][K_pad][8] to blocks in the order the tensor-core kernel streams them,
+// blocked[filter tile t][K group g][rs][chunk in group][row in tile][8] (groups of `cg` chunks, the last one shorter;
+// tiles of `n_tile` rows, rows past K_pad zero): n_tiles * RS * (C_pad/8) * n_tile * 8 elements
+void launch_reblock_bank(const __nv_bfloat16* packed, int RS, int cchunks, int K_pad, int n_tile, int n_tiles, int cg,
+                         __nv_bfloat16* blocked, cudaStream_t st);
 // FC matrix: packed[k][cp] = w[k][chan_src[cp]] * scale
 void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int C_pad, float scale, float* out,
                       cudaStream_t st);
@@ -106,9 +111,11 @@ void launch_repack_chain(const float* w, int C, const int32_t* row_src, int K_pa
                          __nv_bfloat16* out, cudaStream_t st);
 
 // Memory-bound operators ------------------------------------------------------------------
+// Both convert images n0 .. n0 + n_count - 1 of a batch of N images (`in` and `out` are the whole batch's buffers).
 void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
-                            int C_pad, cudaStream_t st);
-void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, cudaStream_t st);
+                            int C_pad, int n0, int n_count, cudaStream_t st);
+void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, int n0, int n_count,
+                                 cudaStream_t st);
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,
                     int stride, int pad, cudaStream_t st);
 void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
@@ -127,6 +134,7 @@ struct ConvPlanTC {
     int flat;             // 1: stride-1 "same" convolution, activation tiles fetched as contiguous runs
                           //    of flat positions (bulk copies); 0: gathered by loader threads
     int b_resident;       // flat only: the whole filter bank stays in shared memory
+    int blocked_bank;     // streamed filters: the bank must be stored block by block (launch_reblock_bank)
     int cg;               // channel chunks (of 8) per K block
     int groups;           // K blocks per filter tap = ceil((C_pad/8) / cg)
     int halo;             // flat: vectors fetched before and after the 128 positions of a tile
@@ -145,6 +153,23 @@ void conv_tc_filter_tile(const ConvArgs& a, int K_pad, int* n_tile, int* n_tiles
 // Returns 0 on success, otherwise writes a message.
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len);
 void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st);
+
+// First convolution (7x7 / stride 2 / pad 3, at most 3 input channels, ReLU) and the 3x3 / stride 2 / pad 1 max pooling
+// behind it as one kernel that reads the NCHW bf16 network input and writes the pooled tensor.
+struct StemPoolArgs {
+    const void* x;        // network input, N x C x H x W, NCHW, bf16
+    void* y;              // pooled tensor, planar-8 with border, (H/4) x (W/4) pixels, K_pad channels, N images
+    const void* w;        // filters [20 chunks of 8 k][K_pad rows][8] bf16, k = (r * 7 + s) * C + c, zero for k >= 49 C
+    const float* bias;    // [K_pad]
+    int N, C, H, W, K_pad;
+    int n0, n_count;      // the images this launch handles (the tensor's plane pitch is that of all N)
+};
+struct StemPoolPlan { int valid, tiles, tmem_cols; unsigned smem_bytes; };
+bool stem_pool_supported(int C, int H, int W, int K_pad);
+int plan_stem_pool(const StemPoolArgs& a, StemPoolPlan* plan, char* err, size_t err_len);
+void launch_stem_pool(const StemPoolPlan& plan, const StemPoolArgs& a, int* d_status, cudaStream_t st);
+// its filters: out[k / 8][kr][k % 8] = w[row_src[kr]][c][r][s] with k = (r * 7 + s) * C + c (zero rows / zero k padding)
+void launch_repack_stem_direct(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st);
 
 // A run of stride-1 3x3 convolutions executed by one kernel with the activations in shared memory.
 constexpr int kChainMaxLayers = 40;

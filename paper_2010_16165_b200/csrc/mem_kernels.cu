@@ -41,17 +41,20 @@ __device__ __forceinline__ void store_vec8(void* base, size_t vec, const float (
 
 // NCHW (fp32 or bf16) -> planar-8 with border.  Thread = (chunk, flat position); reads of one
 // channel plane are coalesced along w, writes are contiguous vectors.
+// Images n0 .. n0 + n_count - 1 of a batch of N (the others are left alone: a caller that receives its input in
+// pieces converts each piece as it arrives).
 template <bool OUT_BF16>
 __global__ void input_to_planar_kernel(const void* __restrict__ in, int in_is_bf16, void* __restrict__ out, int N, int C,
-                                       int H, int W, int chunks) {
+                                       int H, int W, int chunks, int n0, int n_count) {
     const int Wp = W + 2, P2 = (H + 2) * Wp;
     const size_t plane = (size_t)N * P2;
-    const size_t total = plane * chunks;
+    const size_t part = (size_t)n_count * P2;
+    const size_t total = part * chunks;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int j = (int)(i / plane);
-        const size_t f = i - (size_t)j * plane;
-        const size_t n = f / P2;
-        const int rem = (int)(f - n * P2);
+        const int j = (int)(i / part);
+        const size_t f = i - (size_t)j * part;
+        const size_t n = n0 + f / P2;
+        const int rem = (int)(f % P2);
         const int h = rem / Wp - 1, w = rem % Wp - 1;
         float v[8];
 #pragma unroll
@@ -66,7 +69,7 @@ __global__ void input_to_planar_kernel(const void* __restrict__ in, int in_is_bf
                 }
             }
         }
-        store_vec8<OUT_BF16>(out, i, v);
+        store_vec8<OUT_BF16>(out, (size_t)j * plane + n * P2 + rem, v);
     }
 }
 
@@ -78,16 +81,16 @@ __global__ void input_to_planar_kernel(const void* __restrict__ in, int in_is_bf
 //     O'(chunks 3-5):  O'[p][q][j] = x[c][2p - 1][2q + s - 3]      (odd rows, shifted down by one)
 //     O (chunks 6-8):  O [p][q][j] = x[c][2p + 1][2q + s - 3]
 // (chunk 9 is zero padding to an even chunk count).  Output row p needs input rows 2p-3 .. 2p+3, which
-// are O'(p-1), E(p-1), O'(p), E(p), O'(p+1), E(p+1), O(p+1): vertical offsets -1, 0, +1 only.
+// are O'(p-1), E(p-1), O'(p), E(p), O(p), E(p+1), O(p+1): vertical offsets -1, 0, +1 only.
 // One block per (image, output row incl. the two border rows): the three input rows the output row needs are
 // staged in shared memory (coalesced reads, each input element read once per block), then every thread builds
 // packed vectors from them.  32-bit index arithmetic only.
 __global__ void input_to_stem_planar_kernel(const void* __restrict__ in, int in_is_bf16, __nv_bfloat16* __restrict__ out,
-                                            int N, int C, int H, int W) {
+                                            int N, int C, int H, int W, int n0) {
     extern __shared__ float rows[];                  // [3 rows: 2p-1, 2p, 2p+1][C][W + 6], zero where outside the image
     __shared__ int tap_off[24];                      // packed channel j = s*C + c -> c*(W+6) + s, or -1 (padding)
     const int P = H / 2, Q = W / 2, Qp = Q + 2, P2 = (P + 2) * Qp;
-    const int n = blockIdx.x / (P + 2), pp = blockIdx.x - n * (P + 2);
+    const int n = n0 + blockIdx.x / (P + 2), pp = blockIdx.x % (P + 2);
     const int p = pp - 1;
     const size_t plane = (size_t)N * P2;
     uint4* outv = reinterpret_cast<uint4*>(out) + (size_t)n * P2 + (size_t)pp * Qp;
@@ -142,11 +145,11 @@ __global__ void input_to_stem_planar_kernel(const void* __restrict__ in, int in_
 // are compile-time constants, so a vector is eight shared-memory loads at immediate offsets (no table, no
 // divisions), and the rows are staged row by row.  One thread per output column.
 __global__ void input_to_stem_planar_rgb_kernel(const void* __restrict__ in, int in_is_bf16, __nv_bfloat16* __restrict__ out,
-                                                int N, int H, int W) {
+                                                int N, int H, int W, int n0) {
     constexpr int C = 3;
     extern __shared__ float rows[];                  // [3 rows: 2p-1, 2p, 2p+1][C][W + 6], zero where outside the image
     const int P = H / 2, Q = W / 2, Qp = Q + 2, P2 = (P + 2) * Qp;
-    const int n = blockIdx.x / (P + 2), pp = blockIdx.x - n * (P + 2);
+    const int n = n0 + blockIdx.x / (P + 2), pp = blockIdx.x % (P + 2);
     const int p = pp - 1;
     const size_t plane = (size_t)N * P2;
     Vec8h* outv = reinterpret_cast<Vec8h*>(out) + (size_t)n * P2 + (size_t)pp * Qp;
@@ -425,16 +428,17 @@ inline int grid_for(size_t n, int threads) {
 }  // namespace
 
 void launch_input_to_planar(const void* in, int in_is_bf16, void* out, int out_is_bf16, int N, int C, int H, int W,
-                            int C_pad, cudaStream_t st) {
-    const size_t n = (size_t)N * (H + 2) * (W + 2) * (C_pad / 8);
-    if (out_is_bf16) input_to_planar_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8);
-    else input_to_planar_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8);
+                            int C_pad, int n0, int n_count, cudaStream_t st) {
+    const size_t n = (size_t)n_count * (H + 2) * (W + 2) * (C_pad / 8);
+    if (out_is_bf16) input_to_planar_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8, n0, n_count);
+    else input_to_planar_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(in, in_is_bf16, out, N, C, H, W, C_pad / 8, n0, n_count);
 }
 
-void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, cudaStream_t st) {
+void launch_input_to_stem_planar(const void* in, int in_is_bf16, void* out, int N, int C, int H, int W, int n0, int n_count,
+                                 cudaStream_t st) {
     const size_t smem = (size_t)3 * C * (W + 6) * sizeof(float);      // <= 36 KB for the supported widths
-    if (C == 3) input_to_stem_planar_rgb_kernel<<<N * (H / 2 + 2), 128, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, H, W);
-    else input_to_stem_planar_kernel<<<N * (H / 2 + 2), 256, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W);
+    if (C == 3) input_to_stem_planar_rgb_kernel<<<n_count * (H / 2 + 2), 128, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, H, W, n0);
+    else input_to_stem_planar_kernel<<<n_count * (H / 2 + 2), 256, smem, st>>>(in, in_is_bf16, (__nv_bfloat16*)out, N, C, H, W, n0);
 }
 
 void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, int C_pad, int P, int Q, int R,

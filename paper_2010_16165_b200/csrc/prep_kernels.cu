@@ -217,6 +217,45 @@ __global__ void repack_stem_kernel(const float* __restrict__ w, int C, const int
     }
 }
 
+__global__ void repack_stem_direct_kernel(const float* __restrict__ w, int C, const int32_t* __restrict__ row_src, int K_pad,
+                                          __nv_bfloat16* __restrict__ out) {
+    const int total = 20 * K_pad * 8;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const int e = i % 8, kr = (i / 8) % K_pad, chunk = i / (8 * K_pad);
+        const int k = chunk * 8 + e;
+        float v = 0.0f;
+        const int ks = row_src[kr];
+        if (ks >= 0 && k < 49 * C) {
+            const int r = k / (7 * C), rem = k - r * 7 * C, s = rem / C, c = rem - s * C;
+            v = w[(((size_t)ks * C + c) * 7 + r) * 7 + s];
+        }
+        out[i] = __float2bfloat16_rn(v);
+    }
+}
+
+__global__ void reblock_bank_kernel(const uint4* __restrict__ packed, int RS, int cchunks, int K_pad, int n_tile, int n_tiles,
+                                    int cg, uint4* __restrict__ blocked) {
+    const size_t total = (size_t)n_tiles * RS * cchunks * n_tile;          // 16-byte rows
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        // i = ((t * cchunks*RS ... decoded block by block: tile t, then group g (cgg chunks), tap, chunk, row
+        const size_t per_tile = (size_t)RS * cchunks * n_tile;
+        const int t = (int)(i / per_tile);
+        size_t r = i - (size_t)t * per_tile;
+        const size_t full_group = (size_t)RS * cg * n_tile;
+        const int g = (int)(r / full_group);
+        r -= (size_t)g * full_group;
+        int cgg = cchunks - g * cg;
+        if (cgg > cg) cgg = cg;
+        const int tap = (int)(r / ((size_t)cgg * n_tile));
+        r -= (size_t)tap * cgg * n_tile;
+        const int c = (int)(r / n_tile), row = (int)(r - (size_t)c * n_tile);
+        const int k = t * n_tile + row;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (k < K_pad) v = packed[((size_t)tap * cchunks + (g * cg + c)) * K_pad + k];
+        blocked[i] = v;
+    }
+}
+
 __global__ void repack_fc_kernel(const float* __restrict__ w, int C, int K, const int32_t* __restrict__ chan_src,
                                  int C_pad, float scale, float* __restrict__ out) {
     const size_t total = (size_t)K * C_pad;
@@ -301,6 +340,16 @@ void launch_repack_chain(const float* w, int C, const int32_t* row_src, int K_pa
 
 void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st) {
     repack_stem_kernel<<<blocks_for((size_t)240 * K_pad, 256), 256, 0, st>>>(w, C, row_src, K_pad, out);
+}
+
+void launch_repack_stem_direct(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st) {
+    repack_stem_direct_kernel<<<blocks_for((size_t)160 * K_pad, 256), 256, 0, st>>>(w, C, row_src, K_pad, out);
+}
+
+void launch_reblock_bank(const __nv_bfloat16* packed, int RS, int cchunks, int K_pad, int n_tile, int n_tiles, int cg,
+                         __nv_bfloat16* blocked, cudaStream_t st) {
+    const size_t n = (size_t)n_tiles * RS * cchunks * n_tile;
+    reblock_bank_kernel<<<blocks_for(n, 256), 256, 0, st>>>((const uint4*)packed, RS, cchunks, K_pad, n_tile, n_tiles, cg, (uint4*)blocked);
 }
 
 void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int C_pad, float scale, float* out,

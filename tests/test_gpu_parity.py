@@ -425,7 +425,7 @@ def _compare_stored_ops(B, g, w, gp, fpo, idx):
         try:
             got = B.fp_query_array(g.h, B.FP_Q_OP_OUTPUT, i, np.float32, n_img * C * info.P * info.Q)
         except B.FpError as e:
-            assert e.status == B.FP_ERR_UNSUPPORTED and info.chain >= 0      # inside a fused run: never stored
+            assert e.status == B.FP_ERR_UNSUPPORTED      # inside a fused run, or pooled inside the first convolution's kernel: never stored
             continue
         got = got.reshape((n_img,) + ref.shape[1:])[idx].astype(np.float64)
         e = np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30)
@@ -494,12 +494,23 @@ def test_config3_resnet110_b1024(B, fpo):
 def test_config4_resnet18_b64(B, fpo):
     w = wl.workload(4)
     _full_config(B, fpo, w, 2, stored_ops=True)
-    # the last stage's second convolutions keep 359 of 512 filters and compute only those (scattered output)
-    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC)
+
+
+def test_wide_stream_writers_compute_kept_filters_only(B, fpo):
+    """ResNet-18 at batch 256: the last stage's second convolutions keep 359 of 512 filters and, with enough position
+    tiles to fill the GPU several times over, compute only those (scattered output); the result still equals the oracle's
+    removal.  (At batch 64 the same layers have 41 position tiles and keep zero rows: fewer columns would only idle SMs.)"""
+    w = wl.workload(4, batch=256)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, use_graph=1)
     try:
         B.fp_prune(g.h, w.ratios)
+        got = g.forward(w.x, torch.cuda.Stream())
         wide = [o for o in B.op_infos(g.h) if o.kind == 0 and o.res_mode == 1 and o.K == 359]
         assert wide and all(o.K_pad <= 384 for o in wide), [(o.K, o.K_pad) for o in wide]
+        idx = [0, 255]
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        assert err(got[idx], fpo.fused_forward(gp, w.x[idx])) < TOL_BF16
+        assert _compare_stored_ops(B, g, w, gp, fpo, idx) >= 2
     finally:
         g.close()
 
@@ -540,6 +551,46 @@ def test_config1_aggressive_fused_unpruned_and_pruned(B, fpo):
         assert err(g.forward(w.x), fpo.fused_forward(gp, w.x)) < TOL_BF16
         for ci, m in B.masks_and_ranks(g.h).items():
             np.testing.assert_array_equal(m[0], masks[ci])
+    finally:
+        g.close()
+
+
+def _stem_net(H, W, K, in_C=3, name="stem_pool"):
+    net = wl.Net(in_C, H, W, name)
+    x = net.relu(net.bn(net.conv(-1, K, in_C, 7, 2, 3), K))
+    x = net.maxpool(x, K)
+    x = net.relu(net.bn(net.conv(x, 24, K, 3, 1, 1), 24))
+    x = net.gavgpool(x, 24)
+    net.fc(x, 6, 24)
+    net.n_blocks = 0
+    return net
+
+
+@pytest.mark.parametrize("shape", [(32, 32, 16, 3, 2), (36, 64, 40, 3, 5), (24, 112, 64, 3, 3), (16, 8, 16, 1, 2), (224, 224, 64, 3, 2)])
+@pytest.mark.parametrize("p", [0.0, 0.3])
+def test_first_convolution_and_pooling_in_one_kernel(B, fpo, shape, p):
+    """7x7 / 2 convolution + ReLU + 3x3 / 2 max pooling from the NCHW bf16 input in one kernel: one, two and three position
+    tiles per unit, an odd number of pooled rows, one input channel, the 224 x 224 size; the pooled tensor and the logits
+    against the oracle, and a smaller batch than the handle was built for."""
+    H, W, K, C, batch = shape
+    w = wl.Workload("stem_pool", _stem_net(H, W, K, C), batch, 31, True, wl.uniform_ratios(p), f"uniform {p}")
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, max_batch=batch + 1)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        assert B.fp_query_int(g.h, B.FP_Q_N_LAUNCHES) == 4          # stem + pooling, convolution, two head kernels
+        got = g.forward(w.x)
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        ref_all = fpo.fused_forward(gp, w.x, return_all=True)
+        pooled_ref = ref_all[gp.ops[1]["out"]]
+        info = B.op_infos(g.h)[2]
+        pooled = B.fp_query_array(g.h, B.FP_Q_OP_OUTPUT, 2, np.float32, batch * pooled_ref.shape[1] * info.P * info.Q)
+        assert err(pooled.reshape(pooled_ref.shape).astype(np.float64), pooled_ref) < TOL_BF16
+        assert err(got, fpo.fused_forward(gp, w.x)) < TOL_BF16
+        np.testing.assert_array_equal(g.forward(w.x[:1]), got[:1])
+        out = np.empty((batch, g.n_classes), dtype=np.float32)
+        x_host = torch.from_numpy(w.x).to(torch.bfloat16)            # host buffer in the network's input type
+        B.fp_forward_host(g.h, x_host, batch, out)                   # the input arrives in pieces, one kernel launch per piece
+        np.testing.assert_array_equal(out.astype(np.float64), got)
     finally:
         g.close()
 
