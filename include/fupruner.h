@@ -125,6 +125,21 @@ fp_status fp_fuse(const fp_model_desc* desc, const float* d_weights, size_t n_we
                   const float* d_bn, size_t n_bn, int32_t max_batch, fp_handle* out);
 
 /*
+ * fp_fuse_with_allocator - fp_fuse with the caller's device allocator (Sec. IV-A's problem statement leaves memory
+ * to the host framework): every device buffer of the handle - fused and packed filter banks, activations, scratch,
+ * now and in later fp_prune / fp_soft_prune_finish / fp_query calls - is taken with alloc(bytes, user) and given
+ * back with dealloc(ptr, user), e.g. a framework's caching allocator, so the library itself never calls cudaMalloc.
+ *   alloc     returns a device pointer aligned to 256 bytes, or NULL (reported as FP_ERR_NOMEM); may be called from
+ *             any thread that calls into the library; must stay valid until fp_destroy.
+ *   dealloc   called once for every pointer alloc returned, at the latest in fp_destroy.
+ * alloc == dealloc == NULL is fp_fuse.
+ */
+fp_status fp_fuse_with_allocator(const fp_model_desc* desc, const float* d_weights, size_t n_weights,
+                                 const float* d_bn, size_t n_bn, int32_t max_batch,
+                                 void* (*alloc)(size_t bytes, void* user), void (*dealloc)(void* ptr, void* user),
+                                 void* user, fp_handle* out);
+
+/*
  * fp_prune - filter pruning (Sec. IV-C, Algorithm 1 selection + final extraction).  Scores
  * every convolution's filters on the device on the fused, unpruned fp32 weights (Eq. 6 or
  * the l1 sum), ranks ascending by (score, filter index), masks the lowest q, then removes
@@ -186,7 +201,9 @@ typedef enum {
                                 last input must still be alive), and a layer inside a fused run, whose output
                                 never reaches memory, is refused with FP_ERR_UNSUPPORTED - the run's last
                                 layer can be read */
-    FP_Q_DEVICE_STATUS = 12, /* int32: 0, or FP_ERR_TIMEOUT if a bounded device wait ran out       */
+    FP_Q_DEVICE_STATUS = 12, /* int32: 0, or FP_ERR_TIMEOUT if a bounded device wait ran out since the last query
+                                (the flag is cleared by the query that reports it); synchronises with the device's
+                                earlier work through the copy that reads it                             */
     FP_Q_N_LAUNCHES = 13,    /* int32: kernels one fp_forward launches                             */
     FP_Q_OP_TIMES = 14       /* float[N_OPS]: milliseconds per fused operator of a forward of the last batch size,
                                 measured now as differences of the times of the forward's prefixes (launches 0..i
@@ -272,6 +289,19 @@ fp_status fp_soft_prune_finish(fp_handle h);
 #define FP_STATIC_RANK_MAX_FILTERS 4096
 fp_status fp_rank_filters_static(const float* d_filters, int32_t K, int32_t per_filter, int32_t norm, int32_t q,
                                  int32_t* d_rank, uint8_t* d_mask, void* stream);
+
+/*
+ * fp_debug_expire_wait - diagnostic (no counterpart in the paper): makes one bounded device-side wait run out on
+ * purpose, to show that the kernels' way out works.  Every wait inside the tensor-core kernels (for a bulk copy, for
+ * the tensor cores, for the other warps) has a time limit; when one runs out the CTA raises the handle's status word,
+ * all of its roles leave their loops, tensor memory is released and the kernel returns.  This call launches the first
+ * stride-1 convolution of the graph that runs as a kernel of its own with the first round of its activation copies
+ * left out and a limit of one millisecond, so exactly that happens; nothing faults and nothing hangs.  The
+ * activations of the handle are garbage afterwards (run fp_forward again), and the next
+ * fp_query(FP_Q_DEVICE_STATUS) reports FP_ERR_TIMEOUT, once.  Asynchronous on `stream`.
+ * Errors: FP_ERR_ARG, FP_ERR_UNSUPPORTED (no such convolution in the graph), FP_ERR_CUDA.
+ */
+fp_status fp_debug_expire_wait(fp_handle h, void* stream);
 
 fp_status fp_destroy(fp_handle h);
 

@@ -25,7 +25,8 @@ FP_NORM_L1, FP_NORM_L2 = 0, 1
  FP_Q_OP_TIMES, FP_Q_CONV_BANK_ELEMS) = range(16)
 
 EXPORTS = ["fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_score", "fp_query", "fp_destroy",
-           "fp_last_error", "fp_rank_filters_static", "fp_soft_prune_epoch", "fp_soft_prune_finish"]
+           "fp_last_error", "fp_rank_filters_static", "fp_soft_prune_epoch", "fp_soft_prune_finish",
+           "fp_debug_expire_wait", "fp_fuse_with_allocator"]
 FP_STATIC_RANK_MAX_FILTERS = 4096
 
 
@@ -51,6 +52,36 @@ class fp_op_info(ctypes.Structure):
                 ("bytes_fixed", ctypes.c_double), ("chain", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p)
+DEALLOC_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_void_p)
+
+
+class TorchAllocator:
+    """PyTorch's caching allocator as the library's device allocator (argument marshalling only: the two callbacks hand
+    sizes and pointers through).  Keep the object alive as long as the handle."""
+
+    def __init__(self):
+        import torch
+        self.n_alloc = self.n_free = 0
+        self.live = {}
+
+        def _alloc(nbytes, _user):
+            try:
+                ptr = torch.cuda.caching_allocator_alloc(int(nbytes))
+            except Exception:
+                return None
+            self.n_alloc += 1
+            self.live[ptr] = int(nbytes)
+            return ptr
+
+        def _free(ptr, _user):
+            self.n_free += 1
+            self.live.pop(ptr, None)
+            torch.cuda.caching_allocator_delete(ptr)
+
+        self.alloc, self.dealloc = ALLOC_FN(_alloc), DEALLOC_FN(_free)
+
+
 class FpError(RuntimeError):
     def __init__(self, status, message):
         super().__init__(f"fupruner status {status}: {message}")
@@ -70,6 +101,9 @@ def lib():
         L.fp_last_error.restype = ctypes.c_char_p
         L.fp_fuse.argtypes = [ctypes.POINTER(fp_model_desc), ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
                               ctypes.c_size_t, ctypes.c_int32, ctypes.POINTER(ctypes.c_void_p)]
+        L.fp_fuse_with_allocator.argtypes = [ctypes.POINTER(fp_model_desc), ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
+                                             ctypes.c_size_t, ctypes.c_int32, ALLOC_FN, DEALLOC_FN, ctypes.c_void_p,
+                                             ctypes.POINTER(ctypes.c_void_p)]
         L.fp_prune.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         L.fp_forward.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         L.fp_forward_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
@@ -78,6 +112,7 @@ def lib():
         L.fp_destroy.argtypes = [ctypes.c_void_p]
         L.fp_soft_prune_epoch.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         L.fp_soft_prune_finish.argtypes = [ctypes.c_void_p]
+        L.fp_debug_expire_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         L.fp_rank_filters_static.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
@@ -99,14 +134,19 @@ def make_nodes(node_dicts):
 
 
 def fp_fuse(net, d_weights, d_bn, max_batch, compute=FP_COMPUTE_BF16_TC, in_dtype=FP_DTYPE_F32, use_graph=0,
-            keep_outputs=0, scatter=0):
-    """net: workloads.Net; d_weights/d_bn: CUDA float32 torch tensors.  Returns an opaque handle."""
+            keep_outputs=0, scatter=0, allocator=None):
+    """net: workloads.Net; d_weights/d_bn: CUDA float32 torch tensors; allocator: None (the library uses cudaMalloc) or an
+    object with ctypes callbacks `alloc` / `dealloc` (TorchAllocator).  Returns an opaque handle."""
     nodes = make_nodes(net.nodes)
     desc = fp_model_desc(len(net.nodes), nodes, net.in_C, net.in_H, net.in_W, in_dtype, compute,
                          float(net.bn_eps), use_graph, keep_outputs, scatter)
     h = ctypes.c_void_p()
-    _check(lib().fp_fuse(ctypes.byref(desc), d_weights.data_ptr(), d_weights.numel(), d_bn.data_ptr(),
-                         d_bn.numel(), max_batch, ctypes.byref(h)))
+    if allocator is None:
+        _check(lib().fp_fuse(ctypes.byref(desc), d_weights.data_ptr(), d_weights.numel(), d_bn.data_ptr(),
+                             d_bn.numel(), max_batch, ctypes.byref(h)))
+    else:
+        _check(lib().fp_fuse_with_allocator(ctypes.byref(desc), d_weights.data_ptr(), d_weights.numel(), d_bn.data_ptr(),
+                                            d_bn.numel(), max_batch, allocator.alloc, allocator.dealloc, None, ctypes.byref(h)))
     return h
 
 
@@ -186,6 +226,11 @@ def fp_soft_prune_epoch(h, ratios=None, d_updates=None, norm=FP_NORM_L2):
 
 def fp_soft_prune_finish(h):
     _check(lib().fp_soft_prune_finish(h))
+
+
+def fp_debug_expire_wait(h, stream=None):
+    """Diagnostic: lets one bounded device-side wait run out (see the header); the next FP_Q_DEVICE_STATUS reports it."""
+    _check(lib().fp_debug_expire_wait(h, stream.cuda_stream if stream is not None else None))
 
 
 def conv_bank_elems(h):

@@ -62,6 +62,8 @@ struct TcParams {
     long long bank_tile_bytes;          // streamed filters: bytes of one filter tile's part of the bank (all taps, all chunks)
     int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
     int scatter_bytes;                  // scattered output: channel -> accumulator column map and the tiles' chunk ranges
+    long long wait_cycles;              // limit of every barrier wait in SM clock cycles (0: about a second)
+    int skip_round;                     // diagnostic: the activation producer leaves out this round's copies (-1: none)
     int* status;
 };
 
@@ -170,6 +172,7 @@ conv_tc_kernel(const TcParams p) {
                               : MODE == MODE_FLAT_STREAM ? (uint32_t)(p.b_stages * p.b_stage_bytes) : 0u;
     const uint32_t a_base = b_base + ((b_region + 127u) & ~127u);
     volatile int* abort_flag = &ctrl->abort_flag;
+    const long long wait_limit = p.wait_cycles > 0 ? p.wait_cycles : kWaitCycles;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t a_full0 = ctrl_addr + (uint32_t)offsetof(Ctrl, a_full);
@@ -263,7 +266,7 @@ conv_tc_kernel(const TcParams p) {
             for (int g = 0; g < p.groups; ++g) {
                 if (turn == prod) {
                     bool w = true;
-                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit);
                     w = __shfl_sync(0xffffffffu, w, 0);
                     if (!w) { ok = false; break; }
                     int cgg = p.cchunks - g * p.cg;
@@ -298,22 +301,25 @@ conv_tc_kernel(const TcParams p) {
             // side by side instead of one after the other.
             bool ok = true;
             uint32_t stage = 0, phase = 0;
+            int round = 0;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
                 const long long f0 = (long long)fdiv((uint32_t)tile, p.div_ntiles) * p.tps * 128;
                 for (int g = 0; g < p.groups; ++g) {
                     bool w = true;
-                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit);
                     w = __shfl_sync(0xffffffffu, w, 0);
                     if (!w) { ok = false; break; }
                     int cgg = p.cchunks - g * p.cg;
                     if (cgg > p.cg) cgg = p.cg;
                     const uint32_t fb = a_full0 + 8 * stage;
                     const uint32_t dst = a_base + stage * p.a_stage_bytes;
-                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
-                    __syncwarp();
-                    if (lane < cgg)
-                        bulk_copy(dst + lane * p.rows_a * 16, xv + (long long)(g * p.cg + lane) * p.plane_in + f0 - p.halo,
-                                  (uint32_t)(p.rows_a * 16), fb);
+                    if (round++ != p.skip_round) {       // (a diagnostic launch leaves one round out: its stage never fills)
+                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
+                        __syncwarp();
+                        if (lane < cgg)
+                            bulk_copy(dst + lane * p.rows_a * 16, xv + (long long)(g * p.cg + lane) * p.plane_in + f0 - p.halo,
+                                      (uint32_t)(p.rows_a * 16), fb);
+                    }
                     if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -332,7 +338,7 @@ conv_tc_kernel(const TcParams p) {
                     if (p.groups > 1) { tap0 = kb / p.groups; g = kb - tap0 * p.groups; ntap = 1; cgg = p.cchunks - g * p.cg; if (cgg > p.cg) cgg = p.cg; }
                     else { tap0 = kb * p.tpk; g = 0; ntap = p.taps - tap0 < p.tpk ? p.taps - tap0 : p.tpk; cgg = p.cchunks; }
                     bool w = true;
-                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                    if (lane == 0) w = mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit);
                     w = __shfl_sync(0xffffffffu, w, 0);
                     if (!w) { ok = false; break; }
                     const uint32_t fb = a_full0 + 8 * stage;
@@ -359,11 +365,11 @@ conv_tc_kernel(const TcParams p) {
             uint32_t acc_phase0 = 0, acc_phase1 = 0;
             int local = 0;
             bool ok = true;
-            if (MODE == MODE_FLAT_RESIDENT) ok = mbar_wait(b_full0, 0, abort_flag);
+            if (MODE == MODE_FLAT_RESIDENT) ok = mbar_wait(b_full0, 0, abort_flag, wait_limit);
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++local) {
                 const int acc = local & 1;
                 const uint32_t ph = acc ? acc_phase1 : acc_phase0;
-                if (!mbar_wait(tempty0 + 8 * acc, ph ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tempty0 + 8 * acc, ph ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                 if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
                 tc_fence_after();
                 const int nt = tile - (int)fdiv((uint32_t)tile, p.div_ntiles) * p.n_tiles;
@@ -375,7 +381,7 @@ conv_tc_kernel(const TcParams p) {
                     const uint32_t a_ks = 2u * (uint32_t)p.rows_a, b_ks = 2u * (uint32_t)p.n_tile;
                     const uint32_t d_acc = d_tmem + (uint32_t)(issuer * p.n_tile);
                     for (int g = 0; g < p.groups && ok; ++g) {
-                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag, wait_limit)) { ok = false; break; }
                         tc_fence_after();
                         int cgg = p.cchunks - g * p.cg;
                         if (cgg > p.cg) cgg = p.cg;
@@ -399,7 +405,7 @@ conv_tc_kernel(const TcParams p) {
                     // Descriptors differ only in their 16-byte start-address field, so the inner loops
                     // just add row counts to the low word (rows are 16 bytes: one row = one address unit).
                     for (int g = 0; g < p.groups && ok; ++g) {
-                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag, wait_limit)) { ok = false; break; }
                         tc_fence_after();
                         int cgg = p.cchunks - g * p.cg;
                         if (cgg > p.cg) cgg = p.cg;
@@ -424,7 +430,7 @@ conv_tc_kernel(const TcParams p) {
                             for (int sx = 0; sx < p.a.S; ++sx) {
                                 // streamed filters: one block per (K group, tap).  Every 128-position tile of the step
                                 // uses it: its own accumulator and issuing warp, its activation rows 128 further on
-                                if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag)) { ok = false; break; }
+                                if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag, wait_limit)) { ok = false; break; }
                                 tc_fence_after();
                                 const uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
                                 issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_row + (uint32_t)sx + (uint32_t)(issuer * 128), b_lo,
@@ -442,7 +448,7 @@ conv_tc_kernel(const TcParams p) {
                 } else {
                     const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
                     for (int kb = 0; kb < p.kblocks; ++kb) {
-                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag, wait_limit)) { ok = false; break; }
                         tc_fence_after();
                         int planes;
                         if (p.groups > 1) { const int g = kb % p.groups; planes = p.cchunks - g * p.cg; if (planes > p.cg) planes = p.cg; }
@@ -509,7 +515,7 @@ conv_tc_kernel(const TcParams p) {
                     if (c_begin + i * 8 < c_end) rq[i] = __ldg(res + vec0 + (long long)((c_begin >> 3) + i) * p.plane_out);
             }
             if (t == 0) {
-                ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag);
+                ok = mbar_wait(tfull0 + 8 * acc, ph, abort_flag, wait_limit);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (acc) acc_phase1 ^= 1; else acc_phase0 ^= 1;
@@ -702,7 +708,7 @@ conv_tc_kernel(const TcParams p) {
                     if (cgg > p.cg) cgg = p.cg;
                     for (int tap = 0; tap < p.taps; ++tap) {
                         bool w = true;
-                        if (lane == 0) w = mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag);
+                        if (lane == 0) w = mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit);
                         w = __shfl_sync(0xffffffffu, w, 0);
                         if (!w) { ok = false; break; }
                         const uint32_t fb = b_full0 + 8 * stage;
@@ -752,7 +758,7 @@ conv_tc_kernel(const TcParams p) {
                     v[i] = make_uint4(0, 0, 0, 0);
                     if (valid) v[i] = __ldg(xv + base + e.x);
                 }
-                if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit)) { ok = false; break; }
                 uint8_t* dst = smem_raw + (a_base - ctrl_addr) + stage * stage_bytes + m * 16;
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
@@ -1013,7 +1019,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     return 0;
 }
 
-void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st) {
+void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st, int skip_round, long long wait_cycles) {
     TcParams p;
     memset(&p, 0, sizeof(p));
     p.a = a;
@@ -1039,6 +1045,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.lut_bytes = plan.flat ? 0 : p.kblocks * 64;
     p.scatter_bytes = a.scatter ? round_up_i((a.out_C_pad + plan.n_tiles + 1) * 4, 16) + 8 * 32 * 33 * 4 : 0;
     p.status = d_status;
+    p.skip_round = skip_round; p.wait_cycles = wait_cycles;
     p.div_ntiles = make_fastdiv((uint32_t)plan.n_tiles);
     p.div_p2out = make_fastdiv((uint32_t)p.P2_out);
     p.div_qp = make_fastdiv((uint32_t)p.Qp);

@@ -152,14 +152,17 @@ struct ConvPlanTC {
 void conv_tc_filter_tile(const ConvArgs& a, int K_pad, int* n_tile, int* n_tiles);
 // Returns 0 on success, otherwise writes a message.
 int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len);
-void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st);
+// skip_round / wait_cycles: diagnostic launch (see fp_debug_expire_wait): the activation producer of a stride-1 layer leaves
+// out one round of copies and every wait gives up after wait_cycles SM clock cycles; -1 / 0 for a normal launch
+void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cudaStream_t st, int skip_round = -1,
+                    long long wait_cycles = 0);
 
 // First convolution (7x7 / stride 2 / pad 3, at most 3 input channels, ReLU) and the 3x3 / stride 2 / pad 1 max pooling
 // behind it as one kernel that reads the NCHW bf16 network input and writes the pooled tensor.
 struct StemPoolArgs {
     const void* x;        // network input, N x C x H x W, NCHW, bf16
     void* y;              // pooled tensor, planar-8 with border, (H/4) x (W/4) pixels, K_pad channels, N images
-    const void* w;        // filters [20 chunks of 8 k][K_pad rows][8] bf16, k = (r * 7 + s) * C + c, zero for k >= 49 C
+    const void* w;        // filters [20 chunks of 8 k][K_pad rows][8] bf16, k = (r * C + c) * 7 + s, zero for k >= 49 C
     const float* bias;    // [K_pad]
     int N, C, H, W, K_pad;
     int n0, n_count;      // the images this launch handles (the tensor's plane pitch is that of all N)
@@ -168,7 +171,7 @@ struct StemPoolPlan { int valid, tiles, tmem_cols; unsigned smem_bytes; };
 bool stem_pool_supported(int C, int H, int W, int K_pad);
 int plan_stem_pool(const StemPoolArgs& a, StemPoolPlan* plan, char* err, size_t err_len);
 void launch_stem_pool(const StemPoolPlan& plan, const StemPoolArgs& a, int* d_status, cudaStream_t st);
-// its filters: out[k / 8][kr][k % 8] = w[row_src[kr]][c][r][s] with k = (r * 7 + s) * C + c (zero rows / zero k padding)
+// its filters: out[k / 8][kr][k % 8] = w[row_src[kr]][c][r][s] with k = (r * C + c) * 7 + s (zero rows / zero k padding)
 void launch_repack_stem_direct(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st);
 
 // A run of stride-1 3x3 convolutions executed by one kernel with the activations in shared memory.

@@ -226,7 +226,7 @@ __global__ void repack_stem_direct_kernel(const float* __restrict__ w, int C, co
         float v = 0.0f;
         const int ks = row_src[kr];
         if (ks >= 0 && k < 49 * C) {
-            const int r = k / (7 * C), rem = k - r * 7 * C, s = rem / C, c = rem - s * C;
+            const int rc = k / 7, s = k - rc * 7, r = rc / C, c = rc - r * C;
             v = w[(((size_t)ks * C + c) * 7 + r) * 7 + s];
         }
         out[i] = __float2bfloat16_rn(v);

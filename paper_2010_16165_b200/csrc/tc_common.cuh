@@ -55,15 +55,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uin
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the time limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  Returns false when the time limit (SM clock cycles) ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit_cycles = kWaitCycles) {
     if (mbar_test_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait(bar, parity, 2000u)) return true;
         if ((i & 15) == 15) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) return false;
+            if (clock64() - t0 > limit_cycles) return false;
         }
     }
     return false;

@@ -359,6 +359,61 @@ def test_batch_edges_and_graph_and_host(B, fpo):
         g.close()
 
 
+def test_a_device_wait_that_runs_out_is_reported_and_survived(B, fpo):
+    """Every wait inside the tensor-core kernels is bounded.  A diagnostic launch leaves out one round of a convolution's
+    activation copies with a limit of a millisecond: the waiting thread gives up, the status word is raised, all roles of the
+    CTA leave, tensor memory is released, the kernel returns.  The status is reported once, and the same handle then runs a
+    forward with the bits it produced before."""
+    w = wl.tiny_cifar(widths=(16, 32, 64), in_hw=16, batch=4, p=0.3)
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, keep_outputs=1)            # every layer is a kernel of its own
+    try:
+        B.fp_prune(g.h, w.ratios)
+        before = g.forward(w.x)
+        B.fp_debug_expire_wait(g.h)
+        torch.cuda.synchronize()                                   # returns: nothing hangs, nothing faults
+        assert B.fp_query_int(g.h, B.FP_Q_DEVICE_STATUS) == B.FP_ERR_TIMEOUT
+        assert B.fp_query_int(g.h, B.FP_Q_DEVICE_STATUS) == 0      # reported once
+        after = g.forward(w.x)                                     # forward() checks the status too
+        np.testing.assert_array_equal(before, after)
+        gp, _, _, _ = oracle_pruned(fpo, w)
+        assert err(after, fpo.fused_forward(gp, w.x)) < TOL_BF16
+    finally:
+        g.close()
+
+
+def test_callers_allocator_serves_every_buffer(B, fpo):
+    """fp_fuse_with_allocator: the library takes all of its device memory from the caller's allocator (here PyTorch's
+    caching allocator through two callbacks) - at fuse time, when fp_prune rebuilds the graph and for debug dumps - and
+    gives all of it back by fp_destroy; results are the same bits as with its own cudaMalloc."""
+    w = wl.tiny_cifar(widths=(16, 32, 64), in_hw=16, batch=3, n_per_stage=2, p=0.3)
+    ref_g = Gpu(B, w, B.FP_COMPUTE_BF16_TC)
+    try:
+        B.fp_prune(ref_g.h, w.ratios)
+        want = ref_g.forward(w.x)
+    finally:
+        ref_g.close()
+    alloc = B.TorchAllocator()
+    dw, dbn = to_dev(w.weights), to_dev(w.bn)
+    h = B.fp_fuse(w.net, dw, dbn, w.batch, B.FP_COMPUTE_BF16_TC, B.FP_DTYPE_F32, 0, 0, 0, alloc)
+    try:
+        n_fuse = alloc.n_alloc
+        assert n_fuse > 10
+        B.fp_prune(h, w.ratios)
+        assert alloc.n_alloc > n_fuse and alloc.n_free > 0          # the graph was rebuilt out of the same allocator
+        out = torch.empty(w.batch, 5, device="cuda")
+        dx = to_dev(w.x)
+        B.fp_forward(h, dx, w.batch, out)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(out.cpu().numpy().astype(np.float64), want)
+        info = [o for o in B.op_infos(h)]
+        last_conv = max(i for i, o in enumerate(info) if o.kind == 0)
+        o = info[last_conv]
+        B.fp_query_array(h, B.FP_Q_OP_OUTPUT, last_conv, np.float32, w.batch * 64 * o.P * o.Q)    # the dump's scratch too
+    finally:
+        B.fp_destroy(h)
+    assert alloc.n_alloc == alloc.n_free and not alloc.live
+
+
 def test_error_codes(B):
     w = wl.tiny_cifar()
     dw, dbn = to_dev(w.weights), to_dev(w.bn)
