@@ -460,7 +460,13 @@ void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, con
     if (is_bf16) pool_sum_kernel<true><<<blocks, 256, 0, st>>>(x, N, H, W, C_pad / 8, pool_scratch);
     else pool_sum_kernel<false><<<blocks, 256, 0, st>>>(x, N, H, W, C_pad / 8, pool_scratch);
     const int classes = (n_classes + kFcClasses - 1) / kFcClasses;
-    fc_kernel<4><<<dim3((N + 3) / 4, classes), 256, 4 * kFcSlab * sizeof(float), st>>>(pool_scratch, N, C_pad, fcw, fcb, n_classes, logits);
+    // Every block re-reads the FC rows of its classes: with many channels and images that traffic (through L2) is what
+    // bounds the kernel, so wide heads take 16 images per block (ResNet-50 at batch 128: 2048 channels, 8 MB of FC
+    // weights read 8 times instead of 32); narrow ones keep 4, where more blocks matter more.
+    if (C_pad >= 1024 && N >= 64)
+        fc_kernel<16><<<dim3((N + 15) / 16, classes), 256, 16 * kFcSlab * sizeof(float), st>>>(pool_scratch, N, C_pad, fcw, fcb, n_classes, logits);
+    else
+        fc_kernel<4><<<dim3((N + 3) / 4, classes), 256, 4 * kFcSlab * sizeof(float), st>>>(pool_scratch, N, C_pad, fcw, fcb, n_classes, logits);
 }
 
 void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
