@@ -926,8 +926,12 @@ fp_status replan(fp_handle h) {
                 const int taps = packed_stem ? 3 : f.R * f.S, cchunks = (packed_stem ? 80 : f.C_pad) / 8;
                 void* blocked;
                 TRY(dev_alloc(h, h->pack_buffers, &blocked, (size_t)f.tc.n_tiles * taps * cchunks * f.tc.n_tile * 16));
-                fp::launch_reblock_bank((const __nv_bfloat16*)f.d_wp, taps, cchunks, f.K_pad, f.tc.n_tile, f.tc.n_tiles, f.tc.cg,
-                                        (__nv_bfloat16*)blocked, st);
+                if (f.tc.blocked_bank == 1)          // 1x1 layer, unified stages: [tile][K group][tap][chunk][row]
+                    fp::launch_reblock_bank((const __nv_bfloat16*)f.d_wp, taps, cchunks, f.K_pad, f.tc.n_tile, f.tc.n_tiles, f.tc.cg,
+                                            (__nv_bfloat16*)blocked, st);
+                else                                 // gathered layer with several filter tiles: [tile][(tap, chunk) plane][row]
+                    fp::launch_reblock_bank((const __nv_bfloat16*)f.d_wp, 1, taps * cchunks, f.K_pad, f.tc.n_tile, f.tc.n_tiles,
+                                            taps * cchunks, (__nv_bfloat16*)blocked, st);
                 f.d_wp = blocked;
             }
         } else if (op.kind == 1) {

@@ -343,13 +343,13 @@ conv_tc_kernel(const TcParams p) {
                     if (!w) { ok = false; break; }
                     const uint32_t fb = a_full0 + 8 * stage;
                     const uint32_t dst = a_base + stage * (p.a_stage_bytes + p.b_stage_bytes) + p.a_stage_bytes;
-                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(ntap * cgg * nrows * 16));
-                    __syncwarp();
-                    if (lane < ntap * cgg) {
-                        const int tt = lane / cgg, c = lane - tt * cgg;
-                        bulk_copy(dst + lane * p.n_tile * 16,
-                                  wv + ((long long)(tap0 + tt) * p.cchunks + g * p.cg + c) * p.a.K_pad + nt * p.n_tile,
-                                  (uint32_t)(nrows * 16), fb);
+                    // the K block's planes are consecutive (tap, chunk) planes of the bank, which is stored filter tile by
+                    // filter tile ([tile][plane][row]; with one tile that is the packed layout itself): one copy
+                    if (lane == 0) {
+                        const uint32_t bytes = (uint32_t)(ntap * cgg * p.n_tile * 16);
+                        mbar_expect_tx(fb, bytes);
+                        bulk_copy(dst, reinterpret_cast<const uint8_t*>(p.a.w) + (long long)nt * p.bank_tile_bytes +
+                                           (long long)(tap0 * p.cchunks + g * p.cg) * p.n_tile * 16, bytes, fb);
                     }
                     if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
                 }
@@ -1032,6 +1032,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             while (plan->a_stages > 2 && smem + plan->a_stages * stage > kSmemPerSm / 2 - 1024u) --plan->a_stages;   // two CTAs must fit
         }
         plan->b_stages = plan->a_stages;
+        if (n_tiles > 1) plan->blocked_bank = 2;        // [filter tile][plane][row]: a K block's filters are one run
         smem += plan->a_stages * stage;
     }
     if (plan->tps < 1) plan->tps = 1;
@@ -1051,7 +1052,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     // loaders' latency there (measured on ResNet-50, batch 128: every strided layer about 30 % faster with four).
     const int epi = (n_tile >= 64 && (plan->flat || m_tiles * n_tiles <= sms)) ? 8 : 4;
     plan->epi_warps = epi;
-    const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : plan->blocked_bank ? MODE_FLAT_UNIFIED : MODE_FLAT_STREAM;
+    const int mode = !plan->flat ? MODE_GATHER : bank_fits ? MODE_FLAT_RESIDENT : plan->blocked_bank == 1 ? MODE_FLAT_UNIFIED : MODE_FLAT_STREAM;
     const void* fn = kernel_for(mode, epi);
     // a per-device attribute: set it for the device this plan is made on (cheap, so not cached)
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
@@ -1091,7 +1092,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.total_tiles = (int)(((m_tiles + p.tps - 1) / p.tps) * plan.n_tiles);
     const int gplanes = plan.groups > 1 ? plan.cg : plan.tpk * p.cchunks;      // gather: planes per stage
     p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : gplanes * 128 * 16;
-    p.b_stage_bytes = plan.blocked_bank ? p.taps * plan.cg * plan.n_tile * 16 : plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
+    p.b_stage_bytes = plan.blocked_bank == 1 ? p.taps * plan.cg * plan.n_tile * 16 : plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
     p.bank_tile_bytes = (long long)p.taps * p.cchunks * plan.n_tile * 16;
     p.tpk = plan.tpk > 0 ? plan.tpk : 1;
     p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
@@ -1109,7 +1110,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid);
-    const int mode = !plan.flat ? MODE_GATHER : plan.b_resident ? MODE_FLAT_RESIDENT : plan.blocked_bank ? MODE_FLAT_UNIFIED : MODE_FLAT_STREAM;
+    const int mode = !plan.flat ? MODE_GATHER : plan.b_resident ? MODE_FLAT_RESIDENT : plan.blocked_bank == 1 ? MODE_FLAT_UNIFIED : MODE_FLAT_STREAM;
     cfg.blockDim = dim3((unsigned)(64 + 32 * plan.epi_warps + extra_threads(mode)));
     cfg.dynamicSmemBytes = plan.smem_bytes;
     cfg.stream = st;

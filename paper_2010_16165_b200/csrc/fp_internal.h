@@ -134,7 +134,8 @@ struct ConvPlanTC {
     int flat;             // 1: stride-1 "same" convolution, activation tiles fetched as contiguous runs
                           //    of flat positions (bulk copies); 0: gathered by loader threads
     int b_resident;       // flat only: the whole filter bank stays in shared memory
-    int blocked_bank;     // streamed filters: the bank must be stored block by block (launch_reblock_bank)
+    int blocked_bank;     // 1: 1x1 layer with unified stages, bank stored block by block; 2: gathered layer with several
+                          // filter tiles, bank stored tile by tile (launch_reblock_bank either way)
     int cg;               // channel chunks (of 8) per K block
     int groups;           // K blocks per filter tap = ceil((C_pad/8) / cg)
     int halo;             // flat: vectors fetched before and after the 128 positions of a tile
