@@ -59,6 +59,7 @@ struct Tensor {
     void* d = nullptr;
     size_t bytes = 0;
     int producer = -1;         // index into ops, -1 = network input
+    int split = 0;             // stored parity-split (fp::ConvArgs): only stride-2 convolutions read it
 };
 
 struct FConv {
@@ -79,6 +80,7 @@ struct FConv {
     int n_tile_forced = 0;     // scatter: filters per CTA tile the packed bank was laid out for
     int32_t* d_out_map = nullptr;   // scatter: output channel -> packed filter row (-1 = no filter kept)
     int32_t* d_chunk0 = nullptr;    // scatter: first output chunk of every filter tile, and the end
+    int n_mult = 1;            // 4: a 1x1 layer over a parity-split tensor runs on its 4 N half-size images
     int K_kept = 0, K_rows = 0, K_pad = 0, C_kept = 0, C_pad = 0;
     void* d_wp = nullptr;      // packed filters in the compute type, K_pad x R x S x C_pad
     float* d_bp = nullptr;
@@ -647,6 +649,7 @@ bool chain_candidate(fp_handle h, const FConv& f) {
     if (h->compute != FP_COMPUTE_BF16_TC || h->keep_outputs || f.scatter) return false;
     if (f.R != 3 || f.S != 3 || f.stride != 1 || f.pad != 1) return false;
     if ((h->stem_packed || h->stem_fused) && f.src == 0) return false;
+    if (h->tensors[f.src].split || h->tensors[f.out].split) return false;
     const Tensor& s = h->tensors[f.src];
     return fp::chain_layer_supported(s.H, s.W, f.K_pad, f.C_pad);
 }
@@ -738,14 +741,68 @@ fp_status find_chains(fp_handle h, const std::vector<std::vector<Use>>& uses) {
     return FP_OK;
 }
 
+// How a convolution reads a parity-split input tensor: 0 it cannot, 'A' 3x3 / stride 2 / pad 1 (nine taps over the four
+// parity images), 'B' 1x1 / stride 2 (the parity-00 image), 'C' 1x1 / stride 1 without shortcut (position by position:
+// its output is then split the same way).
+char split_reader(const FConv& f) {
+    if (f.R == 3 && f.S == 3 && f.stride == 2 && f.pad == 1) return 'A';
+    if (f.R == 1 && f.S == 1 && f.stride == 2 && f.pad == 0) return 'B';
+    if (f.R == 1 && f.S == 1 && f.stride == 1 && f.pad == 0 && f.res_mode == 0) return 'C';
+    return 0;
+}
+
+// Which tensors are stored parity-split (tensor-core path): tensors written by a convolution of their own kernel, with
+// even height and width, that only stride-2 convolutions read - directly, or through 1x1 layers whose output is split
+// in turn (the first 1x1 of a strided bottleneck block).  A stride-2 convolution over such a tensor is a stride-1
+// convolution over contiguous runs (bulk copies) instead of a gather.
+void decide_splits(fp_handle h, const std::vector<std::vector<Use>>& uses) {
+    const int nt = (int)h->tensors.size();
+    for (Tensor& t : h->tensors) t.split = 0;
+    if (h->compute != FP_COMPUTE_BF16_TC) return;
+    std::vector<int> cand(nt, 0);
+    for (int t = 1; t < nt; ++t) {
+        const Tensor& T = h->tensors[t];
+        if (T.producer < 0 || h->ops[T.producer].kind != 0 || T.H % 2 || T.W % 2 || T.H < 2 || T.W < 2 || uses[t].empty()) continue;
+        const FConv& pf = h->convs[h->ops[T.producer].idx];
+        if (pf.src == 0 && (pf.R == 7 || h->stem_packed)) continue;                    // the first convolution has forms of its own
+        cand[t] = 1;
+    }
+    for (bool changed = true; changed;) {
+        changed = false;
+        for (int t = 1; t < nt; ++t) {
+            if (!cand[t]) continue;
+            bool ok = true;
+            for (const Use& u : uses[t]) {
+                if (u.how != 0 || h->ops[u.op].kind != 0) { ok = false; break; }
+                const FConv& f = h->convs[h->ops[u.op].idx];
+                const char kind = split_reader(f);
+                if (!kind || (kind == 'C' && !cand[f.out])) { ok = false; break; }
+            }
+            if (!ok) { cand[t] = 0; changed = true; }
+        }
+    }
+    for (int t = 1; t < nt; ++t) h->tensors[t].split = cand[t];
+}
+
 // Geometry of the launch of fused convolution f (no pointers, no channel counts of the output).
 void conv_geometry(fp_handle h, const FConv& f, fp::ConvArgs* a) {
     const Tensor& src = h->tensors[f.src];
     const Tensor& out = h->tensors[f.out];
     a->N = h->max_batch; a->H = src.H; a->W = src.W; a->C_pad = src.C_pad; a->P = out.H; a->Q = out.W;
     a->R = f.R; a->S = f.S; a->stride = f.stride; a->pad = f.pad; a->relu = f.relu;
+    a->y_split = 0; a->x_plane_mult = 0; a->x_s2d = 0;
     if (h->stem_packed && f.src == 0) {      // 3x1 stride-1 convolution over the packed input, at the output resolution
         a->H = out.H; a->W = out.W; a->C_pad = 80; a->R = 3; a->S = 1; a->stride = 1; a->pad = 1;
+    }
+    if (src.split) {
+        const char kind = split_reader(f);
+        a->H = src.H / 2; a->W = src.W / 2; a->stride = 1;
+        if (kind == 'A') { a->x_s2d = 1; }
+        else if (kind == 'B') { a->x_plane_mult = 4; }
+        else { a->N = 4 * h->max_batch; a->P = out.H / 2; a->Q = out.W / 2; }        // 'C': 4 N half-size images in, the same out
+        if (kind != 'C' && out.split) a->y_split = 1;
+    } else if (out.split) {
+        a->y_split = 1;
     }
 }
 
@@ -776,6 +833,8 @@ fp_status replan(fp_handle h) {
         if (f.src == 0 && h->compute == FP_COMPUTE_BF16_TC && uses[0].size() == 1 && f.R == 7 && f.S == 7 &&
             f.stride == 2 && f.pad == 3 && f.C <= 3 && h->in_H % 2 == 0 && h->in_W % 2 == 0)
             h->stem_packed = 1;
+    decide_splits(h, uses);
+    for (FConv& f : h->convs) f.n_mult = (h->tensors[f.src].split && split_reader(f) == 'C') ? 4 : 1;
     // ... and, where a 3x3 / stride-2 max pooling is the only reader of that convolution and the input is bf16, input
     // conversion, convolution and pooling run as one kernel (decided below, once the filter count is known).
     h->stem_fused = 0;
@@ -986,6 +1045,8 @@ fp_status replan(fp_handle h) {
             // planar-8 with border, plus guard vectors before and after (halo reads of the first/last tiles)
             const size_t vec_bytes = 8 * h->act_elem();
             t.bytes = ((size_t)(t.C_pad / 8) * h->max_batch * (t.H + 2) * (t.W + 2) + 2 * (size_t)fp::kGuardVectors) * vec_bytes;
+            if (t.split)
+                t.bytes = ((size_t)(t.C_pad / 8) * 4 * h->max_batch * (t.H / 2 + 2) * (t.W / 2 + 2) + 2 * (size_t)fp::kGuardVectors) * vec_bytes;
             if (tid == 0 && h->stem_packed)
                 t.bytes = ((size_t)10 * h->max_batch * (t.H / 2 + 2) * (t.W / 2 + 2) + 2 * (size_t)fp::kGuardVectors) * vec_bytes;
             int best = -1;
@@ -1082,7 +1143,7 @@ void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float*
     } else if (op.kind == 0) {
         FConv& f = h->convs[op.idx];
         fp::ConvArgs a = f.args;
-        a.N = batch;
+        a.N = batch * f.n_mult;
         if (h->compute == FP_COMPUTE_BF16_TC) fp::launch_conv_tc(f.tc, a, h->d_status, st);
         else fp::launch_conv_simt(a, bf16, st);
     } else if (op.kind == 1) {
@@ -1386,7 +1447,7 @@ extern "C" fp_status fp_debug_expire_wait(fp_handle h, void* stream) {
         const Op& op = h->ops[i];
         if (op.kind != 0 || h->op_chain[i] >= 0 || (h->stem_fused && i == 1)) continue;
         const FConv& f = h->convs[op.idx];
-        if (!f.tc.valid || !f.tc.flat || f.tc.blocked_bank) continue;
+        if (!f.tc.valid || !f.tc.flat || f.tc.blocked_bank || h->tensors[f.src].split || h->tensors[f.out].split) continue;
         // the first round of the activation producer is left out, so the MMA-issuing thread's wait for that stage runs
         // out after a millisecond (two million cycles), raises the status word and takes every role of the CTA with it
         fp::launch_conv_tc(f.tc, f.args, h->d_status, (cudaStream_t)stream, 0, 2000000LL);
@@ -1560,7 +1621,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
                 CK(cudaDeviceSynchronize());
             }
             TRY(dev_alloc_raw(h, (void**)&d_tmp, cnt * sizeof(float)));
-            fp::launch_planar_to_nchw_f32(t.d, h->act_is_bf16(), d_tmp, h->last_batch, t.H, t.W, t.C_pad, t.C, 0);
+            fp::launch_planar_to_nchw_f32(t.d, h->act_is_bf16(), d_tmp, h->last_batch, t.H, t.W, t.C_pad, t.C, t.split, 0);
             cudaError_t e = cudaMemcpy(h_out, d_tmp, cnt * sizeof(float), cudaMemcpyDeviceToHost);
             dev_free(h, d_tmp);
             if (e != cudaSuccess) return fail(FP_ERR_CUDA, "fp_query: copy failed: %s", cudaGetErrorString(e));

@@ -62,6 +62,11 @@ struct TcParams {
     long long bank_tile_bytes;          // streamed filters: bytes of one filter tile's part of the bank (all taps, all chunks)
     int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
     int scatter_bytes;                  // scattered output: channel -> accumulator column map and the tiles' chunk ranges
+    int a_par;                          // activation runs per channel chunk in a stage: 1, or 4 parity images (x_s2d)
+    long long par_stride;               // x_s2d: vectors between the parity images of one chunk (N * P2)
+    int tap_off[9];                     // x_s2d: start row of each tap's operand within a chunk's part of the stage
+    int y_split, y_P2h, y_Wh2;          // split output: half-resolution grid
+    long long plane_y;                  // vectors per chunk plane of the output tensor
     long long wait_cycles;              // limit of every barrier wait in SM clock cycles (0: about a second)
     int skip_round;                     // diagnostic: the activation producer leaves out this round's copies (-1: none)
     int* status;
@@ -314,11 +319,15 @@ conv_tc_kernel(const TcParams p) {
                     const uint32_t fb = a_full0 + 8 * stage;
                     const uint32_t dst = a_base + stage * p.a_stage_bytes;
                     if (round++ != p.skip_round) {       // (a diagnostic launch leaves one round out: its stage never fills)
-                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
+                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(p.a_par * cgg * p.rows_a * 16));
                         __syncwarp();
-                        if (lane < cgg)
-                            bulk_copy(dst + lane * p.rows_a * 16, xv + (long long)(g * p.cg + lane) * p.plane_in + f0 - p.halo,
+                        // one run per channel chunk - or, over a parity-split tensor, one per chunk and parity image
+                        for (int i = lane; i < p.a_par * cgg; i += 32) {
+                            const int c = p.a_par == 1 ? i : i >> 2, pp = p.a_par == 1 ? 0 : i & 3;
+                            bulk_copy(dst + i * p.rows_a * 16,
+                                      xv + (long long)(g * p.cg + c) * p.plane_in + (long long)pp * p.par_stride + f0 - p.halo,
                                       (uint32_t)(p.rows_a * 16), fb);
+                        }
                     }
                     if (++stage == (uint32_t)p.a_stages) { stage = 0; phase ^= 1; }
                 }
@@ -410,14 +419,20 @@ conv_tc_kernel(const TcParams p) {
                         int cgg = p.cchunks - g * p.cg;
                         if (cgg > p.cg) cgg = p.cg;
                         const int ksteps = cgg >> 1;
-                        uint32_t a_row = ((a_base + a_stage * p.a_stage_bytes) >> 4) | ((uint32_t)p.rows_a << 16);
+                        uint32_t a_row = ((a_base + a_stage * p.a_stage_bytes) >> 4) | ((uint32_t)(p.a_par * p.rows_a) << 16);
                         uint32_t b_tap = 0;
                         if (MODE == MODE_FLAT_RESIDENT)
                             b_tap = ((b_base >> 4) + (uint32_t)(g * p.cg * p.a.K_pad + nt * p.n_tile)) | ((uint32_t)p.a.K_pad << 16);
-                        const uint32_t a_ks = 2u * (uint32_t)p.rows_a;
+                        const uint32_t a_ks = 2u * (uint32_t)(p.a_par * p.rows_a);
                         const uint32_t b_ks = 2u * (uint32_t)(MODE == MODE_FLAT_RESIDENT ? p.a.K_pad : p.n_tile);
                         const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.a.K_pad);
-                        if (MODE == MODE_FLAT_RESIDENT) {
+                        if (MODE == MODE_FLAT_RESIDENT && p.a.x_s2d) {
+                            // nine taps over the four parity images: each tap's operand starts at its own row of the stage
+                            for (int tap = 0; tap < 9; ++tap)
+                                issue_ksteps(ksteps, d_tmem, a_row + (uint32_t)p.tap_off[tap], b_tap + (uint32_t)tap * b_tap_step, a_ks, b_ks,
+                                             idesc, tap ? 1u : accumulate);
+                            accumulate = 1;
+                        } else if (MODE == MODE_FLAT_RESIDENT) {
                             if (p.a.R == 3 && p.a.S == 3)
                                 issue_flat_resident_k<3, 3>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
                             else if (p.a.R == 3)
@@ -425,7 +440,8 @@ conv_tc_kernel(const TcParams p) {
                             else
                                 issue_flat_resident_k<1, 1>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
                             accumulate = 1;
-                        } else
+                        } else {
+                        const uint32_t a_row0 = a_row;
                         for (int r = 0; r < p.a.R && ok; ++r) {
                             for (int sx = 0; sx < p.a.S; ++sx) {
                                 // streamed filters: one block per (K group, tap).  Every 128-position tile of the step
@@ -433,13 +449,15 @@ conv_tc_kernel(const TcParams p) {
                                 if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag, wait_limit)) { ok = false; break; }
                                 tc_fence_after();
                                 const uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
-                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_row + (uint32_t)sx + (uint32_t)(issuer * 128), b_lo,
-                                             a_ks, b_ks, idesc, accumulate);
+                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile),
+                                             (p.a.x_s2d ? a_row0 + (uint32_t)p.tap_off[r * 3 + sx] : a_row + (uint32_t)sx) + (uint32_t)(issuer * 128),
+                                             b_lo, a_ks, b_ks, idesc, accumulate);
                                 accumulate = 1;
                                 umma_commit(b_empty0 + 8 * b_stage);
                                 if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
                             }
                             a_row += (uint32_t)p.Wp_in;
+                        }
                         }
                         if (!ok) break;
                         umma_commit(a_empty0 + 8 * a_stage);     // releases the stage once these MMAs have read it
@@ -497,7 +515,17 @@ conv_tc_kernel(const TcParams p) {
             const int k_base = nt * p.n_tile;
             int cols = p.a.K_pad - k_base;
             if (cols > p.n_tile) cols = p.n_tile;
-            const long long vec0 = (long long)(k_base >> 3) * p.plane_out + f;     // vector of columns 0..7
+            const long long vec0 = (long long)(k_base >> 3) * p.plane_out + f;     // shortcut operand: vector of columns 0..7
+            // where the output goes: the same position - or, for a parity-split output tensor, pixel (h, w) of image n as
+            // pixel (h >> 1, w >> 1) of image pp * N + n, pp numbering the parities (h & 1, w & 1) as 00, 10, 11, 01 (the
+            // border positions go along: row -1 becomes row -1 of the odd-row images, and so on)
+            long long fy = f;
+            if (p.y_split) {
+                const int h = hp - 1, w = wq - 1;
+                const int pp = (h & 1) ? ((w & 1) ? 2 : 1) : ((w & 1) ? 3 : 0);
+                fy = ((long long)pp * p.a.N + n) * p.y_P2h + ((h >> 1) + 1) * p.y_Wh2 + ((w >> 1) + 1);
+            }
+            const long long yvec0 = (long long)(k_base >> 3) * p.plane_y + fy;
             int c_begin = 0, c_end = cols;
             if (EPI == 8) {
                 const int first = ((cols >> 4) + 1) / 2 * 16;                      // columns of the first half
@@ -605,7 +633,7 @@ conv_tc_kernel(const TcParams p) {
 #pragma unroll
                         for (int i = 0; i < 4; ++i) o2[i] = __floats2bfloat162_rn(fv[2 * i], fv[2 * i + 1]);
                     }
-                    y[(long long)q * p.plane_out + f] = o;
+                    y[(long long)q * p.plane_y + fy] = o;
                 }
             } else if (p.a.res_mode != 2) {
                 // Dense output, no shortcut or a same-shape one: the shortcut's vectors are requested 64 columns ahead into
@@ -619,7 +647,7 @@ conv_tc_kernel(const TcParams p) {
                     tmem_ld16(taddr + c0, v);
                     tmem_ld_wait();
                     if (!exists) return;
-                    uint4* yp = y + vec0 + (long long)(c0 >> 3) * p.plane_out;
+                    uint4* yp = y + yvec0 + (long long)(c0 >> 3) * p.plane_y;
                     const float4* b4 = reinterpret_cast<const float4*>(bias_s + k_base + c0);
 #pragma unroll
                     for (int ch = 0; ch < 2; ++ch) {
@@ -645,7 +673,7 @@ conv_tc_kernel(const TcParams p) {
                             o.z = pack_bf16x2(f4, f5); o.w = pack_bf16x2(f6, f7);
                         }
                         if (!interior) o = make_uint4(0, 0, 0, 0);
-                        yp[(long long)ch * p.plane_out] = o;
+                        yp[(long long)ch * p.plane_y] = o;
                     }
                 };
                 auto refill = [&](int c0, uint4& r0, uint4& r1) {     // shortcut vectors of columns c0 .. c0+15
@@ -668,7 +696,7 @@ conv_tc_kernel(const TcParams p) {
                 tmem_ld16(taddr + c0, v);
                 tmem_ld_wait();
                 if (exists) {
-                const long long out_vec = vec0 + (long long)(c0 >> 3) * p.plane_out;
+                const long long out_vec = yvec0 + (long long)(c0 >> 3) * p.plane_y;
                 uint4 o[2];
                 o[0] = make_uint4(0, 0, 0, 0);
                 o[1] = o[0];
@@ -728,7 +756,7 @@ conv_tc_kernel(const TcParams p) {
                     for (int i = 0; i < 8; ++i) o2[i] = __floats2bfloat162_rn(fv[2 * i], fv[2 * i + 1]);
                 }
                 y[out_vec] = o[0];
-                y[out_vec + p.plane_out] = o[1];
+                y[out_vec + p.plane_y] = o[1];
                 }
                 // rotate the residual queue and refill its tail
 #pragma unroll
@@ -888,6 +916,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     if (a.W > kMaxWidth || a.Q > kMaxWidth) { snprintf(err, err_len, "images wider than %d are not supported", kMaxWidth); return 1; }
     const int cchunks = a.C_pad / 8;
     const int taps = a.R * a.S;
+    const int a_par = a.x_s2d ? 4 : 1;       // activation runs per chunk in a stage (parity images)
     plan->flat = (a.stride == 1 && a.P == a.H && a.Q == a.W &&
                   ((a.R == 1 && a.S == 1 && a.pad == 0) || (a.R == 3 && (a.S == 3 || a.S == 1) && a.pad == 1))) ? 1 : 0;
     plan->cg = cchunks < 8 ? cchunks : 8;
@@ -917,6 +946,9 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         // streamed form, whose steps of several tiles share one halo, even though its filters would fit
         // (measured on the ResNet-18 stem at batch 64: 89 us resident, 61 us streamed).
         const bool wide_halo = 2 * plan->halo > 128;
+        // rows of one activation run: the step's positions with the halo before and after them (the taps of a strided
+        // window over parity images only reach back)
+        auto run_rows = [&](int tps) { return round_up_i(tps * 128 + (a_par > 1 ? 1 : 2) * plan->halo, 8); };
         bool stream = !bank_fits || wide_halo;
         const bool unified = stream && taps == 1;
         if (unified) {
@@ -959,13 +991,19 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             // Streamed filters: every filter block costs the issuing thread a barrier test, a fence and a commit on top
             // of its MMAs, so blocks of 12 chunks (six MMAs) instead of 8 (measured on ResNet-18, batch 64: the streamed
             // layers 8-15 % faster; 16 chunks need so much shared memory that multi-tile steps no longer fit).
-            if (!bank_fits) { plan->cg = cchunks < 12 ? cchunks : 12; plan->groups = (cchunks + plan->cg - 1) / plan->cg; }
+            if (!bank_fits && a_par == 1) { plan->cg = cchunks < 12 ? cchunks : 12; plan->groups = (cchunks + plan->cg - 1) / plan->cg; }
+            // four parity images per chunk: fewer chunks per stage, so that two stages and three filter blocks fit
+            while (a_par > 1 && plan->cg > 2 &&
+                   smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * (unsigned)(a_par * plan->cg * run_rows(1) * 16) > kSmemMax) {
+                plan->cg -= 2;
+                plan->groups = (cchunks + plan->cg - 1) / plan->cg;
+            }
             // Several 128-position tiles per step share every streamed filter block.  Layers with few positions
             // and many filters re-stream the bank once per position tile and are bound by L2 bandwidth, so
             // sharing pays even when it leaves only half of the SMs with a CTA (measured, same network: 368->512
             // filters at 7x7, 55 us with 164 single-tile CTAs, 32 us with 84 two-tile CTAs).
             for (int tps = 4; tps > 1; tps >>= 1) {
-                const unsigned a_try = (unsigned)(plan->cg * round_up_i(tps * 128 + 2 * plan->halo, 8) * 16);
+                const unsigned a_try = (unsigned)(a_par * plan->cg * run_rows(tps) * 16);
                 if (2 * tps * n_tile <= 512 && tps * 128 + plan->halo + 8 <= kGuardVectors &&
                     ((m_tiles + tps - 1) / tps) * n_tiles >= sms * 2 / 5 &&
                     smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * a_try <= kSmemMax) { plan->tps = tps; break; }
@@ -973,14 +1011,14 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         }
         if (bank_fits && wide_halo && plan->tps >= 2) bank_fits = false;
         else if (bank_fits) plan->tps = 1;
-        plan->rows_a = round_up_i(plan->tps * 128 + 2 * plan->halo, 8);
-        const unsigned a_stage = (unsigned)(plan->cg * plan->rows_a * 16);
+        plan->rows_a = run_rows(plan->tps);
+        unsigned a_stage = (unsigned)(a_par * plan->cg * plan->rows_a * 16);
         if (bank_fits) {
             plan->b_resident = 1;
             plan->b_stages = 1;
             const unsigned fixed = smem + (unsigned)round_up_i((int)bank, 128);
             auto fit = [&](int cg, int* stages) {
-                const unsigned st = (unsigned)(cg * plan->rows_a * 16);
+                const unsigned st = (unsigned)(a_par * cg * plan->rows_a * 16);
                 *stages = 4;
                 while (*stages > 2 && fixed + *stages * st > 110 * 1024) --*stages;
                 return fixed + *stages * st;
@@ -999,8 +1037,14 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
                     total = t4;
                 }
             }
+            while (total > kSmemMax && plan->cg > 2) {          // parity images: stages four times the size
+                plan->cg -= 2;
+                plan->groups = (cchunks + plan->cg - 1) / plan->cg;
+                total = fit(plan->cg, &plan->a_stages);
+            }
             smem = total;
         } else {
+            a_stage = (unsigned)(a_par * plan->cg * plan->rows_a * 16);
             plan->b_resident = 0;
             plan->b_stages = 8;      // filter blocks are small next to the copy latency: keep many in flight
             const unsigned b_stage = (unsigned)(plan->cg * n_tile * 16);
@@ -1080,9 +1124,24 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.a = a;
     p.Wp_in = a.W + 2; p.P2_in = (a.H + 2) * (a.W + 2);
     p.Qp = a.Q + 2; p.P2_out = (a.P + 2) * (a.Q + 2);
-    p.plane_in = (long long)a.N * p.P2_in;
+    p.plane_in = (long long)a.N * p.P2_in * (a.x_plane_mult > 1 || a.x_s2d ? 4 : 1);
     p.plane_out = (long long)a.N * p.P2_out;
     p.m_total = p.plane_out;
+    p.plane_y = p.plane_out;
+    if (a.y_split) {
+        p.y_split = 1; p.y_Wh2 = a.Q / 2 + 2; p.y_P2h = (a.P / 2 + 2) * p.y_Wh2;
+        p.plane_y = 4ll * a.N * p.y_P2h;
+    }
+    p.a_par = a.x_s2d ? 4 : 1;
+    p.par_stride = (long long)a.N * p.P2_in;
+    for (int t = 0; t < 9; ++t) {
+        // tap (r, s) of the 3x3 / stride-2 window reads input row 2p + r - 1: odd rows one row up for r = 0, even rows
+        // for r = 1, odd rows for r = 2; columns likewise.  Parity images in the order 00, 10, 11, 01.
+        const int r = t / 3, sx = t % 3;
+        const int pa = r == 1 ? 0 : 1, pb = sx == 1 ? 0 : 1;
+        const int pp = pa ? (pb ? 2 : 1) : (pb ? 3 : 0);
+        p.tap_off[t] = pp * plan.rows_a + plan.halo + (r == 0 ? -(a.W + 2) : 0) + (sx == 0 ? -1 : 0);
+    }
     p.taps = a.R * a.S; p.cchunks = a.C_pad / 8; p.cg = plan.cg; p.groups = plan.groups;
     p.halo = plan.halo; p.rows_a = plan.rows_a; p.a_stages = plan.a_stages; p.b_stages = plan.b_stages;
     p.n_tile = plan.n_tile; p.n_tiles = plan.n_tiles; p.tmem_cols = plan.tmem_cols;
@@ -1091,7 +1150,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.n_producers = plan.a_stages % 4 == 0 ? 4 : plan.a_stages % 3 == 0 ? 3 : plan.a_stages % 2 == 0 ? 2 : 1;
     p.total_tiles = (int)(((m_tiles + p.tps - 1) / p.tps) * plan.n_tiles);
     const int gplanes = plan.groups > 1 ? plan.cg : plan.tpk * p.cchunks;      // gather: planes per stage
-    p.a_stage_bytes = plan.flat ? plan.cg * plan.rows_a * 16 : gplanes * 128 * 16;
+    p.a_stage_bytes = plan.flat ? plan.cg * p.a_par * plan.rows_a * 16 : gplanes * 128 * 16;
     p.b_stage_bytes = plan.blocked_bank == 1 ? p.taps * plan.cg * plan.n_tile * 16 : plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
     p.bank_tile_bytes = (long long)p.taps * p.cchunks * plan.n_tile * 16;
     p.tpk = plan.tpk > 0 ? plan.tpk : 1;

@@ -58,6 +58,15 @@ struct ConvArgs {
     const int32_t* out_map;        // [out_C_pad], device
     const int32_t* tile_chunk0;    // [n_tiles + 1], device
     int n_tile_forced;             // > 0: filters per CTA tile fixed by the caller (scatter), else chosen by the plan
+    // Parity-split tensors (tensor-core path).  A tensor that only stride-2 convolutions read is stored as four
+    // half-resolution tensors, one per (row parity, column parity) of its pixels, in the order 00, 10, 11, 01, laid out
+    // as 4 N images of (H/2) x (W/2) pixels: image pp * N + n holds the pixels (2i + a, 2j + b) of image n.
+    int y_split;                   // write the output that way (the kernel's own grid stays P x Q)
+    int x_plane_mult;              // 0/1: x is a plain tensor; 4: x is a split tensor and this 1x1 layer reads its images
+                                   //      0 .. N-1 only (parity 00 = the pixels a 1x1 / stride-2 convolution reads)
+    int x_s2d;                     // x is a split tensor and this is the 3x3 / stride 2 / pad 1 convolution over the tensor
+                                   // it was split from: H, W, P, Q are the half resolution, stride is given as 1; the nine
+                                   // taps read the parity images at offsets -1 / 0 rows and columns
 };
 
 // Filter preparation --------------------------------------------------------------------
@@ -121,7 +130,7 @@ void launch_maxpool(const void* x, void* y, int is_bf16, int N, int H, int W, in
 void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, const float* fcw, const float* fcb,
                  int n_classes, float* logits, float* pool_scratch, cudaStream_t st);
 void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
-                               cudaStream_t st);
+                               int split, cudaStream_t st);
 
 // Convolutions ------------------------------------------------------------------------------
 // CUDA-core validation kernels: fp32 activations/filters, or bf16 activations/filters with

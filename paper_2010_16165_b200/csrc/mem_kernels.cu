@@ -398,9 +398,10 @@ __global__ void fc_kernel(const float* __restrict__ sums, int N, int C_pad, cons
 
 template <bool BF16>
 __global__ void planar_to_nchw_f32_kernel(const void* __restrict__ x, float* __restrict__ out, int N, int H, int W,
-                                          int chunks, int C_out) {
-    const int Wp = W + 2, P2 = (H + 2) * Wp;
-    const size_t plane = (size_t)N * P2;
+                                          int chunks, int C_out, int split) {
+    // a parity-split tensor (see ConvArgs) is 4 N images of half the size
+    const int Wp = split ? W / 2 + 2 : W + 2, P2 = split ? (H / 2 + 2) * Wp : (H + 2) * Wp;
+    const size_t plane = (size_t)N * P2 * (split ? 4 : 1);
     const size_t total = (size_t)N * chunks * H * W;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const int w = (int)(i % W);
@@ -409,7 +410,12 @@ __global__ void planar_to_nchw_f32_kernel(const void* __restrict__ x, float* __r
         const int j = (int)(t % chunks);
         const size_t n = t / chunks;
         float v[8];
-        load_vec8<BF16>(x, (size_t)j * plane + n * P2 + (size_t)(h + 1) * Wp + (w + 1), v);
+        size_t pos = n * P2 + (size_t)(h + 1) * Wp + (w + 1);
+        if (split) {
+            const int pp = (h & 1) ? ((w & 1) ? 2 : 1) : ((w & 1) ? 3 : 0);
+            pos = ((size_t)pp * N + n) * P2 + (size_t)((h >> 1) + 1) * Wp + ((w >> 1) + 1);
+        }
+        load_vec8<BF16>(x, (size_t)j * plane + pos, v);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const int c = j * 8 + e;
@@ -470,10 +476,10 @@ void launch_head(const void* x, int is_bf16, int N, int H, int W, int C_pad, con
 }
 
 void launch_planar_to_nchw_f32(const void* x, int is_bf16, float* out, int N, int H, int W, int C_pad, int C_out,
-                               cudaStream_t st) {
+                               int split, cudaStream_t st) {
     const size_t n = (size_t)N * (C_pad / 8) * H * W;
-    if (is_bf16) planar_to_nchw_f32_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(x, out, N, H, W, C_pad / 8, C_out);
-    else planar_to_nchw_f32_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(x, out, N, H, W, C_pad / 8, C_out);
+    if (is_bf16) planar_to_nchw_f32_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(x, out, N, H, W, C_pad / 8, C_out, split);
+    else planar_to_nchw_f32_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(x, out, N, H, W, C_pad / 8, C_out, split);
 }
 
 }  // namespace fp
