@@ -116,16 +116,25 @@ __device__ __forceinline__ void issue_ksteps_n(uint32_t d_tmem, uint32_t a_lo, u
 }
 __device__ __forceinline__ void issue_ksteps(int ksteps, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t a_ks,
                                              uint32_t b_ks, uint32_t idesc, uint32_t accumulate) {
-    switch (ksteps) {
-        case 1: issue_ksteps_n<1>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        case 2: issue_ksteps_n<2>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        case 3: issue_ksteps_n<3>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        case 4: issue_ksteps_n<4>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        case 5: issue_ksteps_n<5>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        case 6: issue_ksteps_n<6>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        case 7: issue_ksteps_n<7>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;
-        default: issue_ksteps_n<8>(d_tmem, a_lo, b_lo, a_ks, b_ks, idesc, accumulate); break;     // channel groups hold at most 16 chunks
+    // (a plain counted loop: a switch over unrolled bodies measured the same)
+#pragma unroll 1
+    for (int ks = 0; ks < ksteps; ++ks) {
+        umma_bf16_lo(d_tmem, a_lo, b_lo, idesc, ks ? 1u : accumulate);
+        a_lo += a_ks;
+        b_lo += b_ks;
     }
+}
+
+// The nine taps of a 3x3 / stride-2 window over parity images for one K group, fully unrolled: every tap's operand
+// starts at its own row of the stage (tap_off), its filters follow the previous tap's.  (As a loop over rows and columns
+// that looked its offset up by a computed index, each tap cost the issuing thread about 350 cycles - ResNet-50's
+// three strided 3x3 layers at batch 128: 51 / 48 / 47 us so, 33 / 28 / 27 us unrolled.)
+template <int KSTEPS>
+__device__ __forceinline__ void issue_taps9(uint32_t d_tmem, uint32_t a_row0, const int (&tap_off)[9], uint32_t b_lo, uint32_t b_tap,
+                                            uint32_t a_ks, uint32_t b_ks, uint32_t idesc, uint32_t accumulate) {
+#pragma unroll
+    for (int t = 0; t < 9; ++t)
+        issue_ksteps_n<KSTEPS>(d_tmem, a_row0 + (uint32_t)tap_off[t], b_lo + (uint32_t)t * b_tap, a_ks, b_ks, idesc, t ? 1u : accumulate);
 }
 
 // Shared-memory control block at the start of dynamic shared memory.
@@ -279,12 +288,15 @@ conv_tc_kernel(const TcParams p) {
                     const uint32_t fb = a_full0 + 8 * stage;
                     const uint32_t dst = a_base + stage * stage_bytes;
                     const uint32_t b_bytes = (uint32_t)(p.taps * cgg * p.n_tile * 16);
-                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16) + b_bytes);
+                    const int na = p.a_par * cgg;          // activation runs: one per chunk, or per chunk and parity image (<= 16)
+                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(na * p.rows_a * 16) + b_bytes);
                     __syncwarp();
-                    if (lane < cgg)
-                        bulk_copy(dst + lane * p.rows_a * 16, xv + (long long)(g * p.cg + lane) * p.plane_in + f0 - p.halo,
+                    if (lane < na) {
+                        const int c = p.a_par == 1 ? lane : lane >> 2, pp = p.a_par == 1 ? 0 : lane & 3;
+                        bulk_copy(dst + lane * p.rows_a * 16,
+                                  xv + (long long)(g * p.cg + c) * p.plane_in + (long long)pp * p.par_stride + f0 - p.halo,
                                   (uint32_t)(p.rows_a * 16), fb);
-                    else if (lane >= 16) {
+                    } else if (lane >= 16) {
                         // the group's filter block is one contiguous run of the bank: pieces of 16 KB, one per lane
                         const uint32_t off = (uint32_t)(lane - 16) * 16384u;
                         if (off < b_bytes)
@@ -387,7 +399,7 @@ conv_tc_kernel(const TcParams p) {
                 if (MODE == MODE_FLAT_UNIFIED) {
                     // one wait and one commit per stage; each tile of the step has its own issuing warp and accumulator
                     const uint32_t stage_bytes = (uint32_t)(p.a_stage_bytes + p.b_stage_bytes);
-                    const uint32_t a_ks = 2u * (uint32_t)p.rows_a, b_ks = 2u * (uint32_t)p.n_tile;
+                    const uint32_t a_ks = 2u * (uint32_t)(p.a_par * p.rows_a), b_ks = 2u * (uint32_t)p.n_tile;
                     const uint32_t d_acc = d_tmem + (uint32_t)(issuer * p.n_tile);
                     for (int g = 0; g < p.groups && ok; ++g) {
                         if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag, wait_limit)) { ok = false; break; }
@@ -396,9 +408,15 @@ conv_tc_kernel(const TcParams p) {
                         if (cgg > p.cg) cgg = p.cg;
                         const int ksteps = cgg >> 1;
                         const uint32_t sa = a_base + a_stage * stage_bytes;
-                        uint32_t a_row = ((sa >> 4) + (uint32_t)(issuer * 128)) | ((uint32_t)p.rows_a << 16);
+                        uint32_t a_row = ((sa >> 4) + (uint32_t)(issuer * 128)) | ((uint32_t)(p.a_par * p.rows_a) << 16);
+                        const uint32_t a_row0 = a_row;
                         uint32_t b_lo = ((sa + (uint32_t)p.a_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
                         const uint32_t b_tap = (uint32_t)(cgg * p.n_tile);
+                        if (p.a.x_s2d) {
+                            if (ksteps == 1) issue_taps9<1>(d_acc, a_row0, p.tap_off, b_lo, b_tap, a_ks, b_ks, idesc, accumulate);
+                            else issue_taps9<2>(d_acc, a_row0, p.tap_off, b_lo, b_tap, a_ks, b_ks, idesc, accumulate);
+                            accumulate = 1;
+                        } else
                         for (int r = 0; r < p.a.R; ++r) {
                             for (int sx = 0; sx < p.a.S; ++sx) {
                                 issue_ksteps(ksteps, d_acc, a_row + (uint32_t)sx, b_lo, a_ks, b_ks, idesc, accumulate);
@@ -428,6 +446,8 @@ conv_tc_kernel(const TcParams p) {
                         const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.a.K_pad);
                         if (MODE == MODE_FLAT_RESIDENT && p.a.x_s2d) {
                             // nine taps over the four parity images: each tap's operand starts at its own row of the stage
+                            // (unrolled: an index into the parameters that is not a constant costs some 300 cycles per use)
+#pragma unroll
                             for (int tap = 0; tap < 9; ++tap)
                                 issue_ksteps(ksteps, d_tmem, a_row + (uint32_t)p.tap_off[tap], b_tap + (uint32_t)tap * b_tap_step, a_ks, b_ks,
                                              idesc, tap ? 1u : accumulate);
@@ -441,7 +461,6 @@ conv_tc_kernel(const TcParams p) {
                                 issue_flat_resident_k<1, 1>(ksteps, d_tmem, a_row, b_tap, (uint32_t)p.Wp_in, a_ks, b_ks, b_tap_step, idesc, accumulate);
                             accumulate = 1;
                         } else {
-                        const uint32_t a_row0 = a_row;
                         for (int r = 0; r < p.a.R && ok; ++r) {
                             for (int sx = 0; sx < p.a.S; ++sx) {
                                 // streamed filters: one block per (K group, tap).  Every 128-position tile of the step
@@ -449,8 +468,7 @@ conv_tc_kernel(const TcParams p) {
                                 if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag, wait_limit)) { ok = false; break; }
                                 tc_fence_after();
                                 const uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
-                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile),
-                                             (p.a.x_s2d ? a_row0 + (uint32_t)p.tap_off[r * 3 + sx] : a_row + (uint32_t)sx) + (uint32_t)(issuer * 128),
+                                issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_row + (uint32_t)sx + (uint32_t)(issuer * 128),
                                              b_lo, a_ks, b_ks, idesc, accumulate);
                                 accumulate = 1;
                                 umma_commit(b_empty0 + 8 * b_stage);
@@ -950,9 +968,11 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         // window over parity images only reach back)
         auto run_rows = [&](int tps) { return round_up_i(tps * 128 + (a_par > 1 ? 1 : 2) * plan->halo, 8); };
         bool stream = !bank_fits || wide_halo;
-        const bool unified = stream && taps == 1;
+        const bool unified = stream && (taps == 1 || a_par > 1);
         if (unified) {
-            // 1x1 convolutions with a streamed bank.  A stage holds one K group of channel chunks: its activation
+            // 1x1 convolutions with a streamed bank, and 3x3 / stride-2 convolutions over parity images (whose activation
+            // part of a stage is four times a stride-1 layer's, so that the nine taps' filters beside it are in
+            // proportion).  A stage holds one K group of channel chunks: its activation
             // rows for the `tps` position tiles of a step and its filters - one wait and one commit per stage for the
             // issuing threads, one expected-bytes arrival for the producer.  The K group is the largest that still
             // leaves three stages (two in flight while one is read: at 60-100 B/cycle and a latency of one or two
@@ -966,9 +986,10 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             for (int tps = 4; tps >= 1 && !best_tps; tps >>= 1) {
                 if (2 * tps * n_tile > 512 || tps * 128 + plan->halo + 8 > kGuardVectors) continue;
                 if (tps > 1 && ((m_tiles + tps - 1) / tps) * n_tiles < sms / 2) continue;
-                const int rows = round_up_i(tps * 128 + 2 * plan->halo, 8);
-                for (int cg = (cchunks < 16 ? cchunks : 16) & ~1; cg >= 2; cg -= 2) {
-                    const unsigned st = (unsigned)(cg * rows * 16 + taps * cg * n_tile * 16);
+                const int rows = run_rows(tps);
+                // (parity images: four runs per chunk, at most 16 runs per stage)
+                for (int cg = a_par > 1 ? (cchunks < 4 ? cchunks : 4) : (cchunks < 16 ? cchunks : 16) & ~1; cg >= 2; cg -= 2) {
+                    const unsigned st = (unsigned)(a_par * cg * rows * 16 + taps * cg * n_tile * 16);
                     int stages = (int)(avail / st);
                     if (stages > kMaxStages) stages = kMaxStages;
                     if (stages == 7) stages = 6;          // the producer warps (2, 3 or 4 of them) must divide the stages
@@ -980,12 +1001,12 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             if (!best_tps) { snprintf(err, err_len, "tile does not fit shared memory"); return 1; }
             plan->tps = best_tps; plan->cg = best_cg; plan->a_stages = best_stages;
             plan->groups = (cchunks + best_cg - 1) / best_cg;
-            plan->rows_a = round_up_i(plan->tps * 128 + 2 * plan->halo, 8);
+            plan->rows_a = run_rows(plan->tps);
             plan->b_resident = 0;
             plan->b_stages = 0;
             plan->blocked_bank = 1;
             bank_fits = false;
-            smem += (unsigned)plan->a_stages * (unsigned)(plan->cg * plan->rows_a * 16 + taps * plan->cg * n_tile * 16);
+            smem += (unsigned)plan->a_stages * (unsigned)(a_par * plan->cg * plan->rows_a * 16 + taps * plan->cg * n_tile * 16);
         } else {
         if (stream) {
             // Streamed filters: every filter block costs the issuing thread a barrier test, a fence and a commit on top
