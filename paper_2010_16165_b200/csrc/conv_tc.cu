@@ -462,18 +462,19 @@ conv_tc_kernel(const TcParams p) {
                             accumulate = 1;
                         } else {
                         for (int r = 0; r < p.a.R && ok; ++r) {
+                            // streamed filters: one block per (K group, filter row).  Every 128-position tile of the step
+                            // uses it: its own accumulator and issuing warp, its activation rows 128 further on
+                            if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag, wait_limit)) { ok = false; break; }
+                            tc_fence_after();
+                            uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
                             for (int sx = 0; sx < p.a.S; ++sx) {
-                                // streamed filters: one block per (K group, tap).  Every 128-position tile of the step
-                                // uses it: its own accumulator and issuing warp, its activation rows 128 further on
-                                if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag, wait_limit)) { ok = false; break; }
-                                tc_fence_after();
-                                const uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
                                 issue_ksteps(ksteps, d_tmem + (uint32_t)(issuer * p.n_tile), a_row + (uint32_t)sx + (uint32_t)(issuer * 128),
                                              b_lo, a_ks, b_ks, idesc, accumulate);
                                 accumulate = 1;
-                                umma_commit(b_empty0 + 8 * b_stage);
-                                if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
+                                b_lo += (uint32_t)(cgg * p.n_tile);
                             }
+                            umma_commit(b_empty0 + 8 * b_stage);
+                            if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
                             a_row += (uint32_t)p.Wp_in;
                         }
                         }
@@ -794,8 +795,9 @@ conv_tc_kernel(const TcParams p) {
     } else if (MODE == MODE_FLAT_STREAM) {
         // ------------------------------ filter producer (streamed filters) --------------
         if (warp == 2 + EPI) {
-            // One filter block per (K group, tap).  When a tile takes all filters the block's chunks are one
-            // contiguous run of the packed bank: a single copy; otherwise one lane per chunk copies its rows.
+            // One filter block per (K group, filter row): [tap of the row][chunk][filter].  When a tile takes all filters
+            // a tap's chunks are one contiguous run of the packed bank: one copy per tap; otherwise one copy per
+            // (tap, chunk), spread over the lanes.
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             const bool whole = p.n_tiles == 1;
@@ -806,20 +808,24 @@ conv_tc_kernel(const TcParams p) {
                 for (int g = 0; g < p.groups && ok; ++g) {
                     int cgg = p.cchunks - g * p.cg;
                     if (cgg > p.cg) cgg = p.cg;
-                    for (int tap = 0; tap < p.taps; ++tap) {
+                    for (int r = 0; r < p.a.R; ++r) {
                         bool w = true;
                         if (lane == 0) w = mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit);
                         w = __shfl_sync(0xffffffffu, w, 0);
                         if (!w) { ok = false; break; }
                         const uint32_t fb = b_full0 + 8 * stage;
                         const uint32_t dst = b_base + stage * p.b_stage_bytes;
-                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
+                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(p.a.S * cgg * nrows * 16));
                         __syncwarp();
-                        const uint4* src = wv + ((long long)tap * p.cchunks + g * p.cg) * p.a.K_pad + nt * p.n_tile;
+                        const uint4* src = wv + ((long long)(r * p.a.S) * p.cchunks + g * p.cg) * p.a.K_pad + nt * p.n_tile;
                         if (whole) {
-                            if (lane == 0) bulk_copy(dst, src, (uint32_t)(cgg * nrows * 16), fb);
-                        } else if (lane < cgg) {
-                            bulk_copy(dst + lane * p.n_tile * 16, src + (long long)lane * p.a.K_pad, (uint32_t)(nrows * 16), fb);
+                            if (lane < p.a.S)
+                                bulk_copy(dst + lane * cgg * p.n_tile * 16, src + (long long)lane * p.cchunks * p.a.K_pad, (uint32_t)(cgg * nrows * 16), fb);
+                        } else {
+                            for (int i = lane; i < p.a.S * cgg; i += 32) {
+                                const int sx = i / cgg, c = i - sx * cgg;
+                                bulk_copy(dst + i * p.n_tile * 16, src + ((long long)sx * p.cchunks + c) * p.a.K_pad, (uint32_t)(nrows * 16), fb);
+                            }
                         }
                         if (++stage == (uint32_t)p.b_stages) { stage = 0; phase ^= 1; }
                     }
@@ -1009,26 +1015,27 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
             smem += (unsigned)plan->a_stages * (unsigned)(a_par * plan->cg * plan->rows_a * 16 + taps * plan->cg * n_tile * 16);
         } else {
         if (stream) {
-            // Streamed filters: every filter block costs the issuing thread a barrier test, a fence and a commit on top
-            // of its MMAs, so blocks of 12 chunks (six MMAs) instead of 8 (measured on ResNet-18, batch 64: the streamed
-            // layers 8-15 % faster; 16 chunks need so much shared memory that multi-tile steps no longer fit).
-            if (!bank_fits && a_par == 1) { plan->cg = cchunks < 12 ? cchunks : 12; plan->groups = (cchunks + plan->cg - 1) / plan->cg; }
-            // four parity images per chunk: fewer chunks per stage, so that two stages and three filter blocks fit
-            while (a_par > 1 && plan->cg > 2 &&
-                   smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * (unsigned)(a_par * plan->cg * run_rows(1) * 16) > kSmemMax) {
-                plan->cg -= 2;
-                plan->groups = (cchunks + plan->cg - 1) / plan->cg;
-            }
-            // Several 128-position tiles per step share every streamed filter block.  Layers with few positions
-            // and many filters re-stream the bank once per position tile and are bound by L2 bandwidth, so
-            // sharing pays even when it leaves only half of the SMs with a CTA (measured, same network: 368->512
-            // filters at 7x7, 55 us with 164 single-tile CTAs, 32 us with 84 two-tile CTAs).
-            for (int tps = 4; tps > 1; tps >>= 1) {
-                const unsigned a_try = (unsigned)(a_par * plan->cg * run_rows(tps) * 16);
-                if (2 * tps * n_tile <= 512 && tps * 128 + plan->halo + 8 <= kGuardVectors &&
-                    ((m_tiles + tps - 1) / tps) * n_tiles >= sms * 2 / 5 &&
-                    smem + 3u * (unsigned)(plan->cg * n_tile * 16) + 2u * a_try <= kSmemMax) { plan->tps = tps; break; }
-            }
+            // Streamed filters: a filter block holds one filter row (S taps) of a K group.  Every block costs the issuing
+            // thread a barrier test, a fence and a commit (some 300 cycles) on top of its MMAs, and a block per tap left a
+            // third of the main loop to that.  Several 128-position tiles per step share every block: layers with few
+            // positions and many filters re-stream the bank once per position tile and are bound by L2 bandwidth, so
+            // sharing pays even when it leaves only half of the SMs with a CTA (measured on ResNet-18 at batch 64:
+            // 368->512 filters at 7x7, 55 us with 164 single-tile CTAs, 32 us with 84 two-tile CTAs).  The search prefers
+            // three blocks in flight over two, then more tiles per step, then longer K groups.
+            bool found = false;
+            for (int want_b = 3; want_b >= 2 && !found; --want_b)
+                for (int tps = 4; tps >= 1 && !found; tps >>= 1) {
+                    if (2 * tps * n_tile > 512 || tps * 128 + plan->halo + 8 > kGuardVectors) continue;
+                    if (tps > 1 && ((m_tiles + tps - 1) / tps) * n_tiles < sms * 2 / 5) continue;
+                    const int cg_hi = bank_fits ? plan->cg : (cchunks < 12 ? cchunks : 12), cg_lo = bank_fits ? plan->cg : (cchunks < 4 ? cchunks : 4);
+                    for (int cg = cg_hi; cg >= cg_lo && !found; cg -= 2) {
+                        const unsigned b_try = (unsigned)(a.S * cg * n_tile * 16), a_try = (unsigned)(cg * run_rows(tps) * 16);
+                        if (smem + (unsigned)want_b * b_try + 2u * a_try > kSmemMax) continue;
+                        found = true;
+                        plan->tps = tps; plan->cg = cg; plan->groups = (cchunks + cg - 1) / cg;
+                    }
+                }
+            if (!found && !bank_fits) { snprintf(err, err_len, "tile does not fit shared memory"); return 1; }
         }
         if (bank_fits && wide_halo && plan->tps >= 2) bank_fits = false;
         else if (bank_fits) plan->tps = 1;
@@ -1067,8 +1074,8 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         } else {
             a_stage = (unsigned)(a_par * plan->cg * plan->rows_a * 16);
             plan->b_resident = 0;
-            plan->b_stages = 8;      // filter blocks are small next to the copy latency: keep many in flight
-            const unsigned b_stage = (unsigned)(plan->cg * n_tile * 16);
+            plan->b_stages = 4;
+            const unsigned b_stage = (unsigned)(a.S * plan->cg * n_tile * 16);
             plan->a_stages = plan->tps > 1 ? 2 : 3;
             while (plan->a_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->a_stages;
             while (plan->b_stages > 2 && smem + plan->b_stages * b_stage + plan->a_stages * a_stage > kSmemMax) --plan->b_stages;
@@ -1172,7 +1179,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.total_tiles = (int)(((m_tiles + p.tps - 1) / p.tps) * plan.n_tiles);
     const int gplanes = plan.groups > 1 ? plan.cg : plan.tpk * p.cchunks;      // gather: planes per stage
     p.a_stage_bytes = plan.flat ? plan.cg * p.a_par * plan.rows_a * 16 : gplanes * 128 * 16;
-    p.b_stage_bytes = plan.blocked_bank == 1 ? p.taps * plan.cg * plan.n_tile * 16 : plan.flat ? plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
+    p.b_stage_bytes = plan.blocked_bank == 1 ? p.taps * plan.cg * plan.n_tile * 16 : plan.flat ? a.S * plan.cg * plan.n_tile * 16 : gplanes * plan.n_tile * 16;
     p.bank_tile_bytes = (long long)p.taps * p.cchunks * plan.n_tile * 16;
     p.tpk = plan.tpk > 0 ? plan.tpk : 1;
     p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
