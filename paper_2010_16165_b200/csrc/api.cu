@@ -947,7 +947,7 @@ fp_status replan(fp_handle h) {
                 int32_t* d_row;
                 TRY(upload_i32(h, row_src, &d_row));
                 f.d_row = d_row; f.d_chan = nullptr;
-                TRY(dev_alloc(h, h->pack_buffers, &f.d_wp, (size_t)160 * f.K_pad * 2));
+                TRY(dev_alloc(h, h->pack_buffers, &f.d_wp, (size_t)256 * f.K_pad * 2));
                 TRY(dev_alloc(h, h->pack_buffers, (void**)&f.d_bp, (size_t)f.K_pad * sizeof(float)));
                 fp::launch_repack_stem_direct(f.d_w32, f.C, d_row, f.K_pad, (__nv_bfloat16*)f.d_wp, st);
                 fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);

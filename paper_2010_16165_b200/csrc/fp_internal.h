@@ -172,7 +172,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
 struct StemPoolArgs {
     const void* x;        // network input, N x C x H x W, NCHW, bf16
     void* y;              // pooled tensor, planar-8 with border, (H/4) x (W/4) pixels, K_pad channels, N images
-    const void* w;        // filters [20 chunks of 8 k][K_pad rows][8] bf16, k = (r * C + c) * 7 + s, zero for k >= 49 C
+    const void* w;        // filters [16 taps (ta, tb)][2 chunks of 8][K_pad rows][8] bf16 over the parity channels (launch_repack_stem_direct)
     const float* bias;    // [K_pad]
     int N, C, H, W, K_pad;
     int n0, n_count;      // the images this launch handles (the tensor's plane pitch is that of all N)

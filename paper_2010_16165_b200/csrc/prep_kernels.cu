@@ -217,17 +217,21 @@ __global__ void repack_stem_kernel(const float* __restrict__ w, int C, const int
     }
 }
 
+// Filters of the first convolution for the kernel that fuses it with the pooling: the 7x7 / stride-2 window over C
+// channels as a 4x4 window over the 4 C parity channels of the half-resolution input - tap (ta, tb), channel
+// (2a + b) C + c takes w[k][c][2 ta + a - 1][2 tb + b - 1] (zero where an index is -1) - as [tap][chunk of 8][filter][8].
 __global__ void repack_stem_direct_kernel(const float* __restrict__ w, int C, const int32_t* __restrict__ row_src, int K_pad,
                                           __nv_bfloat16* __restrict__ out) {
-    const int total = 20 * K_pad * 8;
+    const int total = 16 * 2 * K_pad * 8;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-        const int e = i % 8, kr = (i / 8) % K_pad, chunk = i / (8 * K_pad);
-        const int k = chunk * 8 + e;
+        const int e = i % 8, kr = (i / 8) % K_pad, chunk = (i / (8 * K_pad)) % 2, tap = i / (16 * K_pad);
+        const int ch = chunk * 8 + e, ta = tap >> 2, tb = tap & 3;
         float v = 0.0f;
         const int ks = row_src[kr];
-        if (ks >= 0 && k < 49 * C) {
-            const int rc = k / 7, s = k - rc * 7, r = rc / C, c = rc - r * C;
-            v = w[(((size_t)ks * C + c) * 7 + r) * 7 + s];
+        if (ks >= 0 && ch < 4 * C) {
+            const int par = ch / C, c = ch - par * C;
+            const int r = 2 * ta + (par >> 1) - 1, s = 2 * tb + (par & 1) - 1;
+            if (r >= 0 && s >= 0) v = w[(((size_t)ks * C + c) * 7 + r) * 7 + s];
         }
         out[i] = __float2bfloat16_rn(v);
     }
@@ -343,7 +347,7 @@ void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad
 }
 
 void launch_repack_stem_direct(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st) {
-    repack_stem_direct_kernel<<<blocks_for((size_t)160 * K_pad, 256), 256, 0, st>>>(w, C, row_src, K_pad, out);
+    repack_stem_direct_kernel<<<blocks_for((size_t)256 * K_pad, 256), 256, 0, st>>>(w, C, row_src, K_pad, out);
 }
 
 void launch_reblock_bank(const __nv_bfloat16* packed, int RS, int cchunks, int K_pad, int n_tile, int n_tiles, int cg,

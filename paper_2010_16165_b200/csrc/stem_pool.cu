@@ -9,10 +9,17 @@
 //                  with bulk copies into shared memory (16 bytes of zeros on either side of a row are the horizontal
 //                  padding, rows outside the image are cleared by the threads); the next unit's rows are requested
 //                  while this unit is computed.
-//   GEMM           M = the unit's 5 x (W/2) convolution positions in tiles of 128, N = K_pad filters, K = 49 C taps
-//                  padded to 160.  All threads build a tile's A operand (K-major, 16-byte rows: 8 consecutive k of one
-//                  position) from the staged rows through a table of offsets, two A buffers, one thread issues the
-//                  tcgen05 MMAs; the five accumulators stay in tensor memory until the unit's last MMA.
+//   GEMM           The 7x7 / stride-2 window over C channels is a 4x4 / stride-1 window over the 4 C channels of the
+//                  input's four pixel parities at half resolution (input row 2i + a, column 2j + b -> channel
+//                  (2a + b) C + c of half-resolution pixel (i, j); filter tap r = 2 ta + a - 1, s = 2 tb + b - 1, the taps
+//                  with r or s = -1 being zero).  The compute warps rewrite a unit's staged rows once into that form
+//                  - planar, 16 channels in two chunks of 8, eight half-resolution rows of W/2 + 3 pixels - and the
+//                  convolution is then sixteen taps of one K = 16 step each over FLAT positions of that grid, the operand
+//                  of tap (ta, tb) being the same rows ta * pitch + tb further on: no per-position gathering.  M = the
+//                  unit's 5 x pitch positions in tiles of 128 (the three pad columns per row are computed and dropped),
+//                  N = K_pad filters.  One thread issues the tcgen05 MMAs of a unit while the compute warps pool the
+//                  previous unit and rewrite the next one's rows (two parity buffers); the accumulators of the unit's
+//                  tiles stay in tensor memory until the epilogue has read them.
 //   Epilogue       tcgen05.ld -> bias -> ReLU -> bf16 into a shared-memory copy of the five convolution rows (zeros for
 //                  rows outside the image: after the ReLU a zero never wins a window it should not), then the 3x3
 //                  maxima, written with 16-byte stores, 512 contiguous bytes per warp; the units at an image's
@@ -33,21 +40,23 @@ namespace {
 
 constexpr int kBuildWarps = 8;             // compute warps; one more warp fetches the input, another issues the MMAs
 constexpr int kThreads = 32 * (kBuildWarps + 2);
-constexpr int kKChunks = 20;               // K = 160 >= 49 * 3
-constexpr int kRowsIn = 15, kConvRows = 5;
+constexpr int kTaps = 16;                  // 4 x 4 taps over the parity channels, one K = 16 step each
+constexpr int kRowsIn = 15, kConvRows = 5, kHalfRows = 8;
+constexpr int kMaxTiles = 8;
 
 struct SpParams {
     StemPoolArgs a;
     int Hc, Wc, Hp, Wp;            // convolution and pooled sizes
     int pitch;                     // elements per staged input row: W + 16
     int in_bytes;                  // one input buffer: C * 15 * pitch * 2
-    int a_bytes;                   // one A tile: 20 * 128 * 16
-    int b_bytes;                   // filters: 20 * K_pad * 16
+    int pitch_x;                   // half-resolution pixels per row of the parity form: Wc + 3 (columns -2 .. Wc)
+    int x_rows;                    // 16-byte rows per chunk of a parity buffer (8 * pitch_x, plus what the last tile's taps reach)
+    int b_bytes;                   // filters: 16 taps * 2 chunks * K_pad * 16
     int conv_pos;                  // 5 * Wc
-    int tiles;                     // ceil(conv_pos / 128)
+    int tiles;                     // ceil(5 * pitch_x / 128)
     int units_per_image, n_units;  // Hp / 2 (rounded up); images x that
     int tmem_cols;
-    FastDiv div_wc, div_upi, div_wp2;
+    FastDiv div_px, div_upi;
     int* status;
 };
 
@@ -55,54 +64,40 @@ struct SpCtrl {
     uint64_t in_full[2];
     uint64_t in_empty[2];
     uint64_t b_full;
-    uint64_t mma_done[2];
-    uint64_t a_full[2];
+    uint64_t x_full[2];
+    uint64_t tmem_free;
+    uint64_t mma_done[kMaxTiles];
     uint32_t tmem_base;
     int abort_flag;
-    int koff[kKChunks * 8];        // k -> element offset of tap (r, s, c) from a position's window origin
 };
 
-// A position's 147 taps for three input channels, k = (r * 3 + c) * 7 + s, as the K-major operand rows of one half
-// (k in [80 HALF, 80 HALF + 80)) of its 160 k.  The window of a (row, channel) starts at an odd element (column 2w - 3
-// behind 8 elements of padding), so its element 0 is a 16-bit load and (1,2), (3,4), (5,6) are aligned 32-bit loads: 84
-// shared-memory loads per position instead of 147 - the builder is bound by the load/store unit's issue rate.
-// Everything is unrolled: which loads a half needs and where their halves go are compile-time facts.
-template <int HALF>
-__device__ __forceinline__ void build_rgb(const unsigned short* origin, int pitch, uint4* a_dst) {
-    uint32_t wd[40];
+// The staged rows of a unit (C channels x 15 input rows, 8 zero elements on either side of a row) rewritten as the
+// parity form: half-resolution row h (0..7) holds input rows 2h - 1 (parity 0; none for h = 0: zeros, its taps are zero)
+// and 2h (parity 1) of the staged window, pixel jx (0 .. pitch_x - 1) the input columns 2 (jx - 2) and 2 (jx - 2) + 1 -
+// one aligned 32-bit load per (row parity, channel) gives both column parities.  Channel (2a + b) C + c.
+template <int C>
+__device__ __forceinline__ void parity_rows(const unsigned short* in_buf, int pitch, uint4* x_buf, int x_rows, int pitch_x,
+                                            FastDiv div_px, int tid) {
+    const int total = kHalfRows * pitch_x;
+    for (int i = tid; i < total; i += 32 * kBuildWarps) {
+        const int h = (int)fdiv((uint32_t)i, div_px), jx = i - h * pitch_x;
+        uint32_t hv[16];
 #pragma unroll
-    for (int i = 0; i < 40; ++i) wd[i] = 0u;
+        for (int e = 0; e < 16; ++e) hv[e] = 0u;
 #pragma unroll
-    for (int rc = 0; rc < 21; ++rc) {
-        const int k0 = rc * 7;                               // k of this window's element 0
-        if (k0 + 6 < 80 * HALF || k0 >= 80 * HALF + 80) continue;
-        const int r = rc / 3, c = rc - 3 * r;
-        const unsigned short* wdw = origin + (c * kRowsIn + r) * pitch;
-        uint32_t e[7];
-        const bool need0 = k0 >= 80 * HALF && k0 < 80 * HALF + 80;
-        if (need0) e[0] = wdw[0];
+        for (int a = 0; a < 2; ++a) {
+            const int r = 2 * h - 1 + a;
 #pragma unroll
-        for (int pr = 0; pr < 3; ++pr) {
-            const int ka = k0 + 1 + 2 * pr, kb = ka + 1;
-            const bool na = ka >= 80 * HALF && ka < 80 * HALF + 80, nb = kb >= 80 * HALF && kb < 80 * HALF + 80;
-            if (na || nb) {
-                const uint32_t pair = *reinterpret_cast<const uint32_t*>(wdw + 1 + 2 * pr);
-                e[1 + 2 * pr] = pair & 0xffffu;
-                e[2 + 2 * pr] = pair >> 16;
+            for (int c = 0; c < C; ++c) {
+                uint32_t pair = 0u;
+                if (r >= 0) pair = *reinterpret_cast<const uint32_t*>(in_buf + (c * kRowsIn + r) * pitch + 4 + 2 * jx);
+                hv[(2 * a) * C + c] = pair & 0xffffu;
+                hv[(2 * a + 1) * C + c] = pair >> 16;
             }
         }
-#pragma unroll
-        for (int sx = 0; sx < 7; ++sx) {
-            const int k = k0 + sx;
-            if (k >= 80 * HALF && k < 80 * HALF + 80) {
-                const int kk = k - 80 * HALF;
-                wd[kk >> 1] |= (kk & 1) ? (e[sx] << 16) : e[sx];
-            }
-        }
+        x_buf[i] = make_uint4(hv[0] | (hv[1] << 16), hv[2] | (hv[3] << 16), hv[4] | (hv[5] << 16), hv[6] | (hv[7] << 16));
+        x_buf[x_rows + i] = make_uint4(hv[8] | (hv[9] << 16), hv[10] | (hv[11] << 16), hv[12] | (hv[13] << 16), hv[14] | (hv[15] << 16));
     }
-#pragma unroll
-    for (int cc = 0; cc < 10; ++cc)
-        a_dst[(10 * HALF + cc) * 128] = make_uint4(wd[4 * cc], wd[4 * cc + 1], wd[4 * cc + 2], wd[4 * cc + 3]);
 }
 
 // barrier 1: the compute warps only (the input producer runs on its own)
@@ -125,35 +120,33 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
     const uint32_t ctrl_bytes = (uint32_t)((sizeof(SpCtrl) + 127) & ~127u);
     float* bias_s = reinterpret_cast<float*>(smem_raw + ctrl_bytes);                         // K_pad floats
     const uint32_t b_addr = (base + ctrl_bytes + (uint32_t)p.a.K_pad * 4u + 1023u) & ~1023u;
-    const uint32_t a_addr = b_addr + (uint32_t)((p.b_bytes + 127) & ~127);
-    const uint32_t in_addr = a_addr + 2u * (uint32_t)p.a_bytes;
+    const uint32_t x_addr = b_addr + (uint32_t)((p.b_bytes + 127) & ~127);
+    const uint32_t x_bytes = 2u * (uint32_t)p.x_rows * 16u;                                  // one parity buffer: two chunks
+    const uint32_t in_addr = x_addr + 2u * x_bytes;
     const uint32_t conv_addr = in_addr + 2u * (uint32_t)p.in_bytes;
     uint8_t* in_ptr = smem_raw + (in_addr - base);
     uint8_t* conv_ptr = smem_raw + (conv_addr - base);
+    uint8_t* x_ptr = smem_raw + (x_addr - base);
     volatile int* abort_flag = &ctrl->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t in_full0 = base + (uint32_t)offsetof(SpCtrl, in_full);
+    const uint32_t in_empty0 = base + (uint32_t)offsetof(SpCtrl, in_empty);
     const uint32_t b_full = base + (uint32_t)offsetof(SpCtrl, b_full);
+    const uint32_t x_full0 = base + (uint32_t)offsetof(SpCtrl, x_full);
+    const uint32_t tmem_free = base + (uint32_t)offsetof(SpCtrl, tmem_free);
     const uint32_t mma_done0 = base + (uint32_t)offsetof(SpCtrl, mma_done);
     const int C = p.a.C, K_pad = p.a.K_pad, chunks_out = K_pad >> 3;
 
     if (threadIdx.x == 0) {
         mbar_init(in_full0, 1); mbar_init(in_full0 + 8, 1);
-        mbar_init(base + (uint32_t)offsetof(SpCtrl, in_empty), 1); mbar_init(base + (uint32_t)offsetof(SpCtrl, in_empty) + 8, 1);
+        mbar_init(in_empty0, 32 * kBuildWarps); mbar_init(in_empty0 + 8, 32 * kBuildWarps);
         mbar_init(b_full, 1);
-        mbar_init(mma_done0, 1); mbar_init(mma_done0 + 8, 1);
-        mbar_init(base + (uint32_t)offsetof(SpCtrl, a_full), 32 * kBuildWarps); mbar_init(base + (uint32_t)offsetof(SpCtrl, a_full) + 8, 32 * kBuildWarps);
+        mbar_init(x_full0, 32 * kBuildWarps); mbar_init(x_full0 + 8, 32 * kBuildWarps);
+        mbar_init(tmem_free, 32 * kBuildWarps);
+        for (int t = 0; t < kMaxTiles; ++t) mbar_init(mma_done0 + 8 * t, 1);
         ctrl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    for (int k = threadIdx.x; k < kKChunks * 8; k += kThreads) {
-        int off = 0;
-        if (k < 49 * C) {
-            const int rc = k / 7, s = k - rc * 7, r = rc / C, c = rc - r * C;
-            off = (c * kRowsIn + r) * p.pitch + s;
-        }
-        ctrl->koff[k] = off;
     }
     for (int i = threadIdx.x; i < K_pad; i += kThreads) bias_s[i] = p.a.bias[i];
     // the 16 bytes on either side of every staged row stay zero for the whole kernel: copies never touch them
@@ -162,11 +155,15 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
         row[0] = make_uint4(0, 0, 0, 0);
         row[(p.pitch * 2) / 16 - 1] = make_uint4(0, 0, 0, 0);
     }
+    // the parity buffers' rows behind the eight half-resolution rows are read by the last tile's taps (for positions that
+    // are dropped) and never written: zeros, so that no NaN pattern reaches an accumulator
+    for (int i = threadIdx.x; i < (int)(2u * x_bytes / 16u); i += kThreads) reinterpret_cast<uint4*>(x_ptr)[i] = make_uint4(0, 0, 0, 0);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(base + (uint32_t)offsetof(SpCtrl, tmem_base)), "r"((uint32_t)p.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -188,7 +185,6 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
     const int Wq = p.Wp + 2, P2o = (p.Hp + 2) * Wq;
     const long long plane_out = (long long)p.a.N * P2o;
 
-    const uint32_t in_empty0 = base + (uint32_t)offsetof(SpCtrl, in_empty);
     bool ok = true;
 
     if (warp == kBuildWarps) {
@@ -230,113 +226,84 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
         if (!ok && lane == 0) { atomicExch(&ctrl->abort_flag, 1); atomicExch(p.status, 6); }
     } else if (warp == kBuildWarps + 1) {
         // ------------------------------ MMA issuer ------------------------------
-        // One thread: waits until every compute thread has stored its part of a tile's operand, issues the tile's MMAs and
-        // commits them to the barrier that frees the operand buffer (and, behind a unit's last tile, tells the compute
-        // warps that the accumulators are complete).  A thread of its own, so that the compute warps go on building.
+        // One thread: waits until the compute threads have rewritten a unit's rows and have read the previous unit's
+        // accumulators, then issues the unit's MMAs - per tile of 128 flat positions sixteen taps of one K = 16 step,
+        // the operand of tap (ta, tb) starting ta * pitch + tb rows further on - and commits every tile to a barrier of
+        // its own, so that the epilogue starts on the first tile while the others are computed.
         if (lane == 0) {
-            const uint32_t a_full0 = base + (uint32_t)offsetof(SpCtrl, a_full);
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(K_pad >> 3) << 17) | ((128u >> 4) << 24);
-            uint32_t full_phase[2] = {0, 0};
             ok = mbar_wait(b_full, 0, abort_flag);
             int it = 0;
             for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x, ++it) {
+                const int xb = it & 1;
+                if (!mbar_wait(x_full0 + 8 * xb, (uint32_t)((it >> 1) & 1), abort_flag)) { ok = false; break; }
+                if (it > 0 && !mbar_wait(tmem_free, (uint32_t)((it - 1) & 1), abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_unit = ((x_addr + xb * x_bytes) >> 4) | ((uint32_t)p.x_rows << 16);
+                const uint32_t b_lo0 = (b_addr >> 4) | ((uint32_t)K_pad << 16);
                 for (int t = 0; t < p.tiles; ++t) {
-                    const int ab = t & 1;
-                    if (!mbar_wait(a_full0 + 8 * ab, full_phase[ab], abort_flag)) { ok = false; break; }
-                    full_phase[ab] ^= 1;
-                    tc_fence_after();
-                    uint32_t a_lo = ((a_addr + ab * p.a_bytes) >> 4) | (128u << 16);
-                    uint32_t b_lo = (b_addr >> 4) | ((uint32_t)K_pad << 16);
                     const uint32_t d = tmem_base + (uint32_t)(t * K_pad);
+                    uint32_t a_row = a_unit + (uint32_t)(t * 128);
+                    uint32_t b_lo = b_lo0;
 #pragma unroll
-                    for (int ks = 0; ks < kKChunks / 2; ++ks) {
-                        umma_bf16_lo(d, a_lo, b_lo, idesc, ks ? 1u : 0u);
-                        a_lo += 256u;
-                        b_lo += 2u * (uint32_t)K_pad;
+                    for (int ta = 0; ta < 4; ++ta) {
+#pragma unroll
+                        for (int tb = 0; tb < 4; ++tb) {
+                            umma_bf16_lo(d, a_row + (uint32_t)tb, b_lo, idesc, (ta | tb) ? 1u : 0u);
+                            b_lo += 2u * (uint32_t)K_pad;
+                        }
+                        a_row += (uint32_t)p.pitch_x;
                     }
-                    umma_commit(mma_done0 + 8 * ab);
-                    // the last tile has been built: the staged input rows are free for the unit after the next
-                    if (t == p.tiles - 1) mbar_arrive(in_empty0 + 8 * (it & 1));
+                    umma_commit(mma_done0 + 8 * t);
                 }
             }
             if (!ok) { atomicExch(&ctrl->abort_flag, 1); atomicExch(p.status, 6); }
         }
     } else {
     // ------------------------------ the eight compute warps ------------------------------
-    {   // filters have to be in before the first MMA; every thread waits (cheap) so that the vote below is uniform
+    {   // (every thread waits for the filters - cheap - so that the vote below is uniform)
         const bool w = mbar_wait(b_full, 0, abort_flag);
         ok = !bar_or(!w);
     }
-    uint32_t in_phase[2] = {0, 0}, mma_phase[2] = {0, 0};
-    int it = 0;
-    for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x, ++it) {
+    uint32_t in_phase[2] = {0, 0};
+    // rewrites the staged rows of the CTA's unit number `it` into parity buffer it & 1 and hands both on
+    auto rewrite = [&](int it) -> bool {
         const int buf = it & 1;
+        const bool w = mbar_wait(in_full0 + 8 * buf, in_phase[buf], abort_flag);
+        in_phase[buf] ^= 1;
+        if (bar_or(!w)) return false;
+        const unsigned short* in_buf = reinterpret_cast<const unsigned short*>(in_ptr + (size_t)buf * p.in_bytes);
+        uint4* x_buf = reinterpret_cast<uint4*>(x_ptr + (size_t)buf * x_bytes);
+        if (C == 3) parity_rows<3>(in_buf, p.pitch, x_buf, p.x_rows, p.pitch_x, p.div_px, threadIdx.x);
+        else if (C == 2) parity_rows<2>(in_buf, p.pitch, x_buf, p.x_rows, p.pitch_x, p.div_px, threadIdx.x);
+        else parity_rows<1>(in_buf, p.pitch, x_buf, p.x_rows, p.pitch_x, p.div_px, threadIdx.x);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> MMA reads
+        mbar_arrive(x_full0 + 8 * buf);
+        mbar_arrive(in_empty0 + 8 * buf);                              // the staged rows are free for the unit after the next
+        return true;
+    };
+    int it = 0;
+    if (blockIdx.x < p.n_units) ok = ok && rewrite(0);
+    for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x, ++it) {
         const int img = (int)fdiv((uint32_t)u, p.div_upi);
         const int pr = u - img * p.units_per_image;
         const int n = p.a.n0 + img;
-        {
-            const bool w = mbar_wait(in_full0 + 8 * buf, in_phase[buf], abort_flag);
-            in_phase[buf] ^= 1;
-            if (bar_or(!w)) { ok = false; break; }
-        }
-        const uint32_t in_buf = in_addr + buf * p.in_bytes;
-
-        // ---- convolution: build A tile by tile, MMAs behind ----
-        for (int t = 0; t < p.tiles; ++t) {
-            const int ab = t & 1;
-            bool w = true;
-            if (t >= 2) { w = mbar_wait(mma_done0 + 8 * ab, mma_phase[ab], abort_flag); mma_phase[ab] ^= 1; }
-            const int m = t * 128 + (threadIdx.x & 127);
-            if (w && m < p.conv_pos) {
-                const int j = (int)fdiv((uint32_t)m, p.div_wc), wc = m - j * p.Wc;
-                const unsigned short* origin = reinterpret_cast<const unsigned short*>(smem_raw + (in_buf - base)) +
-                                               ((2 * j) * p.pitch + 8 + 2 * wc - 3);
-                const int c0 = (threadIdx.x >> 7) * (kKChunks / 2);
-                uint4* a_dst = reinterpret_cast<uint4*>(smem_raw + (a_addr - base) + ab * p.a_bytes) + (threadIdx.x & 127);
-                if (C == 3) {
-                    if (threadIdx.x < 128) build_rgb<0>(origin, p.pitch, a_dst);
-                    else build_rgb<1>(origin, p.pitch, a_dst);
-                } else {
-                    // all loads first, then all stores: the stores could alias the loads for all the compiler knows, and
-                    // interleaved they would leave one 16-byte group's loads in flight at a time
-                    uint4 v[kKChunks / 2];
-#pragma unroll
-                    for (int cc = 0; cc < kKChunks / 2; ++cc) {
-                        const int ch = c0 + cc;
-                        const int4 o0 = *reinterpret_cast<const int4*>(&ctrl->koff[ch * 8]);
-                        const int4 o1 = *reinterpret_cast<const int4*>(&ctrl->koff[ch * 8 + 4]);
-                        v[cc].x = (uint32_t)origin[o0.x] | ((uint32_t)origin[o0.y] << 16);
-                        v[cc].y = (uint32_t)origin[o0.z] | ((uint32_t)origin[o0.w] << 16);
-                        v[cc].z = (uint32_t)origin[o1.x] | ((uint32_t)origin[o1.y] << 16);
-                        v[cc].w = (uint32_t)origin[o1.z] | ((uint32_t)origin[o1.w] << 16);
-                    }
-#pragma unroll
-                    for (int cc = 0; cc < kKChunks / 2; ++cc) a_dst[(c0 + cc) * 128] = v[cc];
-                }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> MMA reads
-            if (!w) { atomicExch(&ctrl->abort_flag, 1); ok = false; break; }     // the vote after the last tile takes everybody out together
-            mbar_arrive(base + (uint32_t)offsetof(SpCtrl, a_full) + 8 * ab);
-        }
-        {   // the last two tiles' commits (a unit of one tile has only one)
-            bool w = ok;
-            for (int t = p.tiles >= 2 ? p.tiles - 2 : 0; t < p.tiles && w; ++t) {
-                const int ab = t & 1;
-                w = mbar_wait(mma_done0 + 8 * ab, mma_phase[ab], abort_flag);
-                mma_phase[ab] ^= 1;
-            }
-            if (bar_or(!w)) { ok = false; break; }
-            tc_fence_after();
-        }
+        // the next unit's rows first: its MMAs then run while this unit is pooled
+        if (u + (int)gridDim.x < p.n_units && !rewrite(it + 1)) { ok = false; break; }
 
         // ---- epilogue 1: accumulators -> bias, ReLU, bf16 -> the unit's convolution rows in shared memory ----
         {
             const int quarter = warp & 3, half = warp >> 2;      // TMEM lanes 32 * quarter ..; the 16-column groups alternate between the two halves
+            bool w = true;
             for (int t = 0; t < p.tiles; ++t) {
+                if (w) w = __all_sync(0xffffffffu, mbar_wait(mma_done0 + 8 * t, (uint32_t)(it & 1), abort_flag));
+                if (!w) continue;                                // (warp-uniform) the vote below takes everybody out together
+                tc_fence_after();
                 const int m = t * 128 + quarter * 32 + lane;
-                const int j = (int)fdiv((uint32_t)(m < p.conv_pos ? m : 0), p.div_wc);
+                const int j = (int)fdiv((uint32_t)m, p.div_px), q = m - j * p.pitch_x;
+                const bool pos = j < kConvRows && q < p.Wc;      // the pad columns and the rows behind the fifth are dropped
                 const int hc = 4 * pr - 1 + j;
-                const bool live = m < p.conv_pos && hc >= 0 && hc < p.Hc;
+                const bool live = pos && hc >= 0 && hc < p.Hc;
                 uint32_t v[3][16];                               // this warp's column groups of the tile (K_pad <= 96): one wait for all
                 __syncwarp();
 #pragma unroll
@@ -345,7 +312,8 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
                     if (c0 < K_pad) tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(t * K_pad + c0), v[g]);
                 }
                 tmem_ld_wait();
-                if (m < p.conv_pos) {
+                if (pos) {
+                    const int idx = j * p.Wc + q;
 #pragma unroll
                     for (int g = 0; g < 3; ++g) {
                         const int c0 = 16 * half + 32 * g;
@@ -357,7 +325,7 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
                                 const float f1 = live ? __uint_as_float(v[g][2 * i + 1]) + bias_s[c0 + 2 * i + 1] : 0.0f;
                                 reinterpret_cast<uint32_t*>(o)[i] = pack_bf16x2_relu(f0, f1);
                             }
-                            uint4* dst = reinterpret_cast<uint4*>(conv_ptr) + (size_t)(c0 >> 3) * p.conv_pos + m;
+                            uint4* dst = reinterpret_cast<uint4*>(conv_ptr) + (size_t)(c0 >> 3) * p.conv_pos + idx;
                             dst[0] = o[0];
                             dst[p.conv_pos] = o[1];
                         }
@@ -365,8 +333,9 @@ __global__ void __launch_bounds__(kThreads) stem_pool_kernel(const SpParams p) {
                 }
             }
             tc_fence_before();
+            mbar_arrive(tmem_free);                              // the accumulators may be overwritten by the next unit's MMAs
+            if (bar_or(!w)) { ok = false; break; }               // (also: the convolution rows are complete)
         }
-        bar_sync();
 
         // ---- epilogue 2: 3x3 / 2 maxima of the two pooled rows, border columns included; border rows at the image's ends ----
         {
@@ -455,27 +424,32 @@ int pow2_at_least(int v) { int p = 32; while (p < v) p <<= 1; return p; }
 
 }  // namespace
 
+// shared memory of the kernel for one shape, and its tile count / parity-buffer rows
+static unsigned stem_pool_smem(int C, int W, int K_pad, int* tiles_out, int* x_rows_out) {
+    const int Wc = W / 2, pitch_x = Wc + 3;
+    const int tiles = (kConvRows * pitch_x + 127) / 128;
+    const int x_rows = (tiles * 128 + 3 * pitch_x + 3 + 7) & ~7;
+    if (tiles_out) *tiles_out = tiles;
+    if (x_rows_out) *x_rows_out = x_rows;
+    const unsigned ctrl = (unsigned)((sizeof(SpCtrl) + 127) & ~127u);
+    return ctrl + (unsigned)K_pad * 4u + 1024u + (unsigned)((kTaps * 2 * K_pad * 16 + 127) & ~127) + 2u * (unsigned)(2 * x_rows * 16) +
+           2u * (unsigned)(C * kRowsIn * (W + 16) * 2) + (unsigned)((K_pad / 8) * kConvRows * Wc * 16);
+}
+
 bool stem_pool_supported(int C, int H, int W, int K_pad) {
-    if (C < 1 || C > 3 || H % 4 || W % 8 || H < 8 || W < 8 || K_pad % 16 || K_pad < 16) return false;
-    const int Wc = W / 2, tiles = (kConvRows * Wc + 127) / 128;
-    if (tiles * K_pad > 512) return false;
-    const unsigned smem = 1024u + 512u + (unsigned)K_pad * 4u + 1024u + (unsigned)(kKChunks * K_pad * 16 + 128) +
-                          2u * (unsigned)(kKChunks * 128 * 16) + 2u * (unsigned)(C * kRowsIn * (W + 16) * 2) +
-                          (unsigned)((K_pad / 8) * kConvRows * Wc * 16);
+    if (C < 1 || C > 3 || H % 4 || W % 8 || H < 8 || W < 8 || K_pad % 16 || K_pad < 16 || K_pad > 96) return false;
+    int tiles = 0, x_rows = 0;
+    const unsigned smem = stem_pool_smem(C, W, K_pad, &tiles, &x_rows);
+    if (tiles > kMaxTiles || tiles * K_pad > 512) return false;
     return smem <= kSmemMax;
 }
 
 int plan_stem_pool(const StemPoolArgs& a, StemPoolPlan* plan, char* err, size_t err_len) {
     memset(plan, 0, sizeof(*plan));
     if (!stem_pool_supported(a.C, a.H, a.W, a.K_pad)) { snprintf(err, err_len, "first convolution + pooling: shape not supported"); return 1; }
-    const int Wc = a.W / 2;
-    plan->tiles = (kConvRows * Wc + 127) / 128;
+    int x_rows = 0;
+    plan->smem_bytes = stem_pool_smem(a.C, a.W, a.K_pad, &plan->tiles, &x_rows);
     plan->tmem_cols = pow2_at_least(plan->tiles * a.K_pad);
-    const unsigned ctrl = (unsigned)((sizeof(SpCtrl) + 127) & ~127u);
-    plan->smem_bytes = ctrl + (unsigned)a.K_pad * 4u + 1024u + (unsigned)((kKChunks * a.K_pad * 16 + 127) & ~127) +
-                       2u * (unsigned)(kKChunks * 128 * 16) + 2u * (unsigned)(a.C * kRowsIn * (a.W + 16) * 2) +
-                       (unsigned)((a.K_pad / 8) * kConvRows * Wc * 16);
-    if (plan->smem_bytes > kSmemMax) { snprintf(err, err_len, "first convolution + pooling does not fit shared memory"); return 1; }
     if (cudaFuncSetAttribute(stem_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
         snprintf(err, err_len, "cannot raise the dynamic shared memory limit");
         cudaGetLastError();
@@ -492,16 +466,16 @@ void launch_stem_pool(const StemPoolPlan& plan, const StemPoolArgs& a, int* d_st
     p.Hc = a.H / 2; p.Wc = a.W / 2; p.Hp = p.Hc / 2; p.Wp = p.Wc / 2;
     p.pitch = a.W + 16;
     p.in_bytes = a.C * kRowsIn * p.pitch * 2;
-    p.a_bytes = kKChunks * 128 * 16;
-    p.b_bytes = kKChunks * a.K_pad * 16;
+    p.pitch_x = p.Wc + 3;
+    stem_pool_smem(a.C, a.W, a.K_pad, nullptr, &p.x_rows);
+    p.b_bytes = kTaps * 2 * a.K_pad * 16;
     p.conv_pos = kConvRows * p.Wc;
     p.tiles = plan.tiles;
     p.units_per_image = (p.Hp + 1) / 2;
     p.n_units = a.n_count * p.units_per_image;
     p.tmem_cols = plan.tmem_cols;
-    p.div_wc = make_fastdiv((uint32_t)p.Wc);
+    p.div_px = make_fastdiv((uint32_t)p.pitch_x);
     p.div_upi = make_fastdiv((uint32_t)p.units_per_image);
-    p.div_wp2 = make_fastdiv((uint32_t)(p.Wp + 2));
     p.status = d_status;
     int grid = sm_count();
     if (grid > p.n_units) grid = p.n_units;
