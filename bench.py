@@ -333,6 +333,41 @@ def kernel_report(B, m, peaks, peak_kind, reps):
     return roof, side_out, ops, op_ms
 
 
+def timed_queue(torch, stream, flush, step, steps, warmup, sync_ranks=True):
+    """End to end: `steps` asynchronous calls queued back to back on `stream`, an L2 flush before each, between two events.
+    The calls overlap one another where the library lets them (the next step's input crosses the bus while this step's
+    network runs), so the time is that of the whole queue - flushes included - not a sum of per-step brackets.
+    Returns the milliseconds of the whole queue."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            if flush is not None:
+                flush.fill_(1)
+            step()
+        torch.cuda.synchronize()
+        if sync_ranks:
+            barrier()
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(steps):
+            if flush is not None:
+                flush.fill_(1)
+            step()
+        b.record(stream)
+        torch.cuda.synchronize()
+        if sync_ranks:
+            barrier()
+        # the flushes alone, for context (the reported time keeps them in)
+        fa, fb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fa.record(stream)
+        for _ in range(steps):
+            if flush is not None:
+                flush.fill_(1)
+        fb.record(stream)
+        torch.cuda.synchronize()
+    return a.elapsed_time(b), fa.elapsed_time(fb)
+
+
 def measure(torch, B, wl, dev, stream, flush, peaks, peak_kind, config, batch, prune, steps, warmup, args,
             headline=False, sampler=None):
     """One workload: device-resident throughput, end to end from pinned host buffers, kernel classes."""
@@ -340,11 +375,12 @@ def measure(torch, B, wl, dev, stream, flush, peaks, peak_kind, config, batch, p
     m = Model(torch, B, w, dev, no_prune=args.no_prune if headline else False)
     try:
         step_dev = lambda: B.fp_forward(m.h, m.dx, w.batch, m.logits, stream)
-        step_host = lambda: B.fp_forward_host(m.h, m.x_pinned, w.batch, m.logits_pinned, stream)
+        step_host = lambda: B.fp_forward_host_async(m.h, m.x_pinned, w.batch, m.logits_pinned, stream)
         per_step, t0, t1 = timed_steps(torch, stream, flush, step_dev, steps, warmup, sync_ranks=headline)
         assert B.fp_query_int(m.h, B.FP_Q_DEVICE_STATUS) == 0, "a device-side wait timed out"
-        per_step_e2e, _, _ = timed_steps(torch, stream, flush, step_host, steps, warmup, sync_ranks=headline)
-        ms, ms_e2e = sum(per_step), sum(per_step_e2e)
+        ms_e2e, ms_flushes = timed_queue(torch, stream, flush, step_host, steps, warmup, sync_ranks=headline)
+        assert B.fp_query_int(m.h, B.FP_Q_DEVICE_STATUS) == 0, "a device-side wait timed out"
+        ms = sum(per_step)
         roof, side, ops, op_ms = kernel_report(B, m, peaks, peak_kind, 20 if headline else 10)
         flops_img = B.fp_query_array(m.h, B.FP_Q_FLOPS, 0, np.float64, 1)[0]
         bytes2 = B.fp_query_array(m.h, B.FP_Q_BYTES, 0, np.float64, 2)
@@ -359,6 +395,7 @@ def measure(torch, B, wl, dev, stream, flush, peaks, peak_kind, config, batch, p
             "ms_per_step_median": statistics.median(per_step), "ms_per_step_p99": percentile(per_step, 0.99),
             "steps": steps, "launches_per_step": int(n_launch),
             "e2e_images_per_s": w.batch * steps / (ms_e2e * 1e-3), "e2e_ms_per_step": ms_e2e / steps,
+            "e2e_ms_per_step_without_flushes": (ms_e2e - ms_flushes) / steps,
             "h2d_bytes_per_step": int(m.x_pinned.numel() * m.x_pinned.element_size()),
             "d2h_bytes_per_step": int(m.logits_pinned.numel() * 4),
             "roofline": roof,
@@ -371,7 +408,7 @@ def measure(torch, B, wl, dev, stream, flush, peaks, peak_kind, config, batch, p
                            "sum_op_ms": float(sum(op_ms))},
             "side_kernels": side,
         }
-        extra = {"ms": ms, "ms_e2e": ms_e2e, "t0": t0, "t1": t1, "ops": ops, "op_ms": op_ms, "n_launch": n_launch}
+        extra = {"ms": ms, "ms_e2e": ms_e2e, "ms_flushes": ms_flushes, "t0": t0, "t1": t1, "ops": ops, "op_ms": op_ms, "n_launch": n_launch}
         if headline:
             # the same forward back to back for about a second, no flush in between: the clock and power state of a
             # loaded GPU (the measured peaks were taken in that state); inputs + activations exceed L2 on this workload
@@ -462,7 +499,10 @@ def run_gpu(args):
                        "l2": "flushed between timed steps (256 MiB write)", "parallelism": f"replicas x{world}"},
             "ms_per_step_median": r["ms_per_step_median"], "ms_per_step_p99": r["ms_per_step_p99"],
             "e2e": {"value": tot_units / (tot_ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": r["h2d_bytes_per_step"],
-                    "d2h_bytes_per_step": r["d2h_bytes_per_step"], "ms_per_step": tot_ms_e2e / args.steps},
+                    "d2h_bytes_per_step": r["d2h_bytes_per_step"], "ms_per_step": tot_ms_e2e / args.steps,
+                    "ms_per_step_without_flushes": r["e2e_ms_per_step_without_flushes"],
+                    "call": "fp_forward_host_async, the steps queued back to back on one stream (pinned host input and "
+                            "logits every step); timed as one queue between two events, L2 flushes included"},
             "gpu_launches": int(x["n_launch"] * args.steps),
             "clocks": clocks,
             "roofline": r["roofline"],

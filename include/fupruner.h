@@ -173,6 +173,18 @@ fp_status fp_forward(fp_handle h, const void* d_input, int32_t batch, float* d_l
  * runs the network, copies the logits back and waits.  (The end-to-end call.) */
 fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t batch, float* h_logits, void* stream);
 
+/* fp_forward_host_async - fp_forward_host without the wait: the input copy, the network and the copy of the logits are
+ * queued and the call returns.  Where the graph starts with a kernel of its own that takes the input in (the ImageNet
+ * networks), the input crosses the bus on a second stream - in pieces of at least 8 MB, each handed to that kernel as it
+ * arrives - and waits only for the PREVIOUS call's first kernel, the one reader of the staging buffer: a caller who
+ * queues the next call before this one has finished has the next input copied while this forward still runs.
+ *   h_input     host (pinned for the copy to be asynchronous), same layout and type as fp_forward's d_input; must stay
+ *               unchanged until the work queued by this call has finished.
+ *   h_logits    host, batch x n_classes floats; valid once `stream` has been synchronised (or an event recorded on it
+ *               after the call has completed).  Calls on one handle are ordered on `stream`.
+ * Errors: as fp_forward.  Asynchronous on `stream` (and an internal copy stream). */
+fp_status fp_forward_host_async(fp_handle h, const void* h_input, int32_t batch, float* h_logits, void* stream);
+
 /*
  * fp_score - filter scores of one convolution of the fused, unpruned graph (Eq. 6 / l1),
  * computed on the device in fp64 with a fixed summation order: filter flattened in (c,r,s)

@@ -24,7 +24,7 @@ FP_NORM_L1, FP_NORM_L2 = 0, 1
  FP_Q_FLOPS, FP_Q_BYTES, FP_Q_N_OPS, FP_Q_OP_INFO, FP_Q_OP_OUTPUT, FP_Q_DEVICE_STATUS, FP_Q_N_LAUNCHES,
  FP_Q_OP_TIMES, FP_Q_CONV_BANK_ELEMS) = range(16)
 
-EXPORTS = ["fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_score", "fp_query", "fp_destroy",
+EXPORTS = ["fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_forward_host_async", "fp_score", "fp_query", "fp_destroy",
            "fp_last_error", "fp_rank_filters_static", "fp_soft_prune_epoch", "fp_soft_prune_finish",
            "fp_debug_expire_wait", "fp_fuse_with_allocator"]
 FP_STATIC_RANK_MAX_FILTERS = 4096
@@ -107,6 +107,7 @@ def lib():
         L.fp_prune.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         L.fp_forward.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         L.fp_forward_host.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+        L.fp_forward_host_async.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         L.fp_score.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
         L.fp_query.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t]
         L.fp_destroy.argtypes = [ctypes.c_void_p]
@@ -182,6 +183,13 @@ def fp_forward_host(h, h_input, batch, h_logits, stream=None):
     pin = h_input.ctypes.data if isinstance(h_input, np.ndarray) else h_input.data_ptr()
     pout = h_logits.ctypes.data if isinstance(h_logits, np.ndarray) else h_logits.data_ptr()
     _check(lib().fp_forward_host(h, pin, batch, pout, stream.cuda_stream if stream is not None else None))
+
+
+def fp_forward_host_async(h, h_input, batch, h_logits, stream=None):
+    """fp_forward_host without the wait: h_logits is valid once `stream` has been synchronised."""
+    pin = h_input.ctypes.data if isinstance(h_input, np.ndarray) else h_input.data_ptr()
+    pout = h_logits.ctypes.data if isinstance(h_logits, np.ndarray) else h_logits.data_ptr()
+    _check(lib().fp_forward_host_async(h, pin, batch, pout, stream.cuda_stream if stream is not None else None))
 
 
 def fp_score(h, conv_index, norm=FP_NORM_L1):

@@ -148,6 +148,7 @@ struct fp_handle_s {
     void* alloc_user = nullptr;
     int* d_status = nullptr;
     cudaStream_t copy_stream = nullptr;    // fp_forward_host: input pieces are copied here while earlier pieces are converted
+    int stage_used = 0;                    // the staging buffer has been read by a kernel queued behind copy_events[kHostPieces]
     cudaEvent_t copy_events[kHostPieces + 1] = {};
     double* d_scores = nullptr; int32_t* d_rank = nullptr; uint8_t* d_mask = nullptr;
     std::map<GraphKey, cudaGraphExec_t> graphs;
@@ -1458,6 +1459,12 @@ extern "C" fp_status fp_debug_expire_wait(fp_handle h, void* stream) {
 }
 
 extern "C" fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t batch, float* h_logits, void* stream) {
+    TRY(fp_forward_host_async(h, h_input, batch, h_logits, stream));
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    return FP_OK;
+}
+
+extern "C" fp_status fp_forward_host_async(fp_handle h, const void* h_input, int32_t batch, float* h_logits, void* stream) {
     if (!h || !h_input || !h_logits) return fail(FP_ERR_ARG, "fp_forward_host: NULL argument");
     if (batch <= 0) return fail(FP_ERR_ARG, "fp_forward_host: batch must be positive");
     if (batch > h->max_batch) return fail(FP_ERR_BOUNDS, "fp_forward_host: batch %d exceeds max_batch %d", batch, h->max_batch);
@@ -1472,17 +1479,18 @@ extern "C" fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t b
     // (pieces of at least 8 MB: a copy has a fixed cost of some tens of microseconds, measured 1.14 ms end to end with
     // eight 2.4 MB pieces against 0.95 ms with one copy on ResNet-18 at batch 64)
     const size_t total_bytes = (size_t)batch * image_bytes;
-    const int pieces = (h->ops[0].kind == 3 && !h->input_fused && batch >= 2)
-                           ? std::max(1, std::min(std::min(kHostPieces, batch), (int)(total_bytes >> 23))) : 1;
+    const bool own_input_op = h->ops[0].kind == 3 && !h->input_fused;
+    const int pieces = (own_input_op && batch >= 2) ? std::max(1, std::min(std::min(kHostPieces, batch), (int)(total_bytes >> 23))) : 1;
     const int piece_op = h->stem_fused ? 1 : 0, tail_op = h->stem_fused ? 3 : 1;     // the kernel that takes the input in; what follows it
-    if (pieces > 1) {
+    if (own_input_op) {
         if (!h->copy_stream) {
             CK(cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
             for (int i = 0; i <= kHostPieces; ++i) CK(cudaEventCreateWithFlags(&h->copy_events[i], cudaEventDisableTiming));
         }
-        // the copies must not overtake work already queued on `st` that still reads the staging buffer
-        CK(cudaEventRecord(h->copy_events[kHostPieces], st));
-        CK(cudaStreamWaitEvent(h->copy_stream, h->copy_events[kHostPieces], 0));
+        // Only that first kernel reads the staging buffer: the copies wait for the previous call's first kernel(s) - the
+        // event recorded behind them below - and not for the rest of its forward, so that a caller who queues call after
+        // call (fp_forward_host_async) has the next input cross the bus while the network still runs on this one.
+        if (h->stage_used) CK(cudaStreamWaitEvent(h->copy_stream, h->copy_events[kHostPieces], 0));
         for (int c = 0; c < pieces; ++c) {
             const int n0 = (int)((long long)batch * c / pieces), n1 = (int)((long long)batch * (c + 1) / pieces);
             CK(cudaMemcpyAsync((uint8_t*)h->d_in_stage + (size_t)n0 * image_bytes, (const uint8_t*)h_input + (size_t)n0 * image_bytes,
@@ -1492,13 +1500,14 @@ extern "C" fp_status fp_forward_host(fp_handle h, const void* h_input, int32_t b
             launch_op(h, piece_op, h->d_in_stage, batch, h->d_logits_stage, st, n0, n1 - n0);
         }
         CK(cudaGetLastError());
+        CK(cudaEventRecord(h->copy_events[kHostPieces], st));         // the staging buffer is free again
+        h->stage_used = 1;
         TRY(forward_from(h, h->d_in_stage, batch, h->d_logits_stage, st, tail_op));
     } else {
         CK(cudaMemcpyAsync(h->d_in_stage, h_input, (size_t)batch * image_bytes, cudaMemcpyHostToDevice, st));
         TRY(forward_from(h, h->d_in_stage, batch, h->d_logits_stage, st, 0));
     }
     CK(cudaMemcpyAsync(h_logits, h->d_logits_stage, (size_t)batch * h->n_classes * sizeof(float), cudaMemcpyDeviceToHost, st));
-    CK(cudaStreamSynchronize(st));
     return FP_OK;
 }
 

@@ -21,7 +21,7 @@ def test_library_exports_every_declared_symbol():
     path = build.build()
     lib = ctypes.CDLL(path)
     names = declared_functions()
-    assert {"fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_score", "fp_query", "fp_destroy",
+    assert {"fp_fuse", "fp_prune", "fp_forward", "fp_forward_host", "fp_forward_host_async", "fp_score", "fp_query", "fp_destroy",
             "fp_last_error"} <= names
     for n in names:
         assert hasattr(lib, n), f"{n} is declared in include/ but not exported"

@@ -650,6 +650,37 @@ def test_first_convolution_and_pooling_in_one_kernel(B, fpo, shape, p):
         g.close()
 
 
+def test_queued_host_calls_overlap_copies_without_mixing_inputs(B, fpo):
+    """fp_forward_host_async: three calls with three different pinned inputs queued back to back on one stream (the
+    second and third inputs are copied while the forward before them still runs - they wait only for its first
+    kernel); every call's logits equal those of the blocking call on the same input."""
+    H, W, K, C, batch = 64, 64, 32, 3, 6
+    w = wl.Workload("stem_pool", _stem_net(H, W, K, C), batch, 37, True, wl.uniform_ratios(0.3), "uniform 0.3")
+    g = Gpu(B, w, B.FP_COMPUTE_BF16_TC, max_batch=batch)
+    try:
+        B.fp_prune(g.h, w.ratios)
+        rng = np.random.default_rng(5)
+        xs = [torch.from_numpy((w.x * s + rng.standard_normal(w.x.shape).astype(np.float32) * 0.1)).to(torch.bfloat16).pin_memory()
+              for s in (1.0, -0.5, 0.25)]
+        want = []
+        for x in xs:
+            out = np.empty((batch, g.n_classes), dtype=np.float32)
+            B.fp_forward_host(g.h, x, batch, out)
+            want.append(out)
+        assert not np.array_equal(want[0], want[1])
+        outs = [torch.empty((batch, g.n_classes), dtype=torch.float32).pin_memory() for _ in xs]
+        stream = torch.cuda.Stream()
+        for rep in range(3):
+            for x, o in zip(xs, outs):
+                B.fp_forward_host_async(g.h, x, batch, o, stream)
+            stream.synchronize()
+            for o, ref in zip(outs, want):
+                np.testing.assert_array_equal(o.numpy(), ref)
+        assert B.fp_query_int(g.h, B.FP_Q_DEVICE_STATUS) == 0
+    finally:
+        g.close()
+
+
 def test_maxpool_windows_of_negative_values(B, fpo):
     """Max pooling right after a batch norm without ReLU, every other channel shifted far below zero, so a padded
     position that took part in a window as 0 (instead of being ignored) would win it.  Odd height, a width that
