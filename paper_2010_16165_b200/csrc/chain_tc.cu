@@ -150,6 +150,11 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // the layer table in shared memory: an index into the kernel's parameters that is not a compile-time constant costs
+    // some 300 cycles per use, and every layer of the run starts with one
+    __shared__ ChainLayer s_layers[kChainMaxLayers];
+    for (int i = threadIdx.x; i < p.a.n_layers * (int)(sizeof(ChainLayer) / 4); i += blockDim.x)
+        reinterpret_cast<int*>(s_layers)[i] = reinterpret_cast<const int*>(p.a.layers)[i];
     // The W guard rows before and after each chunk plane are only read for rows whose results are discarded,
     // but they must hold finite values (the epilogue masks neighbour terms by multiplying with 0): zero them once.
     {
@@ -192,11 +197,11 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 if (lane == 0) w = mbar_wait(w_empty0 + 8 * wb, wph ^ 1, abort_flag);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) { ok = false; break; }
-                const int bytes = p.a.layers[l].blob_bytes;
+                const int bytes = s_layers[l].blob_bytes;
                 const uint32_t fb = w_full0 + 8 * wb;
                 if (lane == 0) mbar_expect_tx(fb, (uint32_t)bytes);
                 __syncwarp();
-                const uint8_t* src = reinterpret_cast<const uint8_t*>(p.a.w) + p.a.layers[l].blob_off;
+                const uint8_t* src = reinterpret_cast<const uint8_t*>(p.a.w) + s_layers[l].blob_off;
                 for (int off = lane * 4096; off < bytes; off += 32 * 4096) {
                     const int n = bytes - off < 4096 ? bytes - off : 4096;
                     bulk_copy(wbuf0 + wb * p.wbuf_bytes + off, src + off, (uint32_t)n, fb);
@@ -213,13 +218,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         // order, which the parity waits on the stage's barriers rely on.
         const int iss = warp == 1 ? 0 : warp - (1 + kEpiThreads / 32);
         // The whole warp runs the loop in step (one lane issues): operand descriptors are then warp-uniform values.
+        // (Every lane tests the barriers: one lane testing and a shuffle of the result measured 10-20 % slower per step.)
         if (iss < p.issuers) {
             const bool leader = lane == 0;
             bool ok = true;
             uint32_t it = 0, ring_pos = 0, ring_phase = 0;     // position in this issuer's ring of accumulator stages
             for (int g = blockIdx.x; g < p.n_groups && ok; g += gridDim.x) {
                 for (int l = 0; l < L && ok; ++l, ++it) {
-                    const ChainLayer& ly = p.a.layers[l];
+                    const ChainLayer& ly = s_layers[l];
                     const uint32_t wb = it & 1, wph = (it >> 1) & 1;
                     // Tile t's input is complete when its barrier has completed `it` + 1 times (once per group load
                     // and per layer).  Completions alternate between two barriers per tile, so that a parity test
@@ -392,7 +398,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             }
             // ---- layers ----
             for (int l = 0; l < L && ok; ++l, ++it) {
-                const ChainLayer& ly = p.a.layers[l];
+                const ChainLayer& ly = s_layers[l];
                 const uint32_t wb = it & 1, wph = (it >> 1) & 1;
                 const bool last = l == L - 1;
                 if (!mbar_wait(w_full0 + 8 * wb, wph, abort_flag)) { ok = false; break; }     // the bias is in the blob
@@ -487,7 +493,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             if (!ok) break;
             // ---- zero border of the group's output images in global memory ----
             {
-                const int out_chunks = p.a.layers[L - 1].K_pad >> 3;
+                const int out_chunks = s_layers[L - 1].K_pad >> 3;
                 const int border = 2 * p.Wp + 2 * H;
                 const int total = p.G * border * out_chunks;
                 for (int i = etid; i < total; i += kEpiThreads) {
