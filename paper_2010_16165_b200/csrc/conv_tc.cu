@@ -16,14 +16,21 @@
 //                 shared-memory block read from a start address shifted by (r-1)*(W+2)+(s-1) rows,
 //                 so each activation is fetched once per tile, not once per tap.  The zero border
 //                 in memory is the convolution's padding.  Filters either stay resident in shared
-//                 memory for the whole kernel (small banks) or are streamed per (tap, K block).
-//   GATHER mode   any other geometry (stride 2, 7x7, ...): 128 loader threads fetch the vectors of
+//                 memory for the whole kernel (small banks), are streamed per (filter row, K block) into a ring of
+//                 their own, or share a stage with the activations of their K block (1x1 layers, and the strided
+//                 3x3 layers below: one ring, several producer warps).
+//   Parity-split  a 3x3 / stride-2 / pad-1 convolution over a tensor stored as four half-resolution parity images
+//   inputs        (ConvArgs in fp_internal.h) is a FLAT convolution too: four contiguous runs per chunk, tap (r,s)
+//                 reading the run of parity ((r+1)&1, (s+1)&1) at an offset of -1 or 0 rows and columns; a 1x1 /
+//                 stride-2 convolution reads the parity-00 images alone.  The epilogue can write a tensor in that form.
+//   GATHER mode   any other geometry (strided layers over plain tensors, 7x7, ...): 128 loader threads fetch the vectors of
 //                 their output position for each (tap, K block) with 16-byte loads, zero where the
 //                 window leaves the image.
 //   Warp roles    warp 0: bulk-copy producer (one lane per chunk copy).  warp 1: tensor-memory allocation, lane 0 issues
-//                 the MMAs.  warps 2-5: epilogue, one thread per accumulator row.  warp 6 lane 0:
-//                 filter producer when filters are streamed in a FLAT mode.  warps 6-9: loader
-//                 threads in GATHER mode.
+//                 the MMAs.  Then 4 or 8 epilogue warps, one thread per accumulator row (8: each takes half of the
+//                 columns).  Behind them: the filter producer and up to three more MMA-issuing warps (one per position
+//                 tile of a step) when filters are streamed; three more producer and three more issuing warps with
+//                 unified stages; the four loader warps in GATHER mode.
 //   Pipelines     full/empty mbarrier rings for the shared-memory stages; two accumulator stages in
 //                 tensor memory so the epilogue of one tile overlaps the MMAs of the next.
 //   Waits         every mbarrier wait is bounded; when one runs out the CTA raises a status word in
