@@ -924,6 +924,11 @@ void choose_filter_tile(const ConvArgs& a, int K_pad, int* n_tile_out, int* n_ti
             n_tiles *= 2;
             n_tile = round_up_i((K_pad + n_tiles - 1) / n_tiles, 16);
         }
+        // A 1x1 layer with a long reduction and 129-192 filters is bound by the MMA count: one tile of all filters (one
+        // position tile per step: tensor memory) instead of two of half the width, an MMA costing the pipe about the
+        // same for 80 filters as for 160 (measured, ResNet-50 batch 128: 1024 -> 160 at 14x14 30.6 -> 28.5 us,
+        // 512 -> 160 at 28x28 45.1 -> 42.1 us; with 320 filters two tiles of 160 lose against three of 112).
+        if (taps == 1 && flat && K_pad > 128 && K_pad <= 192 && m_tiles >= sms) { n_tiles = 1; n_tile = K_pad; }
     }
     *n_tile_out = n_tile;
     *n_tiles_out = (K_pad + n_tile - 1) / n_tile;
