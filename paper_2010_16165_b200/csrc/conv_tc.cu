@@ -263,7 +263,8 @@ conv_tc_kernel(const TcParams p) {
         mbar_expect_tx(b_full0, (uint32_t)p.b_bank_bytes);
         for (int off = 0; off < p.b_bank_bytes; off += 32768) {
             const int n = p.b_bank_bytes - off < 32768 ? p.b_bank_bytes - off : 32768;
-            bulk_copy(b_base + off, reinterpret_cast<const uint8_t*>(p.a.w) + off, (uint32_t)n, b_full0);
+            bulk_copy(b_base + off, reinterpret_cast<const uint8_t*>(p.a.w) + (long long)(blockIdx.x % p.n_tiles) * p.b_bank_bytes + off,
+                      (uint32_t)n, b_full0);
         }
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -442,10 +443,10 @@ conv_tc_kernel(const TcParams p) {
                         uint32_t a_row = ((a_base + a_stage * p.a_stage_bytes) >> 4) | ((uint32_t)(p.a_par * p.rows_a) << 16);
                         uint32_t b_tap = 0;
                         if (MODE == MODE_FLAT_RESIDENT)
-                            b_tap = ((b_base >> 4) + (uint32_t)(g * p.cg * p.a.K_pad + nt * p.n_tile)) | ((uint32_t)p.a.K_pad << 16);
+                            b_tap = ((b_base >> 4) + (uint32_t)(g * p.cg * p.n_tile)) | ((uint32_t)p.n_tile << 16);   // this CTA's filter tile only
                         const uint32_t a_ks = 2u * (uint32_t)(p.a_par * p.rows_a);
-                        const uint32_t b_ks = 2u * (uint32_t)(MODE == MODE_FLAT_RESIDENT ? p.a.K_pad : p.n_tile);
-                        const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.a.K_pad);
+                        const uint32_t b_ks = 2u * (uint32_t)p.n_tile;
+                        const uint32_t b_tap_step = (uint32_t)(p.cchunks * p.n_tile);
                         if (MODE == MODE_FLAT_RESIDENT && p.a.x_s2d) {
                             // nine taps over the four parity images: each tap's operand starts at its own row of the stage
                             // (unrolled: an index into the parameters that is not a constant costs some 300 cycles per use)
@@ -958,8 +959,18 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
     int n_tile, n_tiles;
     if (a.n_tile_forced > 0) { n_tile = a.n_tile_forced; n_tiles = (a.K_pad + n_tile - 1) / n_tile; }
     else choose_filter_tile(a, a.K_pad, &n_tile, &n_tiles);
-    const long long bank = (long long)taps * a.C_pad * a.K_pad * 2;
-    bool bank_fits = plan->flat && bank <= 100 * 1024;
+    // Resident filters: a CTA keeps ITS filter tile's part of the bank (the grid is a multiple of the number of filter
+    // tiles, so a CTA's tiles all have the same one), all taps and channels of it, in shared memory for the whole
+    // kernel.  (With the whole bank as the unit, the layers that write ResNet-50's residual stream at 14x14 and 7x7 -
+    // 160 -> 1024 and 320 -> 2048 filters, 327 KB and 1.3 MB - streamed their filters with one CTA on an SM; their
+    // time goes to the epilogue, which a second CTA's warps double.)
+    // Measured at batch 128 (single layers, cold L2): 80 -> 512 at 28x28 59.4 -> 51.6 us (20 KB instead of the whole 82 KB:
+    // more activation stages), 160 -> 1024 at 14x14 45.3 -> 39.6 us; but 320 -> 2048 at 7x7 38.9 -> 47.6 us and the
+    // 256 -> 512 projection 55.1 -> 59.1 us, whose 64-80 KB tile parts leave two stages of four channel chunks: a layer
+    // whose whole bank does not fit takes the resident form only with a part of at most 48 KB.
+    const long long bank = (long long)taps * a.C_pad * n_tile * 2;
+    const long long whole_bank = (long long)taps * a.C_pad * a.K_pad * 2;
+    bool bank_fits = plan->flat && bank <= 100 * 1024 && (whole_bank <= 100 * 1024 || bank <= 48 * 1024);
     plan->n_tile = n_tile; plan->n_tiles = n_tiles;
 
     unsigned smem = (unsigned)sizeof(Ctrl) + (unsigned)a.K_pad * 4u + 1024u;
@@ -1049,6 +1060,7 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
         if (bank_fits) {
             plan->b_resident = 1;
             plan->b_stages = 1;
+            if (n_tiles > 1) plan->blocked_bank = 2;        // [filter tile][(tap, chunk) plane][row]: a tile's part is one run
             const unsigned fixed = smem + (unsigned)round_up_i((int)bank, 128);
             auto fit = [&](int cg, int* stages) {
                 const unsigned st = (unsigned)(a_par * cg * plan->rows_a * 16);
@@ -1188,7 +1200,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.bank_tile_bytes = (long long)p.taps * p.cchunks * plan.n_tile * 16;
     p.tpk = plan.tpk > 0 ? plan.tpk : 1;
     p.kblocks = plan.groups > 1 ? p.taps * plan.groups : (p.taps + p.tpk - 1) / p.tpk;
-    p.b_bank_bytes = p.taps * a.C_pad * a.K_pad * 2;
+    p.b_bank_bytes = p.taps * a.C_pad * plan.n_tile * 2;        // resident filters: one filter tile's part
     p.lut_bytes = plan.flat ? 0 : p.kblocks * 64;
     p.scatter_bytes = a.scatter ? round_up_i((a.out_C_pad + plan.n_tiles + 1) * 4, 16) + 8 * 32 * 33 * 4 : 0;
     p.status = d_status;
@@ -1198,6 +1210,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.div_qp = make_fastdiv((uint32_t)p.Qp);
     int grid = sm_count() * plan.ctas_per_sm;
     if (grid > p.total_tiles) grid = p.total_tiles;
+    if (plan.b_resident && plan.n_tiles > 1 && grid > plan.n_tiles) grid -= grid % plan.n_tiles;   // a CTA's tiles share a filter tile
     if (grid < 1) grid = 1;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
