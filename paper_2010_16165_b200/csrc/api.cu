@@ -81,6 +81,9 @@ struct FConv {
     int32_t* d_out_map = nullptr;   // scatter: output channel -> packed filter row (-1 = no filter kept)
     int32_t* d_chunk0 = nullptr;    // scatter: first output chunk of every filter tile, and the end
     int n_mult = 1;            // 4: a 1x1 layer over a parity-split tensor runs on its 4 N half-size images
+    int proj = -1;             // >= 0: the projection shortcut (index into convs) whose filters are stacked behind this layer's
+    int absorbed = 0;          // 1: this projection runs inside the layer that adds its result; its operator launches nothing
+    void* d_wp_plain = nullptr;     // the packed bank before any re-blocking ([tap][chunk][K_pad][8])
     int K_kept = 0, K_rows = 0, K_pad = 0, C_kept = 0, C_pad = 0;
     void* d_wp = nullptr;      // packed filters in the compute type, K_pad x R x S x C_pad
     float* d_bp = nullptr;
@@ -835,7 +838,10 @@ fp_status replan(fp_handle h) {
             f.stride == 2 && f.pad == 3 && f.C <= 3 && h->in_H % 2 == 0 && h->in_W % 2 == 0)
             h->stem_packed = 1;
     decide_splits(h, uses);
-    for (FConv& f : h->convs) f.n_mult = (h->tensors[f.src].split && split_reader(f) == 'C') ? 4 : 1;
+    for (FConv& f : h->convs) {
+        f.n_mult = (h->tensors[f.src].split && split_reader(f) == 'C') ? 4 : 1;
+        f.proj = -1; f.absorbed = 0;
+    }
     // ... and, where a 3x3 / stride-2 max pooling is the only reader of that convolution and the input is bf16, input
     // conversion, convolution and pooling run as one kernel (decided below, once the filter count is known).
     h->stem_fused = 0;
@@ -957,11 +963,32 @@ fp_status replan(fp_handle h) {
             }
             // launch plan of the tensor-core kernel (geometry only; the pointers follow once memory is planned)
             f.tc.valid = 0;
+            // A 1x1 layer that adds a projection shortcut (a 1x1 convolution, stride 1 or 2, no ReLU, read by nobody else)
+            // takes the projection in: its filters are stacked behind this layer's along the channels and its input
+            // tensor becomes a second input of this layer (Sec. IV-B's [W2' || S_w] for this one kind of block) - the
+            // projection's output is neither written nor read back.  A stride-2 projection must read a parity-split
+            // tensor (its pixels are then the parity-00 images, on this layer's position grid).  Not with keep_outputs
+            // (every operator's output is wanted then) and not where either layer scatters its output.
+            int pj = -1;
+            if (h->compute == FP_COMPUTE_BF16_TC && !h->keep_outputs && f.res_mode == 1 && f.R == 1 && f.S == 1 && f.stride == 1 &&
+                f.pad == 0 && !f.scatter && !src.split && !out.split && uses[f.res_tid].size() == 1) {
+                const Tensor& rt = h->tensors[f.res_tid];
+                if (rt.producer >= 0 && h->ops[rt.producer].kind == 0) {
+                    const int cand = h->ops[rt.producer].idx;
+                    const FConv& q = h->convs[cand];
+                    const Tensor& X = h->tensors[q.src];
+                    if (q.R == 1 && q.S == 1 && q.pad == 0 && q.res_mode == 0 && !q.relu && !q.scatter && !q.compact && q.K == f.K &&
+                        q.K_pad == f.K_pad && q.n_mult == 1 && q.tc.valid && q.d_wp_plain && !(h->stem_packed && q.src == 0) &&
+                        ((q.stride == 1 && !X.split) || (q.stride == 2 && X.split)))
+                        pj = cand;
+                }
+            }
+            const int C_pad_total = f.C_pad + (pj >= 0 ? h->convs[pj].C_pad : 0);
             if (h->compute == FP_COMPUTE_BF16_TC) {
                 fp::ConvArgs ga;
                 memset(&ga, 0, sizeof(ga));
                 conv_geometry(h, f, &ga);
-                ga.C_pad = (h->stem_packed && f.src == 0) ? 80 : f.C_pad;
+                ga.C_pad = (h->stem_packed && f.src == 0) ? 80 : C_pad_total;
                 ga.K_pad = f.K_pad;
                 ga.scatter = f.scatter; ga.out_C_pad = out.C_pad; ga.n_tile_forced = f.n_tile_forced;
                 char msg[256];
@@ -981,9 +1008,23 @@ fp_status replan(fp_handle h) {
             else fp::launch_repack_conv(f.d_w32, f.C, f.R * f.S, d_row, f.K_pad, d_chan, f.C_pad,
                                    bf16 ? (__nv_bfloat16*)f.d_wp : nullptr, bf16 ? nullptr : (float*)f.d_wp, st);
             fp::launch_pack_bias(f.d_b32, d_row, f.K_pad, f.d_bp, st);
+            f.d_wp_plain = f.d_wp;
+            if (pj >= 0) {
+                // [chunk][K_pad][8]: this layer's chunks, then the projection's; the biases add up
+                FConv& q = h->convs[pj];
+                const size_t b1 = (size_t)f.C_pad * f.K_pad * h->act_elem(), b2 = (size_t)q.C_pad * f.K_pad * h->act_elem();
+                void* cat; float* bsum;
+                TRY(dev_alloc(h, h->pack_buffers, &cat, b1 + b2));
+                TRY(dev_alloc(h, h->pack_buffers, (void**)&bsum, (size_t)f.K_pad * sizeof(float)));
+                CK(cudaMemcpyAsync(cat, f.d_wp, b1, cudaMemcpyDeviceToDevice, st));
+                CK(cudaMemcpyAsync((uint8_t*)cat + b1, q.d_wp_plain, b2, cudaMemcpyDeviceToDevice, st));
+                fp::launch_add_bias(f.d_bp, q.d_bp, f.K_pad, bsum, st);
+                f.d_wp = cat; f.d_bp = bsum;
+                f.proj = pj; q.absorbed = 1;
+            }
             if (f.tc.valid && f.tc.blocked_bank) {
                 // the streamed form of the kernel reads its bank block by block: one copy per pipeline stage
-                const int taps = packed_stem ? 3 : f.R * f.S, cchunks = (packed_stem ? 80 : f.C_pad) / 8;
+                const int taps = packed_stem ? 3 : f.R * f.S, cchunks = (packed_stem ? 80 : C_pad_total) / 8;
                 void* blocked;
                 TRY(dev_alloc(h, h->pack_buffers, &blocked, (size_t)f.tc.n_tiles * taps * cchunks * f.tc.n_tile * 16));
                 if (f.tc.blocked_bank == 1)          // 1x1 layer, unified stages: [tile][K group][tap][chunk][row]
@@ -1021,6 +1062,11 @@ fp_status replan(fp_handle h) {
         std::vector<int> last_use(nt, -1);
         for (int t = 0; t < nt; ++t)
             for (const Use& u : uses[t]) last_use[t] = std::max(last_use[t], u.op);
+        for (int i = 0; i < (int)h->ops.size(); ++i)           // a layer that took a projection in also reads the projection's input
+            if (h->ops[i].kind == 0 && h->convs[h->ops[i].idx].proj >= 0) {
+                const int x = h->convs[h->convs[h->ops[i].idx].proj].src;
+                last_use[x] = std::max(last_use[x], i);
+            }
         struct Buf { void* p; size_t bytes; int free_after; };
         std::vector<Buf> bufs;
         for (int i = 0; i < (int)h->ops.size(); ++i) {
@@ -1038,6 +1084,10 @@ fp_status replan(fp_handle h) {
             else if (op.kind == 1) tid = h->pools[op.idx].out;
             else if (op.kind == 3) tid = 0;
             if (h->stem_fused && (i == 0 || i == 1)) {          // neither the converted input nor the first convolution's output exists
+                h->tensors[tid].d = nullptr;
+                continue;
+            }
+            if (op.kind == 0 && h->convs[op.idx].absorbed) {    // a projection computed inside the layer that adds it
                 h->tensors[tid].d = nullptr;
                 continue;
             }
@@ -1079,7 +1129,13 @@ fp_status replan(fp_handle h) {
         a.scatter = f.scatter; a.out_C_pad = out.C_pad; a.out_map = f.d_out_map; a.tile_chunk0 = f.d_chunk0;
         a.n_tile_forced = f.n_tile_forced;
         a.res_mode = f.res_mode;
-        if (f.res_mode) {
+        if (f.proj >= 0) {
+            const FConv& q = h->convs[f.proj];
+            const Tensor& X = h->tensors[q.src];
+            a.C_pad = f.C_pad + q.C_pad;
+            a.x2 = X.d; a.x2_chunk0 = f.C_pad / 8; a.x2_plane_mult = X.split ? 4 : 1;
+            a.res_mode = 0;
+        } else if (f.res_mode) {
             const Tensor& r = h->tensors[f.res_tid];
             a.res = r.d; a.res_H = r.H; a.res_W = r.W; a.res_C_pad = r.C_pad; a.res_C = r.C;
             a.res_pad_lo = f.res_pad_lo; a.res_stride = f.res_stride;
@@ -1128,6 +1184,7 @@ void launch_op(fp_handle h, int op_index, const void* d_input, int batch, float*
         fp::launch_stem_pool(h->stem_plan, a, h->d_status, st);
         return;
     }
+    if (op.kind == 0 && h->convs[op.idx].absorbed) return;        // runs inside the layer that adds its result
     if (op.kind == 0 && h->op_chain[op_index] >= 0) {
         const Chain& ch = h->chains[h->op_chain[op_index]];
         if (op_index != ch.first_op) return;       // the run's first operator launches all of it
@@ -1448,7 +1505,7 @@ extern "C" fp_status fp_debug_expire_wait(fp_handle h, void* stream) {
         const Op& op = h->ops[i];
         if (op.kind != 0 || h->op_chain[i] >= 0 || (h->stem_fused && i == 1)) continue;
         const FConv& f = h->convs[op.idx];
-        if (!f.tc.valid || !f.tc.flat || f.tc.blocked_bank || h->tensors[f.src].split || h->tensors[f.out].split) continue;
+        if (!f.tc.valid || !f.tc.flat || f.tc.blocked_bank || h->tensors[f.src].split || h->tensors[f.out].split || f.proj >= 0 || f.absorbed) continue;
         // the first round of the activation producer is left out, so the MMA-issuing thread's wait for that stage runs
         // out after a millisecond (two million cycles), raises the status word and takes every role of the CTA with it
         fp::launch_conv_tc(f.tc, f.args, h->d_status, (cudaStream_t)stream, 0, 2000000LL);
@@ -1527,10 +1584,18 @@ static void fill_op_info(fp_handle h, int i, fp_op_info* o) {
         o->res_mode = f.res_mode; o->relu = f.relu;
         o->flops_per_image = 2.0 * t.H * t.W * (double)f.K_kept * f.C_kept * f.R * f.S;
         double b = (double)s.H * s.W * s.C * e + (double)t.H * t.W * t.C * e;
-        if (f.res_mode == 1) b += (double)t.H * t.W * t.C * e;
+        if (f.res_mode == 1 && f.proj < 0) b += (double)t.H * t.W * t.C * e;
         if (f.res_mode == 2) b += (double)t.H * t.W * h->tensors[f.res_tid].C * e;
         o->bytes_per_image = b;
         o->bytes_fixed = (double)f.K_kept * f.C_kept * f.R * f.S * e + 4.0 * f.K_kept;
+        if (f.proj >= 0) {
+            // the projection shortcut computed inside this layer: its input at this layer's resolution, its filters, its flops
+            const FConv& q = h->convs[f.proj];
+            o->bytes_per_image += (double)t.H * t.W * q.C_kept * e;
+            o->bytes_fixed += (double)q.K_kept * q.C_kept * e + 4.0 * q.K_kept;
+            o->flops_per_image += 2.0 * t.H * t.W * (double)q.K_kept * q.C_kept;
+        }
+        if (f.absorbed) { o->flops_per_image = 0.0; o->bytes_per_image = 0.0; o->bytes_fixed = 0.0; }
     } else if (op.kind == 1) {
         const Pool& p = h->pools[op.idx];
         const Tensor& s = h->tensors[p.src];
@@ -1573,6 +1638,7 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             for (const Chain& ch : h->chains) n -= (int)ch.convs.size() - 1; // a fused run is one
             n -= h->input_fused;
             n -= 2 * h->stem_fused;                                          // conversion, convolution and pooling are one
+            for (const FConv& c : h->convs) n -= c.absorbed;                 // a projection inside the layer that adds it
             *(int32_t*)h_out = n;
             return FP_OK;
         }
@@ -1616,8 +1682,9 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
             const Op& op = h->ops[index];
             const int tid = op.kind == 0 ? h->convs[op.idx].out : op.kind == 1 ? h->pools[op.idx].out : 0;
             const Tensor& t = h->tensors[tid];
-            if (!t.d) return fail(FP_ERR_UNSUPPORTED, "fp_query: operator %d runs inside a fused run of layers and its output never "
-                                  "reaches memory (set keep_outputs to run every layer on its own)", index);
+            if (!t.d) return fail(FP_ERR_UNSUPPORTED, "fp_query: operator %d runs inside another kernel (a fused run of layers, or the layer "
+                                  "that adds this projection shortcut) and its output never reaches memory (set keep_outputs to run "
+                                  "every layer on its own)", index);
             const size_t cnt = (size_t)h->last_batch * t.C * t.H * t.W;
             TRY(need(cnt * sizeof(float)));
             float* d_tmp;
@@ -1666,7 +1733,8 @@ extern "C" fp_status fp_query(fp_handle h, int32_t what, int32_t index, void* h_
                 // first run) adds nothing to the prefix
                 const Op& op = h->ops[i];
                 const bool silent = (op.kind == 0 && h->op_chain[i] >= 0 && h->chains[h->op_chain[i]].first_op != i) ||
-                                    (op.kind == 3 && (h->input_fused || h->stem_fused)) || (h->stem_fused && i == 2);
+                                    (op.kind == 3 && (h->input_fused || h->stem_fused)) || (h->stem_fused && i == 2) ||
+                                    (op.kind == 0 && h->convs[op.idx].absorbed);
                 if (silent) { prefix[i] = i ? prefix[i - 1] : 0.f; continue; }
                 cudaGraph_t g = nullptr;
                 cudaGraphExec_t ge = nullptr;

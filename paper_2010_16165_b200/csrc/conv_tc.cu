@@ -69,6 +69,7 @@ struct TcParams {
     long long bank_tile_bytes;          // streamed filters: bytes of one filter tile's part of the bank (all taps, all chunks)
     int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
     int scatter_bytes;                  // scattered output: channel -> accumulator column map and the tiles' chunk ranges
+    long long plane_in2;                // vectors per channel chunk of the second input tensor (ConvArgs::x2)
     int a_par;                          // activation runs per channel chunk in a stage: 1, or 4 parity images (x_s2d)
     long long par_stride;               // x_s2d: vectors between the parity images of one chunk (N * P2)
     int tap_off[9];                     // x_s2d: start row of each tap's operand within a chunk's part of the stage
@@ -254,6 +255,12 @@ conv_tc_kernel(const TcParams p) {
 
     const uint4* __restrict__ xv = reinterpret_cast<const uint4*>(p.a.x);
     const uint4* __restrict__ wv = reinterpret_cast<const uint4*>(p.a.w);
+    // channel chunk -> its plane: the chunks behind x2_chunk0 are the second input tensor's
+    const uint4* __restrict__ x2v = reinterpret_cast<const uint4*>(p.a.x2);
+    const int chunk2 = p.a.x2_chunk0 > 0 ? p.a.x2_chunk0 : 0x7fffffff;
+    auto chunk_plane = [&](int chunk) -> const uint4* {
+        return chunk < chunk2 ? xv + (long long)chunk * p.plane_in : x2v + (long long)(chunk - chunk2) * p.plane_in2;
+    };
 
     // Programmatic dependent launch: everything above, and the filter-bank copy below, touches
     // nothing the previous kernel in the stream writes, so it may overlap that kernel's tail.  The
@@ -300,7 +307,7 @@ conv_tc_kernel(const TcParams p) {
                     if (lane < na) {
                         const int c = p.a_par == 1 ? lane : lane >> 2, pp = p.a_par == 1 ? 0 : lane & 3;
                         bulk_copy(dst + lane * p.rows_a * 16,
-                                  xv + (long long)(g * p.cg + c) * p.plane_in + (long long)pp * p.par_stride + f0 - p.halo,
+                                  chunk_plane(g * p.cg + c) + (long long)pp * p.par_stride + f0 - p.halo,
                                   (uint32_t)(p.rows_a * 16), fb);
                     } else if (lane >= 16) {
                         // the group's filter block is one contiguous run of the bank: pieces of 16 KB, one per lane
@@ -342,7 +349,7 @@ conv_tc_kernel(const TcParams p) {
                         for (int i = lane; i < p.a_par * cgg; i += 32) {
                             const int c = p.a_par == 1 ? i : i >> 2, pp = p.a_par == 1 ? 0 : i & 3;
                             bulk_copy(dst + i * p.rows_a * 16,
-                                      xv + (long long)(g * p.cg + c) * p.plane_in + (long long)pp * p.par_stride + f0 - p.halo,
+                                      chunk_plane(g * p.cg + c) + (long long)pp * p.par_stride + f0 - p.halo,
                                       (uint32_t)(p.rows_a * 16), fb);
                         }
                     }
@@ -1170,6 +1177,7 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.Wp_in = a.W + 2; p.P2_in = (a.H + 2) * (a.W + 2);
     p.Qp = a.Q + 2; p.P2_out = (a.P + 2) * (a.Q + 2);
     p.plane_in = (long long)a.N * p.P2_in * (a.x_plane_mult > 1 || a.x_s2d ? 4 : 1);
+    p.plane_in2 = (long long)a.N * p.P2_in * (a.x2_plane_mult > 1 ? 4 : 1);
     p.plane_out = (long long)a.N * p.P2_out;
     p.m_total = p.plane_out;
     p.plane_y = p.plane_out;

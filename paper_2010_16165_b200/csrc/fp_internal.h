@@ -64,6 +64,14 @@ struct ConvArgs {
     int y_split;                   // write the output that way (the kernel's own grid stays P x Q)
     int x_plane_mult;              // 0/1: x is a plain tensor; 4: x is a split tensor and this 1x1 layer reads its images
                                    //      0 .. N-1 only (parity 00 = the pixels a 1x1 / stride-2 convolution reads)
+    // A second input tensor along the reduction (tensor-core path, 1x1 / stride-1 layers): channel chunks >= x2_chunk0 of
+    // the C_pad channels come from x2 (chunk - x2_chunk0 of it), a tensor on the same position grid - the input of a
+    // projection shortcut, whose filters are then stacked behind this layer's along the channels (Sec. IV-B: one
+    // convolution [W2' || S_w] instead of two and an add).  x2_plane_mult 4: x2 is parity-split and its images 0..N-1
+    // (parity 00) are the ones read, as for a 1x1 / stride-2 convolution.
+    const void* x2;
+    int x2_chunk0;                 // 0: no second input
+    int x2_plane_mult;
     int x_s2d;                     // x is a split tensor and this is the 3x3 / stride 2 / pad 1 convolution over the tensor
                                    // it was split from: H, W, P, Q are the half resolution, stride is given as 1; the nine
                                    // taps read the parity images at offsets -1 / 0 rows and columns
@@ -113,6 +121,7 @@ void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int
                       cudaStream_t st);
 // 7x7 first convolution as a 3x1 convolution over the packed network input (80 channels)
 void launch_repack_stem(const float* w, int C, const int32_t* row_src, int K_pad, __nv_bfloat16* out, cudaStream_t st);
+void launch_add_bias(const float* a, const float* b, int n, float* out, cudaStream_t st);          // out = a + b (fp32)
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st);
 // 3x3 filters of one layer of a fused run: blob[r][cp/8][48*(kr/16) + 16*s + kr%16][cp%8], the three
 // horizontal taps stacked along the filter (N) axis of the MMA (see chain_tc.cu)

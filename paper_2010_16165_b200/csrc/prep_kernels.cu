@@ -361,6 +361,15 @@ void launch_repack_fc(const float* w, int C, int K, const int32_t* chan_src, int
     repack_fc_kernel<<<blocks_for((size_t)K * C_pad, 256), 256, 0, st>>>(w, C, K, chan_src, C_pad, scale, out);
 }
 
+__global__ void add_bias_kernel(const float* __restrict__ a, const float* __restrict__ b, int n, float* __restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = a[i] + b[i];
+}
+
+void launch_add_bias(const float* a, const float* b, int n, float* out, cudaStream_t st) {
+    add_bias_kernel<<<(n + 127) / 128, 128, 0, st>>>(a, b, n, out);
+}
+
 void launch_pack_bias(const float* b, const int32_t* row_src, int K_pad, float* out, cudaStream_t st) {
     pack_bias_kernel<<<(K_pad + 127) / 128, 128, 0, st>>>(b, row_src, K_pad, out);
 }
