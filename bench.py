@@ -292,6 +292,8 @@ def kernel_report(B, m, peaks, peak_kind, reps):
             s[2] += o.bytes_per_image * w.batch + o.bytes_fixed
             continue
         c = classes["chain_tc_kernel" if o.chain >= 0 else "conv_tc_kernel"]
+        if o.chain < 0 and t <= 0 and o.flops_per_image == 0:
+            continue                   # a projection shortcut computed inside the layer that adds it: no launch of its own
         if o.chain < 0 or o.chain not in seen_runs:
             c[0] += 1
             seen_runs.add(o.chain)
