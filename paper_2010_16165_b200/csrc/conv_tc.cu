@@ -1089,6 +1089,22 @@ int plan_conv_tc(const ConvArgs& a, ConvPlanTC* plan, char* err, size_t err_len)
                     total = t4;
                 }
             }
+            // A 1x1 layer with a long reduction whose bank leaves the two-CTA form three stages of four chunks is bound by
+            // the bytes it has in flight (512 -> 80 at 28x28: 2 x 24 KB per SM, 46.6 us): one CTA with up to eight stages of
+            // eight chunks is taken where that at least doubles them (40.3 us; layers that already have four 16 KB stages
+            // per CTA lose their second CTA for nothing: 256 -> 48 at 56x56 54.8 -> 62.8 us).
+            if (taps == 1 && a_par == 1 && cchunks >= 16) {
+                const unsigned st8 = (unsigned)(8 * plan->rows_a * 16);
+                int stages = fixed + st8 < kSmemMax ? (int)((kSmemMax - fixed) / st8) : 0;
+                if (stages > kMaxStages) stages = kMaxStages;
+                const bool two_ctas = total + 1024u <= kSmemPerSm / 2;
+                const unsigned now = (two_ctas ? 2u : 1u) * (unsigned)plan->a_stages * (unsigned)(plan->cg * plan->rows_a * 16);
+                if (stages >= 4 && (unsigned)stages * st8 >= 2u * now) {
+                    plan->cg = 8; plan->groups = (cchunks + 7) / 8;
+                    plan->a_stages = stages;
+                    total = fixed + (unsigned)stages * st8;
+                }
+            }
             while (total > kSmemMax && plan->cg > 2) {          // parity images: stages four times the size
                 plan->cg -= 2;
                 plan->groups = (cchunks + plan->cg - 1) / plan->cg;
