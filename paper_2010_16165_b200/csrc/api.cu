@@ -81,7 +81,8 @@ struct FConv {
     int32_t* d_out_map = nullptr;   // scatter: output channel -> packed filter row (-1 = no filter kept)
     int32_t* d_chunk0 = nullptr;    // scatter: first output chunk of every filter tile, and the end
     int n_mult = 1;            // 4: a 1x1 layer over a parity-split tensor runs on its 4 N half-size images
-    int proj = -1;             // >= 0: the projection shortcut (index into convs) whose filters are stacked behind this layer's
+    int proj = -1;             // >= 0: the projection shortcut (index into convs) that this layer computes itself
+    int proj_kind = 0;         // 1: filters stacked along the channels (1x1 layer); 2: extra centre-tap K groups (streamed 3x3 layer)
     int absorbed = 0;          // 1: this projection runs inside the layer that adds its result; its operator launches nothing
     void* d_wp_plain = nullptr;     // the packed bank before any re-blocking ([tap][chunk][K_pad][8])
     int K_kept = 0, K_rows = 0, K_pad = 0, C_kept = 0, C_pad = 0;
@@ -840,7 +841,7 @@ fp_status replan(fp_handle h) {
     decide_splits(h, uses);
     for (FConv& f : h->convs) {
         f.n_mult = (h->tensors[f.src].split && split_reader(f) == 'C') ? 4 : 1;
-        f.proj = -1; f.absorbed = 0;
+        f.proj = -1; f.proj_kind = 0; f.absorbed = 0;
     }
     // ... and, where a 3x3 / stride-2 max pooling is the only reader of that convolution and the input is bf16, input
     // conversion, convolution and pooling run as one kernel (decided below, once the filter count is known).
@@ -1020,7 +1021,28 @@ fp_status replan(fp_handle h) {
                 CK(cudaMemcpyAsync((uint8_t*)cat + b1, q.d_wp_plain, b2, cudaMemcpyDeviceToDevice, st));
                 fp::launch_add_bias(f.d_bp, q.d_bp, f.K_pad, bsum, st);
                 f.d_wp = cat; f.d_bp = bsum;
-                f.proj = pj; q.absorbed = 1;
+                f.proj = pj; f.proj_kind = 1; q.absorbed = 1;
+            }
+            // The same for a 3x3 / stride-1 layer with streamed filters (the second layer of a basic block that changes the
+            // resolution): the projection becomes extra K groups with a centre tap only, read from its own packed bank.
+            if (pj < 0 && h->compute == FP_COMPUTE_BF16_TC && !h->keep_outputs && f.res_mode == 1 && f.R == 3 && f.S == 3 &&
+                f.stride == 1 && f.pad == 1 && !f.scatter && !src.split && !out.split && uses[f.res_tid].size() == 1 && f.tc.valid &&
+                f.tc.flat && !f.tc.b_resident && f.tc.blocked_bank == 0 && !(h->stem_packed && f.src == 0)) {
+                const Tensor& rt = h->tensors[f.res_tid];
+                if (rt.producer >= 0 && h->ops[rt.producer].kind == 0) {
+                    const int cand = h->ops[rt.producer].idx;
+                    FConv& q = h->convs[cand];
+                    const Tensor& X = h->tensors[q.src];
+                    if (q.R == 1 && q.S == 1 && q.pad == 0 && q.res_mode == 0 && !q.relu && !q.scatter && !q.compact && q.K == f.K &&
+                        q.K_pad == f.K_pad && q.n_mult == 1 && q.tc.valid && q.d_wp_plain && !(h->stem_packed && q.src == 0) &&
+                        ((q.stride == 1 && !X.split) || (q.stride == 2 && X.split))) {
+                        float* bsum;
+                        TRY(dev_alloc(h, h->pack_buffers, (void**)&bsum, (size_t)f.K_pad * sizeof(float)));
+                        fp::launch_add_bias(f.d_bp, q.d_bp, f.K_pad, bsum, st);
+                        f.d_bp = bsum;
+                        f.proj = cand; f.proj_kind = 2; q.absorbed = 1;
+                    }
+                }
             }
             if (f.tc.valid && f.tc.blocked_bank) {
                 // the streamed form of the kernel reads its bank block by block: one copy per pipeline stage
@@ -1132,8 +1154,9 @@ fp_status replan(fp_handle h) {
         if (f.proj >= 0) {
             const FConv& q = h->convs[f.proj];
             const Tensor& X = h->tensors[q.src];
-            a.C_pad = f.C_pad + q.C_pad;
-            a.x2 = X.d; a.x2_chunk0 = f.C_pad / 8; a.x2_plane_mult = X.split ? 4 : 1;
+            a.x2 = X.d; a.x2_plane_mult = X.split ? 4 : 1;
+            if (f.proj_kind == 1) { a.C_pad = f.C_pad + q.C_pad; a.x2_chunk0 = f.C_pad / 8; }
+            else { a.w2 = q.d_wp_plain; a.x2_C_pad = q.C_pad; }
             a.res_mode = 0;
         } else if (f.res_mode) {
             const Tensor& r = h->tensors[f.res_tid];

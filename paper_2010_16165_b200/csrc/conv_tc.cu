@@ -70,6 +70,7 @@ struct TcParams {
     int lut_bytes;                      // gather: table of plane offsets, 8 entries of 8 bytes per K block
     int scatter_bytes;                  // scattered output: channel -> accumulator column map and the tiles' chunk ranges
     long long plane_in2;                // vectors per channel chunk of the second input tensor (ConvArgs::x2)
+    int cchunks2, groups2;              // streamed 3x3 layer: chunks / extra K groups of the second input (centre tap only)
     int a_par;                          // activation runs per channel chunk in a stage: 1, or 4 parity images (x_s2d)
     long long par_stride;               // x_s2d: vectors between the parity images of one chunk (N * P2)
     int tap_off[9];                     // x_s2d: start row of each tap's operand within a chunk's part of the stage
@@ -335,13 +336,25 @@ conv_tc_kernel(const TcParams p) {
             int round = 0;
             for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
                 const long long f0 = (long long)fdiv((uint32_t)tile, p.div_ntiles) * p.tps * 128;
-                for (int g = 0; g < p.groups; ++g) {
+                for (int g = 0; g < p.groups + p.groups2; ++g) {
                     const bool w = __all_sync(0xffffffffu, mbar_wait(a_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit));
                     if (!w) { ok = false; break; }
                     int cgg = p.cchunks - g * p.cg;
                     if (cgg > p.cg) cgg = p.cg;
                     const uint32_t fb = a_full0 + 8 * stage;
                     const uint32_t dst = a_base + stage * p.a_stage_bytes;
+                    if (g >= p.groups) {
+                        // the K groups of the second input tensor (a projection shortcut's input on this layer's grid)
+                        const int g2 = g - p.groups;
+                        cgg = p.cchunks2 - g2 * p.cg;
+                        if (cgg > p.cg) cgg = p.cg;
+                        if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * p.rows_a * 16));
+                        __syncwarp();
+                        if (lane < cgg)
+                            bulk_copy(dst + lane * p.rows_a * 16, x2v + (long long)(g2 * p.cg + lane) * p.plane_in2 + f0 - p.halo,
+                                      (uint32_t)(p.rows_a * 16), fb);
+                        ++round;
+                    } else
                     if (round++ != p.skip_round) {       // (a diagnostic launch leaves one round out: its stage never fills)
                         if (lane == 0) mbar_expect_tx(fb, (uint32_t)(p.a_par * cgg * p.rows_a * 16));
                         __syncwarp();
@@ -490,6 +503,24 @@ conv_tc_kernel(const TcParams p) {
                         }
                         if (!ok) break;
                         umma_commit(a_empty0 + 8 * a_stage);     // releases the stage once these MMAs have read it
+                        if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
+                    }
+                    // streamed 3x3 layer with a projection shortcut taken in: the K groups of the second input, centre tap only
+                    for (int g2 = 0; MODE == MODE_FLAT_STREAM && g2 < p.groups2 && ok; ++g2) {
+                        if (!mbar_wait(a_full0 + 8 * a_stage, a_phase, abort_flag, wait_limit)) { ok = false; break; }
+                        if (!mbar_wait(b_full0 + 8 * b_stage, b_phase, abort_flag, wait_limit)) { ok = false; break; }
+                        tc_fence_after();
+                        int cgg = p.cchunks2 - g2 * p.cg;
+                        if (cgg > p.cg) cgg = p.cg;
+                        const uint32_t a_row = (((a_base + a_stage * p.a_stage_bytes) >> 4) + (uint32_t)p.halo + (uint32_t)(issuer * 128)) |
+                                               ((uint32_t)p.rows_a << 16);
+                        const uint32_t b_lo = ((b_base + b_stage * p.b_stage_bytes) >> 4) | ((uint32_t)p.n_tile << 16);
+                        issue_ksteps(cgg >> 1, d_tmem + (uint32_t)(issuer * p.n_tile), a_row, b_lo, 2u * (uint32_t)p.rows_a,
+                                     2u * (uint32_t)p.n_tile, idesc, accumulate);
+                        accumulate = 1;
+                        umma_commit(b_empty0 + 8 * b_stage);
+                        if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_phase ^= 1; }
+                        umma_commit(a_empty0 + 8 * a_stage);
                         if (++a_stage == (uint32_t)p.a_stages) { a_stage = 0; a_phase ^= 1; }
                     }
                 } else {
@@ -837,6 +868,24 @@ conv_tc_kernel(const TcParams p) {
                         }
                         if (++stage == (uint32_t)p.b_stages) { stage = 0; phase ^= 1; }
                     }
+                }
+                // the second input's K groups: one block each, the centre tap's filters from the projection's own bank
+                for (int g2 = 0; g2 < p.groups2 && ok; ++g2) {
+                    int cgg = p.cchunks2 - g2 * p.cg;
+                    if (cgg > p.cg) cgg = p.cg;
+                    const bool w = __all_sync(0xffffffffu, mbar_wait(b_empty0 + 8 * stage, phase ^ 1, abort_flag, wait_limit));
+                    if (!w) { ok = false; break; }
+                    const uint32_t fb = b_full0 + 8 * stage;
+                    const uint32_t dst = b_base + stage * p.b_stage_bytes;
+                    if (lane == 0) mbar_expect_tx(fb, (uint32_t)(cgg * nrows * 16));
+                    __syncwarp();
+                    const uint4* src = reinterpret_cast<const uint4*>(p.a.w2) + (long long)(g2 * p.cg) * p.a.K_pad + nt * p.n_tile;
+                    if (whole) {
+                        if (lane == 0) bulk_copy(dst, src, (uint32_t)(cgg * nrows * 16), fb);
+                    } else if (lane < cgg) {
+                        bulk_copy(dst + lane * p.n_tile * 16, src + (long long)lane * p.a.K_pad, (uint32_t)(nrows * 16), fb);
+                    }
+                    if (++stage == (uint32_t)p.b_stages) { stage = 0; phase ^= 1; }
                 }
             }
             if (!ok && lane == 0) raise(ctrl, p.status, 4);
@@ -1194,6 +1243,8 @@ void launch_conv_tc(const ConvPlanTC& plan, const ConvArgs& a, int* d_status, cu
     p.Qp = a.Q + 2; p.P2_out = (a.P + 2) * (a.Q + 2);
     p.plane_in = (long long)a.N * p.P2_in * (a.x_plane_mult > 1 || a.x_s2d ? 4 : 1);
     p.plane_in2 = (long long)a.N * p.P2_in * (a.x2_plane_mult > 1 ? 4 : 1);
+    p.cchunks2 = a.x2_C_pad / 8;
+    p.groups2 = a.x2_C_pad > 0 ? (p.cchunks2 + plan.cg - 1) / plan.cg : 0;
     p.plane_out = (long long)a.N * p.P2_out;
     p.m_total = p.plane_out;
     p.plane_y = p.plane_out;

@@ -70,8 +70,12 @@ struct ConvArgs {
     // convolution [W2' || S_w] instead of two and an add).  x2_plane_mult 4: x2 is parity-split and its images 0..N-1
     // (parity 00) are the ones read, as for a 1x1 / stride-2 convolution.
     const void* x2;
-    int x2_chunk0;                 // 0: no second input
+    int x2_chunk0;                 // 0: no second input stacked along the channels
     int x2_plane_mult;
+    // The same for a 3x3 / stride-1 layer with streamed filters: the projection enters as extra K groups that have a
+    // centre tap only - x2_C_pad channels of x2, filters w2 = [chunk][K_pad][8] (the projection's own packed bank).
+    const void* w2;
+    int x2_C_pad;                  // 0: none
     int x_s2d;                     // x is a split tensor and this is the 3x3 / stride 2 / pad 1 convolution over the tensor
                                    // it was split from: H, W, P, Q are the half resolution, stride is given as 1; the nine
                                    // taps read the parity images at offsets -1 / 0 rows and columns
